@@ -1,0 +1,379 @@
+"""fp64 CPU oracle of the VVS target-model verification step.  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this module;
+the CUDA library never does, and the two share no code.  Everything is written out plainly
+in numpy float64 (a matmul / cumsum / exp from numpy may serve as a step), in the order the
+paper states the method, with no blocking, fusion or reordering.
+
+Naming.  The paper (Sec. 2, "Speculative Decoding") calls the draft distribution p and the
+target distribution q.  This code uses the opposite, more common convention of the task
+statement: **p = target, q = draft**.
+
+What the paper fixes (Sec. 2; Sec. 4.1, 4.3; Algorithm 2 lines 9-11; Supp. "Memory
+Overhead") and what it leaves open is listed per function.  Readings chosen where the paper
+is silent or garbled:
+
+* residual distribution: the paper prints max{0, p - q} in *its* naming (draft - target),
+  un-normalised.  Used here: norm(max(0, target - draft)), the only sign for which strict
+  verification is lossless, which the paper claims (Sec. 6 "lossless").
+* relaxed acceptance (Sec. 2, LANTERN rule, garbled in print): the neighbourhood of a drafted
+  token x is the first k entries of its CSR row, ordered by latent distance with x itself
+  first; the accepted set A is {x} plus the longest distance-ordered prefix of the other
+  entries whose cumulative target mass (not counting p(x)) stays <= delta; acceptance
+  probability min(1, sum_{x' in A} p(x') / q(x)).  **parity unpinned** by the paper beyond
+  "k = 1 or delta = 0 is strict" and the bounds p(x) <= P_A <= p(x) + delta.
+* residual after a relaxed rejection: the plain norm(max(0, p - q)).  **parity unpinned**.
+* classifier-free guidance is not in the paper: l = l_u + s (l_c - l_u) on logits before the
+  softmax; rows ordered [cond_0..cond_{B-1}, uncond_0..uncond_{B-1}].
+* architecture (not in the paper): pre-norm RMSNorm (eps inside the square root, learned
+  scale), SwiGLU MLP, no biases, untied LM head, attention scale 1/sqrt(head_dim).
+* RoPE: consecutive-pair (even, odd) convention; 1-D on the absolute position, or 2-D over a
+  w-wide token grid where prefix positions get no rotation, the first half of the head
+  dimension rotates by grid row and the second half by grid column.  **parity unpinned**
+  (convention only; its rotation properties are pinned).
+* feature cache (Sec. 4.3): feature = final-norm output (LM-head input) of each committed
+  block row, addressed by (row, absolute position) in a ring of `cap` slots; fetch(gamma, s)
+  returns positions newest-s-gamma+1 .. newest-s.  **parity unpinned** for the choice of
+  post-norm features and ring addressing; the index arithmetic itself is pinned.
+* decisions are taken on the float32 target probabilities the step emits: ratios, pooled
+  masses and the sampling CDF accumulate in float64 in ascending / distance order.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+ROPE_NONE, ROPE_1D, ROPE_2D_GRID = 0, 1, 2
+MODE_STRICT, MODE_RELAXED = 0, 1
+
+
+# ---------------------------------------------------------------------------------------
+# storage widening
+
+
+def widen(a: np.ndarray) -> np.ndarray:
+    """Exact widening of stored bits to float64: uint16 = bfloat16 bit patterns, else float."""
+    a = np.asarray(a)
+    if a.dtype == np.uint16:
+        return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    return a.astype(np.float64)
+
+
+# ---------------------------------------------------------------------------------------
+# transformer pieces (architecture per the workload description; the paper only says the
+# target model M_T maps the candidate block to logits and hidden states, Alg. 2 line 9)
+
+
+def rmsnorm(x: np.ndarray, scale: np.ndarray, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) * scale over the last axis."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * scale
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+def rope_angles(pos: int, head_dim: int, mode: int, base: float, grid_w: int = 0,
+                n_prefix: int = 0) -> np.ndarray:
+    """Rotation angle of each of the head_dim/2 consecutive pairs at absolute position pos."""
+    half = head_dim // 2
+    if mode == ROPE_NONE:
+        return np.zeros(half)
+    if mode == ROPE_1D:
+        i = np.arange(half, dtype=np.float64)
+        return pos * base ** (-2.0 * i / head_dim)
+    if mode == ROPE_2D_GRID:
+        if pos < n_prefix:
+            return np.zeros(half)
+        n = pos - n_prefix
+        row, col = n // grid_w, n % grid_w
+        quarter = half // 2
+        j = np.arange(quarter, dtype=np.float64)
+        freq = base ** (-2.0 * j / half)
+        return np.concatenate([row * freq, col * freq])
+    raise ValueError("rope mode")
+
+
+def rope(x: np.ndarray, angles: np.ndarray) -> np.ndarray:
+    """Rotate consecutive pairs (x[2i], x[2i+1]) of the last axis by angles[i]."""
+    c, s = np.cos(angles), np.sin(angles)
+    xe, xo = x[..., 0::2], x[..., 1::2]
+    y = np.empty_like(x)
+    y[..., 0::2] = xe * c - xo * s
+    y[..., 1::2] = xe * s + xo * c
+    return y
+
+
+def softmax(z: np.ndarray) -> np.ndarray:
+    e = np.exp(z - np.max(z, axis=-1, keepdims=True))
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def attention_block_vs_cache(q: np.ndarray, kc: np.ndarray, vc: np.ndarray, fill: int) -> np.ndarray:
+    """Parallel verification attention (Sec. 2: the candidates are appended to the input and
+    scored in one pass): block row t sees cache slots [0, fill) and block rows 0..t, which
+    already sit in slots fill..fill+t of kc/vc.
+
+    q [T, H, hd]; kc, vc [H, S, hd].  Returns [T, H, hd]."""
+    t_len, n_heads, hd = q.shape
+    out = np.zeros_like(q)
+    for h in range(n_heads):
+        for t in range(t_len):
+            n_keys = fill + t + 1
+            s = kc[h, :n_keys] @ q[t, h] / np.sqrt(hd)
+            w = softmax(s)
+            out[t, h] = w @ vc[h, :n_keys]
+    return out
+
+
+def target_forward(ms, weights: dict, tokens: np.ndarray, kc: np.ndarray, vc: np.ndarray,
+                   fill: int) -> np.ndarray:
+    """M_T over one sequence's block (Alg. 2 line 9): returns the features h (final-norm
+    output, i.e. the hidden state before the output head, Sec. 3 "Stale Feature Reusability")
+    for every block row, and appends the block's keys/values to the float64 caches
+    kc, vc [n_layers, H, S, hd] in slots fill..fill+T-1 (the KV entries a later step needs,
+    Sec. 4.1)."""
+    d, n_heads, hd = ms.d_model, ms.n_heads, ms.head_dim
+    t_len = len(tokens)
+    x = widen(weights["tok_emb"][np.asarray(tokens)])
+    ang = [rope_angles(fill + t, hd, ms.rope_mode, ms.rope_base, ms.rope_grid_w, ms.n_prefix)
+           for t in range(t_len)]
+    for l in range(ms.n_layers):
+        w = weights["layers"][l]
+        a = rmsnorm(x, widen(w["norm1"]), ms.rms_eps)
+        qkv = a @ widen(w["w_qkv"]).T
+        q = qkv[:, 0 * d:1 * d].reshape(t_len, n_heads, hd)
+        k = qkv[:, 1 * d:2 * d].reshape(t_len, n_heads, hd)
+        v = qkv[:, 2 * d:3 * d].reshape(t_len, n_heads, hd)
+        for t in range(t_len):
+            q[t] = rope(q[t], ang[t])
+            kc[l, :, fill + t, :] = rope(k[t], ang[t])
+            vc[l, :, fill + t, :] = v[t]
+        o = attention_block_vs_cache(q, kc[l], vc[l], fill).reshape(t_len, d)
+        x = x + o @ widen(w["w_o"]).T
+        m = rmsnorm(x, widen(w["norm2"]), ms.rms_eps)
+        g = m @ widen(w["w_gate"]).T
+        u = m @ widen(w["w_up"]).T
+        x = x + (silu(g) * u) @ widen(w["w_down"]).T
+    return rmsnorm(x, widen(weights["norm_f"]), ms.rms_eps)
+
+
+def lm_head_logits(ms, weights: dict, hidden: np.ndarray) -> np.ndarray:
+    """Logits over the image codebook only: rows vocab_offset .. vocab_offset+V-1 of the head."""
+    w = widen(weights["w_lm"][ms.vocab_offset:ms.vocab_offset + ms.vocab])
+    return hidden @ w.T
+
+
+def guided_logits(l_cond: np.ndarray, l_uncond, cfg_scale: float) -> np.ndarray:
+    """Classifier-free guidance on logits: l_u + s (l_c - l_u); without an uncond row, l_c."""
+    return l_cond if l_uncond is None else l_uncond + cfg_scale * (l_cond - l_uncond)
+
+
+def guided_probs(l_cond: np.ndarray, l_uncond, cfg_scale: float, temperature: float) -> np.ndarray:
+    """Guided logits, then the temperature softmax (the paper samples at temperature 1)."""
+    return softmax(guided_logits(l_cond, l_uncond, cfg_scale) / temperature)
+
+
+# ---------------------------------------------------------------------------------------
+# decision stage (Sec. 2): acceptance, accepted prefix, residual / bonus sample
+
+
+def pooled_mass(p_row: np.ndarray, x: int, row_ptr: np.ndarray, col: np.ndarray, k: int,
+                delta: float) -> float:
+    """Relaxed (LANTERN) numerator: p(x) plus the target mass of the longest distance-ordered
+    prefix of x's other neighbours whose running sum stays <= delta."""
+    nb = col[row_ptr[x]:row_ptr[x + 1]][:k]
+    assert len(nb) == 0 or nb[0] == x, "neighbour rows must list the token itself first"
+    cum = 0.0
+    for xn in nb[1:]:
+        pn = float(p_row[xn])
+        if cum + pn > delta:
+            break
+        cum += pn
+    return float(p_row[x]) + cum
+
+
+def acceptance_ratio(p_mass: float, q_x: float) -> float:
+    """min(1, P / q(x)); a draft with q(x) = 0 is accepted iff P > 0."""
+    if q_x > 0.0:
+        return min(1.0, p_mass / q_x)
+    return 1.0 if p_mass > 0.0 else 0.0
+
+
+def inverse_cdf(r: np.ndarray, u: float):
+    """Smallest index j with sum_{i<=j} r_i > u * sum(r), accumulating in float64 in ascending
+    index; if rounding leaves none, the last index with r_j > 0.  Returns (j, margin) where
+    margin is the distance of u*sum(r) to the nearest edge of bin j, as a fraction of sum(r)."""
+    cdf = np.cumsum(r.astype(np.float64))
+    total = cdf[-1]
+    t = float(u) * total
+    above = np.nonzero(cdf > t)[0]
+    j = int(above[0]) if len(above) else int(np.nonzero(r > 0)[0][-1])
+    lo = cdf[j - 1] if j > 0 else 0.0
+    margin = min(abs(t - lo), abs(cdf[j] - t)) / total
+    return j, margin
+
+
+def decide(p32: np.ndarray, drafts: np.ndarray, n_draft: int, n_forced: int, q32: np.ndarray,
+           u32: np.ndarray, mode: int = MODE_STRICT, row_ptr=None, col=None, k: int = 1,
+           delta: float = float("inf")) -> dict:
+    """Sequential verification of one image's drafts against float32 target rows p32 [T, V].
+
+    Draft i (token drafts[i], draft row q32[i]) is judged against p32[n_forced-1+i] with
+    uniform u32[i]; verification stops at the first rejection.  The next token comes from
+    norm(max(0, p - q)) of the rejecting position, or from the following target row if every
+    draft was accepted (-1 if p32 has no such row); it uses the last uniform u32[-1]."""
+    p32 = np.asarray(p32, dtype=np.float32)
+    q32 = np.asarray(q32, dtype=np.float32)
+    k_max = len(u32) - 1
+    mask = np.zeros(k_max, dtype=np.uint8)
+    margins = np.full(k_max + 1, np.inf)
+    ratios = np.full(k_max, np.nan)
+    n = 0
+    for i in range(n_draft):
+        x = int(drafts[i])
+        row = p32[n_forced - 1 + i]
+        if mode == MODE_RELAXED:
+            mass = pooled_mass(row, x, row_ptr, col, k, delta)
+        else:
+            mass = float(row[x])
+        ratio = acceptance_ratio(mass, float(q32[i, x]))
+        ratios[i] = ratio
+        margins[i] = abs(float(u32[i]) - ratio)
+        if not float(u32[i]) < ratio:
+            break
+        mask[i] = 1
+        n += 1
+    src = n_forced - 1 + n
+    if src >= p32.shape[0]:
+        token = -1
+    else:
+        row = p32[src]
+        if n < n_draft:
+            r = np.maximum(np.float32(0.0), row - q32[n])       # IEEE float32 subtraction
+            if not np.any(r > 0):
+                r = row                                          # p == q numerically
+        else:
+            r = row
+        token, margins[k_max] = inverse_cdf(r, float(u32[k_max]))
+    return {"accept_len": n, "accept_mask": mask, "next_token": int(token),
+            "margins": margins, "ratios": ratios}
+
+
+# ---------------------------------------------------------------------------------------
+# the whole step (Alg. 2 lines 9-10)
+
+
+def epilogue(ms, weights: dict, hidden: np.ndarray, drafts, n_draft, n_forced: int, draft_probs,
+             uniforms, n_cfg: int, cfg_scale: float, temperature: float = 1.0, mode: int = MODE_STRICT,
+             row_ptr=None, col=None, k: int = 1, delta: float = float("inf")) -> dict:
+    """LM head + guidance + softmax + decisions on given features.
+
+    hidden [R, T, d] with R = n_cfg*B rows ordered cond images then uncond images (n_cfg = 2
+    with guidance, else 1); drafts int [B, K]; draft_probs float32 [B, K, V]; uniforms
+    [B, K+1]."""
+    n_images = hidden.shape[0] // n_cfg
+    t_len = hidden.shape[1]
+    probs = np.zeros((n_images, t_len, ms.vocab))
+    logits = np.zeros((n_images, t_len, ms.vocab))
+    out = {"accept_len": np.zeros(n_images, np.int32), "next_token": np.zeros(n_images, np.int32),
+           "accept_mask": np.zeros((n_images, uniforms.shape[1] - 1), np.uint8),
+           "margins": np.zeros((n_images, uniforms.shape[1])),
+           "ratios": np.zeros((n_images, uniforms.shape[1] - 1))}
+    for b in range(n_images):
+        l_c = lm_head_logits(ms, weights, widen(hidden[b]))
+        l_u = lm_head_logits(ms, weights, widen(hidden[n_images + b])) if n_cfg == 2 else None
+        logits[b] = guided_logits(l_c, l_u, cfg_scale)
+        probs[b] = guided_probs(l_c, l_u, cfg_scale, temperature)
+        dec = decide(probs[b].astype(np.float32), drafts[b], int(n_draft[b]), n_forced,
+                     draft_probs[b], uniforms[b], mode, row_ptr, col, k, delta)
+        for key in ("accept_len", "next_token", "accept_mask", "margins", "ratios"):
+            out[key][b] = dec[key]
+    out["target_probs"] = probs
+    out["logits"] = logits
+    return out
+
+
+def verify(ms, weights: dict, block: np.ndarray, n_forced: int, n_draft: np.ndarray,
+           kv_k: np.ndarray, kv_v: np.ndarray, cache_len: np.ndarray, draft_probs: np.ndarray,
+           uniforms: np.ndarray, n_cfg: int, cfg_scale: float, temperature: float = 1.0,
+           mode: int = MODE_STRICT, row_ptr=None, col=None, k: int = 1,
+           delta: float = float("inf")) -> dict:
+    """One verification step for B images.
+
+    block int [B, T] = n_forced committed tokens whose K/V is not yet cached, then K drafts,
+    as embedding-table ids (a draft's codebook index is id - vocab_offset; next_token is
+    returned as an embedding-table id as well).
+    kv_k, kv_v stored caches [n_layers, R, H, S, hd] (read, not modified); cache_len int [R].
+    Returns accept_len, next_token, new_len, accept_mask, target_probs [B,T,V] (float64),
+    hidden [R,T,d] (float64), the new cache rows k_new/v_new [n_layers, R, H, T, hd] and the
+    decision margins."""
+    n_images, t_len = block.shape
+    n_rows = n_images * n_cfg
+    hidden = np.zeros((n_rows, t_len, ms.d_model))
+    k_new = np.zeros((ms.n_layers, n_rows, ms.n_heads, t_len, ms.head_dim))
+    v_new = np.zeros_like(k_new)
+    for r in range(n_rows):
+        b = r % n_images
+        fill = int(cache_len[r])
+        kc = widen(kv_k[:, r])
+        vc = widen(kv_v[:, r])
+        hidden[r] = target_forward(ms, weights, block[b], kc, vc, fill)
+        k_new[:, r] = kc[:, :, fill:fill + t_len]
+        v_new[:, r] = vc[:, :, fill:fill + t_len]
+    drafts = block[:, n_forced:] - ms.vocab_offset            # embedding id -> codebook index
+    out = epilogue(ms, weights, hidden, drafts, n_draft, n_forced, draft_probs, uniforms,
+                   n_cfg, cfg_scale, temperature, mode, row_ptr, col, k, delta)
+    out["next_token"] = np.where(out["next_token"] >= 0, out["next_token"] + ms.vocab_offset,
+                                 -1).astype(np.int32)
+    out["hidden"] = hidden
+    out["k_new"], out["v_new"] = k_new, v_new
+    out["new_len"] = np.array([int(cache_len[r]) + n_forced + int(out["accept_len"][r % n_images])
+                               for r in range(n_rows)], dtype=np.int32)
+    return out
+
+
+# ---------------------------------------------------------------------------------------
+# token-level feature cache (Sec. 4.3; Alg. 2 lines 5 and 11; Supp. "Memory Overhead")
+
+
+class FeatureCache:
+    """Per-row ring of the most recent token-level features, addressed by absolute position."""
+
+    def __init__(self, n_rows: int, cap: int, d: int):
+        self.cap = cap
+        self.feat = np.zeros((n_rows, cap, d))
+        self.fpos = np.full((n_rows, cap), -1, dtype=np.int32)
+        self.newest = np.full(n_rows, -1, dtype=np.int32)
+
+    def store(self, hidden: np.ndarray, base_pos: np.ndarray, n_store: np.ndarray) -> None:
+        """UpdateCache(h_t): row r keeps hidden[r, t] for t < n_store[r] at absolute position
+        base_pos[r] + t (slot = position mod cap; a re-stored position is overwritten, which
+        is how post verification writes features back to their positions, Sec. 4.1)."""
+        for r in range(hidden.shape[0]):
+            for t in range(int(n_store[r])):
+                pos = int(base_pos[r]) + t
+                self.feat[r, pos % self.cap] = hidden[r, t]
+                self.fpos[r, pos % self.cap] = pos
+            if n_store[r] > 0:
+                self.newest[r] = max(self.newest[r], int(base_pos[r]) + int(n_store[r]) - 1)
+
+    def fetch(self, skip_mask: np.ndarray, gamma: np.ndarray, staleness: int, gamma_max: int):
+        """Retrieve(C, a): for rows whose image is skip-masked, the gamma[r] most recent
+        features ending `staleness` positions before the newest one, oldest first.  A position
+        that was never stored or has been overwritten yields out_pos = -1 and a zero row.
+        Rows not masked, and entries j >= gamma[r], are left zero / -1 here."""
+        n_rows, _, d = self.feat.shape
+        n_images = len(skip_mask)
+        out = np.zeros((n_rows, gamma_max, d))
+        out_pos = np.full((n_rows, gamma_max), -1, dtype=np.int32)
+        for r in range(n_rows):
+            if not skip_mask[r % n_images]:
+                continue
+            g = int(gamma[r])
+            for j in range(g):
+                pos = int(self.newest[r]) - staleness - g + 1 + j
+                if pos >= 0 and self.newest[r] >= 0 and self.fpos[r, pos % self.cap] == pos:
+                    out[r, j] = self.feat[r, pos % self.cap]
+                    out_pos[r, j] = pos
+        return out, out_pos
