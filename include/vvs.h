@@ -1,0 +1,248 @@
+/*
+ * vvs.h -- C ABI of the B200 (sm_100a) target-model verification step of VVS speculative
+ * decoding for visual autoregressive models.
+ *
+ * One call of vvs_verify is lines 9-10 of the paper's Algorithm 2 ("VVS with Partial
+ * Verification Skipping"): the target model M_T scores the candidate block in one parallel
+ * pass against its KV cache (Sec. 2, "Speculative Decoding"), and Verify() applies the
+ * sequential acceptance test, stops at the first rejection and resamples (Sec. 2).
+ * vvs_feature_cache_store / _fetch are UpdateCache() (Alg. 2 line 11) and Retrieve()
+ * (Alg. 2 line 5) of the token-level feature cache (Sec. 4.3).
+ *
+ * Naming: p = TARGET distribution, q = DRAFT distribution (the paper's Sec. 2 uses the
+ * opposite letters).
+ *
+ * General rules
+ *   - Every function returns VVS_OK (0) or a negative vvs_status.  Host-side argument errors
+ *     are returned before anything is launched.  No exceptions, no global state.
+ *   - "device" pointers are CUDA device memory of the context's GPU, owned by the caller,
+ *     16-byte aligned unless stated otherwise.  "host" pointers are ordinary host memory.
+ *     The library never frees caller memory and keeps no reference to host arrays after a
+ *     call returns (the per-layer pointer table is copied).
+ *   - All work is enqueued on the CUDA stream passed to the call (a cudaStream_t cast to
+ *     void*; NULL = the default stream) and is asynchronous.  A context holds scratch memory
+ *     used by every call on it: calls on one context must be stream-ordered, one context per
+ *     concurrently used stream.
+ *   - Conditions only the GPU can see (token id out of range, cache overflow computed from
+ *     device-resident lengths, a bounded wait that ran out) set bits in a device status word,
+ *     read with vvs_device_status; the offending access is skipped, never executed.
+ *   - Storage type T is float for VVS_DTYPE_FP32 contexts and bfloat16 for VVS_DTYPE_BF16.
+ *     Accumulation, softmax and normalisation statistics are float32; decisions (acceptance
+ *     ratios, pooled masses, the sampling CDF) accumulate in float64.
+ */
+#ifndef VVS_H_
+#define VVS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum vvs_status {
+  VVS_OK = 0,
+  VVS_ERR_INVALID_ARG = -1,    /* NULL where a pointer is required, bad enum, bad scalar */
+  VVS_ERR_SHAPE = -2,          /* sizes inconsistent with the model description / limits */
+  VVS_ERR_ALIGN = -3,          /* a device pointer is not 16-byte aligned */
+  VVS_ERR_CAPACITY = -4,       /* cache fill + block length exceeds s_max */
+  VVS_ERR_NOT_BOUND = -5,      /* weights (or the neighbour table, in relaxed mode) not bound */
+  VVS_ERR_CUDA = -6,           /* a CUDA runtime call failed */
+  VVS_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait gave up */
+  VVS_ERR_DEVICE_BOUNDS = -8,  /* a device-side index check failed; the access was skipped */
+  VVS_ERR_NOMEM = -9           /* workspace allocation failed */
+} vvs_status;
+
+enum { VVS_DTYPE_FP32 = 0, VVS_DTYPE_BF16 = 1 };
+enum { VVS_ROPE_NONE = 0, VVS_ROPE_1D = 1, VVS_ROPE_2D_GRID = 2 };
+enum { VVS_MODE_STRICT = 0, VVS_MODE_RELAXED = 1 };
+
+/* Bits of the device status word (vvs_device_status). */
+enum {
+  VVS_DEV_BAD_TOKEN = 1,      /* block token outside the embedding table / draft outside codebook */
+  VVS_DEV_CACHE_OVERFLOW = 2, /* cache_len[r] + T > s_max, or cache_len < 0: row skipped */
+  VVS_DEV_BAD_NEIGHBOUR = 4,  /* CSR column outside [0, V) or row_ptr not monotone */
+  VVS_DEV_TIMEOUT = 8,        /* a bounded wait on a barrier ran out */
+  VVS_DEV_FCACHE_MISS = 16,   /* feature-cache fetch asked for a position not in the ring */
+  VVS_DEV_BAD_ARG = 32        /* n_draft / gamma / n_store outside its documented range */
+};
+
+typedef struct vvs_ctx vvs_ctx;
+
+/* Decoder-only transformer of the target model.  The paper treats M_T as given (LlamaGen-XL,
+ * Lumina-mGPT); the architecture is the one those models share: pre-norm RMSNorm with a
+ * learned scale, rotary position embedding, multi-head attention scaled by 1/sqrt(head_dim),
+ * SwiGLU MLP, no biases, untied output head.  d_model must equal n_heads * head_dim. */
+typedef struct vvs_model_desc {
+  int32_t n_layers;
+  int32_t d_model;
+  int32_t n_heads;
+  int32_t head_dim;      /* 64 or 128 */
+  int32_t d_ff;          /* SwiGLU inner width */
+  int32_t vocab;         /* V: size of the image codebook = number of logits per position */
+  int32_t vocab_offset;  /* first row of the image codebook inside w_lm and the id space */
+  int32_t lm_rows;       /* rows of w_lm (>= vocab_offset + vocab) */
+  int32_t tok_rows;      /* rows of tok_emb */
+  int32_t s_max;         /* KV-cache capacity (positions) per sequence */
+  int32_t rope_mode;     /* VVS_ROPE_*; pairs are (2i, 2i+1); 1D: angle = pos * base^(-2i/hd);
+                            2D_GRID: positions < n_prefix unrotated, image token n sits at grid
+                            (n / rope_grid_w, n % rope_grid_w); pairs of the first head half
+                            rotate by row, of the second half by column, with
+                            angle = coord * base^(-2j/(hd/2)), j the pair index in its half */
+  int32_t rope_grid_w;
+  int32_t n_prefix;
+  int32_t dtype;         /* VVS_DTYPE_*: type of weights, KV cache, hidden states */
+  int32_t max_rows;      /* largest R = n_images * n_cfg a call may use */
+  int32_t max_block;     /* largest T = n_forced + n_draft_max a call may use (<= 32) */
+  int32_t max_nbr_k;     /* largest neighbour count k in relaxed mode (>= 1) */
+  float rms_eps;
+  float rope_base;
+} vvs_model_desc;
+
+/* Per-layer weights, device, type T.  Projection matrices are [out_features, in_features]
+ * row-major: w_qkv [3*d_model, d_model] (q rows, then k rows, then v rows; head h owns rows
+ * h*head_dim..), w_o [d_model, d_model], w_gate and w_up [d_ff, d_model],
+ * w_down [d_model, d_ff], norm1 / norm2 [d_model]. */
+typedef struct vvs_layer_weights {
+  const void* w_qkv;
+  const void* w_o;
+  const void* w_gate;
+  const void* w_up;
+  const void* w_down;
+  const void* norm1;
+  const void* norm2;
+} vvs_layer_weights;
+
+typedef struct vvs_weights {
+  const void* tok_emb;             /* device T [tok_rows, d_model] */
+  const void* norm_f;              /* device T [d_model] */
+  const void* w_lm;                /* device T [lm_rows, d_model]; only rows
+                                      vocab_offset .. vocab_offset+vocab-1 are read */
+  const vvs_layer_weights* layers; /* HOST array [n_layers] of device pointers */
+} vvs_weights;
+
+/* Create a context on the current CUDA device and allocate its scratch memory (sized from
+ * max_rows, max_block, max_nbr_k; see vvs_workspace_bytes).  *out is NULL on failure. */
+int vvs_create(const vvs_model_desc* desc, vvs_ctx** out);
+int vvs_destroy(vvs_ctx* ctx);
+/* Scratch bytes vvs_create will allocate for this description (host computation only). */
+int vvs_workspace_bytes(const vvs_model_desc* desc, size_t* out_bytes);
+
+/* Bind caller-owned weights.  Checks non-NULL and 16-byte alignment (VVS_ERR_ALIGN). */
+int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w);
+
+/* Bind the latent-space neighbour table used by relaxed acceptance (Sec. 2, LANTERN rule):
+ * CSR over codebook indices, device int32.  row_ptr [vocab+1]; the neighbours of code x are
+ * col[row_ptr[x] .. row_ptr[x+1]) in ascending latent distance with x ITSELF FIRST (entry 0 is
+ * taken to be x and is not read).  nnz = row_ptr[vocab]. */
+int vvs_bind_neighbors(vvs_ctx* ctx, const int32_t* row_ptr, const int32_t* col, int64_t nnz);
+
+/* Inputs of one verification step.  B = n_images, C = n_cfg, R = B*C sequences ordered
+ * [cond_0 .. cond_{B-1}, uncond_0 .. uncond_{B-1}], F = n_forced >= 1, K = n_draft_max,
+ * T = F + K block rows per sequence. */
+typedef struct vvs_verify_args {
+  int32_t n_images;
+  int32_t n_cfg;          /* 1: no guidance; 2: logits l = l_u + cfg_scale * (l_c - l_u) */
+  int32_t n_forced;       /* committed tokens whose K/V is not cached yet (the last accepted
+                             token; with post verification, Sec. 4.1, also the unverified ones) */
+  int32_t n_draft_max;
+  const int32_t* block;   /* device [B, T] embedding-table ids: F forced tokens, then K drafts.
+                             Drafts must lie in [vocab_offset, vocab_offset + vocab). cond and
+                             uncond sequences of an image carry the same block */
+  const int32_t* n_draft; /* device [B], drafts actually proposed per image (0..K); NULL = K */
+  void* kv_k;             /* device T [n_layers][kv_rows][n_heads][s_max][head_dim], keys after */
+  void* kv_v;             /*   RoPE / values.  Slots cache_len[r] .. cache_len[r]+T-1 of every
+                               layer are WRITTEN by the call (Sec. 4.1: restores KV entries) */
+  int32_t kv_rows;        /* sequence dimension of the cache allocation (>= R) */
+  const int32_t* cache_len;      /* device [R] fill level L_r (positions already cached) */
+  const int32_t* cache_len_host; /* optional HOST copy [R]: enables the VVS_ERR_CAPACITY check
+                                    before launch; NULL = checked on the device only */
+  const float* draft_probs; /* device [B, K, V] drafter distributions q_i over the codebook */
+  const float* uniforms;    /* device [B, K+1] in (0,1): column i < K judges draft i, column K
+                               drives the single residual / bonus sample */
+  float cfg_scale;
+  float temperature;        /* logits are divided by it before the softmax (paper: 1.0) */
+  int32_t mode;             /* VVS_MODE_* */
+  int32_t nbr_k;            /* relaxed: use the first nbr_k entries of each CSR row */
+  float delta;              /* relaxed: pooled neighbour mass (excluding p(x)) stays <= delta;
+                               INFINITY = pool all nbr_k neighbours */
+} vvs_verify_args;
+
+/* Outputs, device memory allocated by the caller.  Optional ones may be NULL and are then
+ * never computed or written. */
+typedef struct vvs_verify_out {
+  int32_t* accept_len;  /* [B] number of accepted drafts (accepted-prefix length) */
+  int32_t* next_token;  /* [B] embedding-table id sampled from norm(max(0, p - q)) at the first
+                           rejected position, or from the bonus row p_{T-1} if all accepted */
+  int32_t* new_len;     /* [R] cache_len + F + accept_len: fill level after the step */
+  uint8_t* accept_mask; /* optional [B, K] */
+  float* target_probs;  /* optional [B, T, V] float32 target distributions after guidance */
+  void* hidden;         /* optional T [R, T, d_model] features (final-norm output) */
+  float* margins;       /* optional [B, K+1]: |u_i - ratio_i| for judged drafts (INFINITY for
+                           drafts not judged) and, in column K, the distance of the sample
+                           point to the nearest CDF bin edge as a fraction of the total mass */
+} vvs_verify_out;
+
+/* The verification step.  Steps: embedding gather; n_layers x { RMSNorm, QKV projection,
+ * RoPE, KV append, block-vs-cache attention causal inside the block, output projection,
+ * RMSNorm, SwiGLU MLP }; final RMSNorm (= features); LM head over the codebook rows; guidance;
+ * softmax; strict min(1, p/q) or relaxed min(1, P_A/q) acceptance with the accepted-prefix
+ * rule; residual / bonus sample.  Rows of the block whose acceptance fails leave garbage K/V
+ * beyond new_len, overwritten by the next call. */
+int vvs_verify(vvs_ctx* ctx, const vvs_verify_args* args, const vvs_verify_out* out, void* stream);
+
+/* The decision part alone on given features: hidden is device T [R, n_rows_per_seq, d_model];
+ * draft i is judged against row first_row + i, the bonus row is first_row + K (if
+ * n_rows_per_seq <= first_row + K there is no bonus row and next_token = -1 when all drafts
+ * pass).  `drafts` is device int32 [B, K] embedding-table ids.  kv_*, cache_len, block and
+ * n_forced of `args` are ignored; out->new_len and out->hidden must be NULL. */
+int vvs_epilogue(vvs_ctx* ctx, const void* hidden, int32_t n_rows_per_seq, int32_t first_row,
+                 const int32_t* drafts, const vvs_verify_args* args, const vvs_verify_out* out,
+                 void* stream);
+
+/* Token-level feature cache (Sec. 4.3): per sequence a ring of `cap` slots holding the most
+ * recent features, addressed by absolute position (slot = pos mod cap).  All arrays are
+ * device memory owned by the caller; vvs_feature_cache_reset marks every slot empty. */
+typedef struct vvs_fcache {
+  void* feat;       /* T [n_rows, cap, d_model] */
+  int32_t* fpos;    /* [n_rows, cap] position held by each slot, -1 = empty */
+  int32_t* newest;  /* [n_rows] newest position ever stored, -1 = none */
+  int32_t n_rows;
+  int32_t cap;      /* the paper keeps n = max accepted length = 5 features per sequence */
+} vvs_fcache;
+
+int vvs_feature_cache_reset(vvs_ctx* ctx, const vvs_fcache* fc, void* stream);
+
+/* UpdateCache(h_t): for each sequence r, copy hidden[r, t, :] for t < n_store[r] into the slot
+ * of position base_pos[r] + t, tag the slot, raise newest[r].  hidden is device
+ * T [n_rows, n_rows_per_seq, d_model]; base_pos, n_store device int32 [n_rows]
+ * (0 <= n_store[r] <= min(n_rows_per_seq, cap)).  Storing a position again overwrites it (how
+ * post verification writes refreshed features back, Sec. 4.1). */
+int vvs_feature_cache_store(vvs_ctx* ctx, const vvs_fcache* fc, const void* hidden,
+                            int32_t n_rows_per_seq, const int32_t* base_pos,
+                            const int32_t* n_store, void* stream);
+
+/* Retrieve(C, a): for sequences of images with skip_mask[b] != 0 (device uint8 [n_images],
+ * row r belongs to image r mod n_images), gather the gamma[r] most recent features ending
+ * `staleness` positions before the newest one, oldest first, into out[r, j, :] (device
+ * T [n_rows, gamma_max, d_model]) and their positions into out_pos[r, j] (device int32
+ * [n_rows, gamma_max]).  A position that is not in the ring gives out_pos = -1, a zero row and
+ * the VVS_DEV_FCACHE_MISS status bit.  Rows of unmasked images and entries j >= gamma[r] are
+ * not touched. */
+int vvs_feature_cache_fetch(vvs_ctx* ctx, const vvs_fcache* fc, const uint8_t* skip_mask,
+                            int32_t n_images, const int32_t* gamma, int32_t gamma_max,
+                            int32_t staleness, void* out, int32_t* out_pos, void* stream);
+
+/* Synchronise `stream`, copy the device status word to *out_bits (VVS_DEV_* bits) and clear
+ * it.  Returns VVS_ERR_DEVICE_TIMEOUT / VVS_ERR_DEVICE_BOUNDS if such a bit was set. */
+int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits);
+
+/* Number of kernels the last vvs_verify / vvs_epilogue call on this context launched. */
+int vvs_last_launch_count(const vvs_ctx* ctx);
+
+const char* vvs_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VVS_H_ */

@@ -1,0 +1,403 @@
+// C ABI of the verify-step library: argument checks, scratch layout, launch sequences.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "vvs_internal.cuh"
+
+using namespace vvs;
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t elem_bytes(const vvs_model_desc& d) { return d.dtype == VVS_DTYPE_BF16 ? 2 : 4; }
+
+// Carves the scratch arena; with base == nullptr only the total size is computed.
+struct Carver {
+  char* base;
+  size_t off = 0;
+  template <typename P>
+  void take(P*& p, size_t bytes) {
+    off = (off + 255) & ~size_t(255);
+    if (base) p = reinterpret_cast<P*>(base + off);
+    off += bytes;
+  }
+};
+
+size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
+  Carver c{base};
+  const size_t es = elem_bytes(d);
+  const size_t M = (size_t)d.max_rows * d.max_block;  // activation rows; also bounds B*T
+  const size_t V = d.vocab, dm = d.d_model, ff = d.d_ff;
+  const size_t n_tiles = (V + 127) / 128;
+  const size_t n_chunks = (V + kSampleChunk - 1) / kSampleChunk;
+  c.take(ws.status, 256);
+  c.take(ws.rope_inv_freq, (size_t)d.head_dim / 2 * 4);
+  if (d.n_layers > 0) {
+    c.take(ws.x, M * dm * 4);
+    c.take(ws.xn, M * dm * es);
+    c.take(ws.qkv, M * 3 * dm * 4);
+    c.take(ws.q, M * dm * es);
+    c.take(ws.attn, M * dm * es);
+    c.take(ws.gu, M * 2 * ff * 4);
+    c.take(ws.act, M * ff * es);
+    c.take(ws.hid, M * dm * es);
+  }
+  c.take(ws.logits_raw, M * V * 4);
+  c.take(ws.logits, M * V * 4);
+  c.take(ws.part_m, n_tiles * M * 4);
+  c.take(ws.part_s, n_tiles * M * 4);
+  c.take(ws.stat_m, M * 4);
+  c.take(ws.stat_inv, M * 4);
+  c.take(ws.l_tok, M * 4);
+  c.take(ws.l_nbr, M * (size_t)d.max_nbr_k * 4);
+  c.take(ws.sel_row, (size_t)d.max_rows * 4);
+  c.take(ws.sel_kind, (size_t)d.max_rows * 4);
+  c.take(ws.p_row, (size_t)d.max_rows * V * 4);
+  c.take(ws.r_part, (size_t)d.max_rows * n_chunks * 8);
+  c.take(ws.p_part, (size_t)d.max_rows * n_chunks * 8);
+  return (c.off + 255) & ~size_t(255);
+}
+
+int check_desc(const vvs_model_desc* d) {
+  if (!d) return VVS_ERR_INVALID_ARG;
+  if (d->dtype != VVS_DTYPE_FP32 && d->dtype != VVS_DTYPE_BF16) return VVS_ERR_INVALID_ARG;
+  if (d->rope_mode < VVS_ROPE_NONE || d->rope_mode > VVS_ROPE_2D_GRID) return VVS_ERR_INVALID_ARG;
+  if (d->n_layers < 0 || d->d_model <= 0 || d->vocab <= 0 || d->vocab_offset < 0) return VVS_ERR_SHAPE;
+  if (d->lm_rows < d->vocab_offset + d->vocab) return VVS_ERR_SHAPE;
+  if (d->d_model % 8) return VVS_ERR_SHAPE;
+  if (d->max_rows < 1 || d->max_block < 1 || d->max_block > 32 || d->max_nbr_k < 1) return VVS_ERR_SHAPE;
+  if (d->n_layers > 0) {
+    if (d->head_dim != 64 && d->head_dim != 128) return VVS_ERR_SHAPE;
+    if (d->n_heads <= 0 || d->n_heads * d->head_dim != d->d_model) return VVS_ERR_SHAPE;
+    if (d->d_ff <= 0 || d->d_ff % 8) return VVS_ERR_SHAPE;
+    if (d->s_max < 1 || d->tok_rows < 1) return VVS_ERR_SHAPE;
+    if (d->rope_mode == VVS_ROPE_2D_GRID && (d->rope_grid_w < 1 || d->n_prefix < 0)) return VVS_ERR_SHAPE;
+    if (!(d->rms_eps > 0.f) || !(d->rope_base > 1.f)) return VVS_ERR_INVALID_ARG;
+  }
+  return VVS_OK;
+}
+
+struct Counter {
+  vvs_ctx* ctx;
+  void operator()(int n = 1) const { ctx->launches += n; }
+};
+
+// LM head over the codebook rows, guidance, softmax statistics, decisions.  Generic path: the
+// per-sequence logits and the guided logits live in scratch.
+template <typename T>
+int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, const int32_t* drafts,
+                  int drafts_ld, const vvs_verify_args* a, const vvs_verify_out* o, bool with_cache,
+                  cudaStream_t s) {
+  const vvs_model_desc& md = ctx->desc;
+  Workspace& ws = ctx->ws;
+  Counter count{ctx};
+  const int B = a->n_images, C = a->n_cfg, R = B * C;
+  const int M = R * rows_per_seq, V = md.vocab, BT = B * rows_per_seq;
+  const T* w_lm = static_cast<const T*>(ctx->w_lm) + (size_t)md.vocab_offset * md.d_model;
+
+  DecideParams p{};
+  p.n_images = B; p.n_cfg = C; p.rows_per_seq = rows_per_seq; p.first_row = first_row;
+  p.n_draft_max = a->n_draft_max; p.vocab = V; p.vocab_offset = md.vocab_offset;
+  p.mode = a->mode; p.nbr_k = a->mode == VVS_MODE_RELAXED ? a->nbr_k : 1; p.kmax = md.max_nbr_k;
+  p.delta = a->delta;
+  p.drafts = drafts; p.drafts_ld = drafts_ld; p.n_draft = a->n_draft;
+  p.draft_probs = a->draft_probs; p.uniforms = a->uniforms;
+  p.row_ptr = ctx->nbr_row_ptr; p.col = ctx->nbr_col;
+  p.cache_len = with_cache ? a->cache_len : nullptr; p.n_forced = a->n_forced;
+  p.accept_len = o->accept_len; p.next_token = o->next_token;
+  p.new_len = with_cache ? o->new_len : nullptr;
+  p.accept_mask = o->accept_mask; p.margins = o->margins;
+
+  launch_gemm_nt<T>(hid, w_lm, ws.logits_raw, M, V, md.d_model, V, false, s); count();
+  launch_guide(ws.logits_raw, ws.logits, B, C, rows_per_seq, V, a->cfg_scale, 1.f / a->temperature, s);
+  count();
+  launch_row_stats(ws.logits, ws.part_m, ws.part_s, BT, V, s); count();
+  launch_finalize_stats(ws, 1, BT, s); count();
+  if (p.n_draft_max > 0) { launch_gather_logits(ws, p, s); count(); }
+  launch_accept(ws, p, s); count();
+  if (o->target_probs) { launch_probs_from_logits(ws.logits, ws, o->target_probs, BT, V, s); count(); }
+  launch_select_p_row(ws, B, V, s); count();
+  launch_sample(ws, p, s); count(2);
+  return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+}
+
+template <typename T>
+int run_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, cudaStream_t s) {
+  const vvs_model_desc& md = ctx->desc;
+  Workspace& ws = ctx->ws;
+  Counter count{ctx};
+  const int B = a->n_images, C = a->n_cfg, R = B * C, Tn = a->n_forced + a->n_draft_max;
+  const int M = R * Tn, d = md.d_model, ff = md.d_ff;
+  T* kv_k = static_cast<T*>(a->kv_k);
+  T* kv_v = static_cast<T*>(a->kv_v);
+  T* xn = static_cast<T*>(ws.xn);
+  T* q = static_cast<T*>(ws.q);
+  T* attn = static_cast<T*>(ws.attn);
+  T* act = static_cast<T*>(ws.act);
+  T* hid = o->hidden ? static_cast<T*>(o->hidden) : static_cast<T*>(ws.hid);
+
+  launch_embed<T>(static_cast<const T*>(ctx->tok_emb), a->block, ws.x, B, C, Tn, d, md.tok_rows,
+                  ws.status, s);
+  count();
+  for (int l = 0; l < md.n_layers; ++l) {
+    const Layer& L = ctx->layers[l];
+    launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm1), xn, M, d, md.rms_eps, s); count();
+    launch_gemm_nt<T>(xn, static_cast<const T*>(L.w_qkv), ws.qkv, M, 3 * d, d, 3 * d, false, s); count();
+    launch_rope_append<T>(ws.qkv, ws.rope_inv_freq, q, kv_k, kv_v, a->cache_len, md, l, a->kv_rows, R,
+                          Tn, ws.status, s);
+    count();
+    launch_attention<T>(q, kv_k, kv_v, a->cache_len, attn, md, l, a->kv_rows, R, Tn, s); count();
+    launch_gemm_nt<T>(attn, static_cast<const T*>(L.w_o), ws.x, M, d, d, d, true, s); count();
+    launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm2), xn, M, d, md.rms_eps, s); count();
+    launch_gemm_nt<T>(xn, static_cast<const T*>(L.w_gate), ws.gu, M, ff, d, 2 * ff, false, s); count();
+    launch_gemm_nt<T>(xn, static_cast<const T*>(L.w_up), ws.gu + ff, M, ff, d, 2 * ff, false, s); count();
+    launch_silu_mul<T>(ws.gu, act, M, ff, s); count();
+    launch_gemm_nt<T>(act, static_cast<const T*>(L.w_down), ws.x, M, d, ff, d, true, s); count();
+  }
+  launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s); count();
+  if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
+  return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
+}
+
+int check_decision_args(const vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o,
+                        int rows_per_seq) {
+  const vvs_model_desc& md = ctx->desc;
+  if (!a || !o) return VVS_ERR_INVALID_ARG;
+  if (!ctx->weights_bound) return VVS_ERR_NOT_BOUND;
+  if (a->n_images < 1 || (a->n_cfg != 1 && a->n_cfg != 2) || a->n_draft_max < 0) return VVS_ERR_SHAPE;
+  if (a->n_images * a->n_cfg > md.max_rows || rows_per_seq > md.max_block || rows_per_seq < 1)
+    return VVS_ERR_SHAPE;
+  if (!a->uniforms || !o->accept_len || !o->next_token) return VVS_ERR_INVALID_ARG;
+  if (a->n_draft_max > 0 && !a->draft_probs) return VVS_ERR_INVALID_ARG;
+  if (!(a->temperature > 0.f) || !std::isfinite(a->temperature) || !std::isfinite(a->cfg_scale))
+    return VVS_ERR_INVALID_ARG;
+  if (a->mode != VVS_MODE_STRICT && a->mode != VVS_MODE_RELAXED) return VVS_ERR_INVALID_ARG;
+  if (a->mode == VVS_MODE_RELAXED) {
+    if (a->nbr_k < 1 || a->nbr_k > md.max_nbr_k) return VVS_ERR_SHAPE;
+    if (!(a->delta >= 0.f)) return VVS_ERR_INVALID_ARG;  // also rejects NaN
+    if (a->nbr_k > 1 && (!ctx->nbr_row_ptr || !ctx->nbr_col)) return VVS_ERR_NOT_BOUND;
+  }
+  if (!aligned16(a->draft_probs) || !aligned16(o->target_probs)) return VVS_ERR_ALIGN;
+  return VVS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int vvs_workspace_bytes(const vvs_model_desc* desc, size_t* out_bytes) {
+  int rc = check_desc(desc);
+  if (rc != VVS_OK) return rc;
+  if (!out_bytes) return VVS_ERR_INVALID_ARG;
+  Workspace tmp;
+  *out_bytes = layout(*desc, tmp, nullptr);
+  return VVS_OK;
+}
+
+int vvs_create(const vvs_model_desc* desc, vvs_ctx** out) {
+  if (out) *out = nullptr;
+  int rc = check_desc(desc);
+  if (rc != VVS_OK) return rc;
+  if (!out) return VVS_ERR_INVALID_ARG;
+  vvs_ctx* ctx = new (std::nothrow) vvs_ctx();
+  if (!ctx) return VVS_ERR_NOMEM;
+  ctx->desc = *desc;
+  if (cudaGetDevice(&ctx->device) != cudaSuccess) { delete ctx; return VVS_ERR_CUDA; }
+  Workspace tmp;
+  ctx->arena_bytes = layout(*desc, tmp, nullptr);
+  if (cudaMalloc(&ctx->arena, ctx->arena_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    delete ctx;
+    return VVS_ERR_NOMEM;
+  }
+  layout(*desc, ctx->ws, static_cast<char*>(ctx->arena));
+  if (cudaMemset(ctx->arena, 0, ctx->arena_bytes) != cudaSuccess) { vvs_destroy(ctx); return VVS_ERR_CUDA; }
+  // rotation angle per unit coordinate of each consecutive pair
+  const int half = desc->head_dim / 2;
+  if (half > 0) {
+    float* f = static_cast<float*>(std::malloc(sizeof(float) * half));
+    if (!f) { vvs_destroy(ctx); return VVS_ERR_NOMEM; }
+    for (int i = 0; i < half; ++i) {
+      if (desc->rope_mode == VVS_ROPE_2D_GRID) {
+        int j = i % (half / 2);
+        f[i] = (float)std::pow((double)desc->rope_base, -2.0 * j / (double)half);
+      } else {
+        f[i] = (float)std::pow((double)desc->rope_base, -2.0 * i / (double)desc->head_dim);
+      }
+    }
+    cudaError_t e = cudaMemcpy(ctx->ws.rope_inv_freq, f, sizeof(float) * half, cudaMemcpyHostToDevice);
+    std::free(f);
+    if (e != cudaSuccess) { vvs_destroy(ctx); return VVS_ERR_CUDA; }
+  }
+  if (desc->n_layers > 0) {
+    ctx->layers = new (std::nothrow) Layer[desc->n_layers]();
+    if (!ctx->layers) { vvs_destroy(ctx); return VVS_ERR_NOMEM; }
+  }
+  *out = ctx;
+  return VVS_OK;
+}
+
+int vvs_destroy(vvs_ctx* ctx) {
+  if (!ctx) return VVS_ERR_INVALID_ARG;
+  if (ctx->arena) cudaFree(ctx->arena);
+  delete[] ctx->layers;
+  delete ctx;
+  return VVS_OK;
+}
+
+int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w) {
+  if (!ctx || !w) return VVS_ERR_INVALID_ARG;
+  const int n = ctx->desc.n_layers;
+  if (!w->w_lm) return VVS_ERR_INVALID_ARG;
+  if (!aligned16(w->w_lm)) return VVS_ERR_ALIGN;
+  if (n > 0) {
+    if (!w->tok_emb || !w->norm_f || !w->layers) return VVS_ERR_INVALID_ARG;
+    if (!aligned16(w->tok_emb) || !aligned16(w->norm_f)) return VVS_ERR_ALIGN;
+    for (int l = 0; l < n; ++l) {
+      const vvs_layer_weights& s = w->layers[l];
+      const void* ptrs[7] = {s.w_qkv, s.w_o, s.w_gate, s.w_up, s.w_down, s.norm1, s.norm2};
+      for (const void* p : ptrs) {
+        if (!p) return VVS_ERR_INVALID_ARG;
+        if (!aligned16(p)) return VVS_ERR_ALIGN;
+      }
+    }
+    for (int l = 0; l < n; ++l) {
+      const vvs_layer_weights& s = w->layers[l];
+      ctx->layers[l] = Layer{s.w_qkv, s.w_o, s.w_gate, s.w_up, s.w_down, s.norm1, s.norm2};
+    }
+  }
+  ctx->tok_emb = w->tok_emb;
+  ctx->norm_f = w->norm_f;
+  ctx->w_lm = w->w_lm;
+  ctx->weights_bound = true;
+  return VVS_OK;
+}
+
+int vvs_bind_neighbors(vvs_ctx* ctx, const int32_t* row_ptr, const int32_t* col, int64_t nnz) {
+  if (!ctx || !row_ptr || !col || nnz < 0) return VVS_ERR_INVALID_ARG;
+  if (!aligned16(row_ptr) || !aligned16(col)) return VVS_ERR_ALIGN;
+  ctx->nbr_row_ptr = row_ptr;
+  ctx->nbr_col = col;
+  ctx->nbr_nnz = nnz;
+  return VVS_OK;
+}
+
+int vvs_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, void* stream) {
+  if (!ctx) return VVS_ERR_INVALID_ARG;
+  const vvs_model_desc& md = ctx->desc;
+  if (md.n_layers < 1) return VVS_ERR_SHAPE;
+  if (!a || !o) return VVS_ERR_INVALID_ARG;
+  if (a->n_forced < 1) return VVS_ERR_SHAPE;
+  const int Tn = a->n_forced + a->n_draft_max;
+  int rc = check_decision_args(ctx, a, o, Tn);
+  if (rc != VVS_OK) return rc;
+  const int R = a->n_images * a->n_cfg;
+  if (!a->block || !a->kv_k || !a->kv_v || !a->cache_len || !o->new_len) return VVS_ERR_INVALID_ARG;
+  if (a->kv_rows < R) return VVS_ERR_SHAPE;
+  if (!aligned16(a->kv_k) || !aligned16(a->kv_v) || !aligned16(o->hidden)) return VVS_ERR_ALIGN;
+  if (a->cache_len_host) {
+    for (int r = 0; r < R; ++r)
+      if (a->cache_len_host[r] < 0 || a->cache_len_host[r] + Tn > md.s_max) return VVS_ERR_CAPACITY;
+  }
+  ctx->launches = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  return md.dtype == VVS_DTYPE_BF16 ? run_verify<__nv_bfloat16>(ctx, a, o, s)
+                                    : run_verify<float>(ctx, a, o, s);
+}
+
+int vvs_epilogue(vvs_ctx* ctx, const void* hidden, int32_t n_rows_per_seq, int32_t first_row,
+                 const int32_t* drafts, const vvs_verify_args* a, const vvs_verify_out* o,
+                 void* stream) {
+  if (!ctx || !hidden) return VVS_ERR_INVALID_ARG;
+  int rc = check_decision_args(ctx, a, o, n_rows_per_seq);
+  if (rc != VVS_OK) return rc;
+  if (first_row < 0 || first_row + a->n_draft_max > n_rows_per_seq) return VVS_ERR_SHAPE;
+  if (a->n_draft_max > 0 && !drafts) return VVS_ERR_INVALID_ARG;
+  if (o->new_len || o->hidden) return VVS_ERR_INVALID_ARG;
+  if (!aligned16(hidden)) return VVS_ERR_ALIGN;
+  ctx->launches = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (ctx->desc.dtype == VVS_DTYPE_BF16)
+    return run_decisions<__nv_bfloat16>(ctx, static_cast<const __nv_bfloat16*>(hidden), n_rows_per_seq,
+                                        first_row, drafts, a->n_draft_max, a, o, false, s);
+  return run_decisions<float>(ctx, static_cast<const float*>(hidden), n_rows_per_seq, first_row, drafts,
+                              a->n_draft_max, a, o, false, s);
+}
+
+static int check_fcache(const vvs_ctx* ctx, const vvs_fcache* fc) {
+  if (!ctx || !fc) return VVS_ERR_INVALID_ARG;
+  if (!fc->feat || !fc->fpos || !fc->newest) return VVS_ERR_INVALID_ARG;
+  if (fc->n_rows < 1 || fc->cap < 1) return VVS_ERR_SHAPE;
+  if (!aligned16(fc->feat)) return VVS_ERR_ALIGN;
+  return VVS_OK;
+}
+
+int vvs_feature_cache_reset(vvs_ctx* ctx, const vvs_fcache* fc, void* stream) {
+  int rc = check_fcache(ctx, fc);
+  if (rc != VVS_OK) return rc;
+  launch_fcache_reset(*fc, static_cast<cudaStream_t>(stream));
+  return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+}
+
+int vvs_feature_cache_store(vvs_ctx* ctx, const vvs_fcache* fc, const void* hidden,
+                            int32_t n_rows_per_seq, const int32_t* base_pos, const int32_t* n_store,
+                            void* stream) {
+  int rc = check_fcache(ctx, fc);
+  if (rc != VVS_OK) return rc;
+  if (!hidden || !base_pos || !n_store) return VVS_ERR_INVALID_ARG;
+  if (n_rows_per_seq < 1) return VVS_ERR_SHAPE;
+  if (!aligned16(hidden)) return VVS_ERR_ALIGN;
+  launch_fcache_store(*fc, hidden, n_rows_per_seq, ctx->desc.d_model, (int)elem_bytes(ctx->desc),
+                      base_pos, n_store, ctx->ws.status, static_cast<cudaStream_t>(stream));
+  return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+}
+
+int vvs_feature_cache_fetch(vvs_ctx* ctx, const vvs_fcache* fc, const uint8_t* skip_mask,
+                            int32_t n_images, const int32_t* gamma, int32_t gamma_max,
+                            int32_t staleness, void* out, int32_t* out_pos, void* stream) {
+  int rc = check_fcache(ctx, fc);
+  if (rc != VVS_OK) return rc;
+  if (!skip_mask || !gamma || !out || !out_pos) return VVS_ERR_INVALID_ARG;
+  if (n_images < 1 || fc->n_rows % n_images != 0 || gamma_max < 1 || staleness < 0) return VVS_ERR_SHAPE;
+  if (!aligned16(out)) return VVS_ERR_ALIGN;
+  launch_fcache_fetch(*fc, skip_mask, n_images, gamma, gamma_max, staleness, ctx->desc.d_model,
+                      (int)elem_bytes(ctx->desc), out, out_pos, ctx->ws.status,
+                      static_cast<cudaStream_t>(stream));
+  return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+}
+
+int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits) {
+  if (!ctx || !out_bits) return VVS_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t bits = 0;
+  VVS_CUDA_OK(cudaMemcpyAsync(&bits, ctx->ws.status, sizeof(bits), cudaMemcpyDeviceToHost, s));
+  VVS_CUDA_OK(cudaMemsetAsync(ctx->ws.status, 0, sizeof(bits), s));
+  VVS_CUDA_OK(cudaStreamSynchronize(s));
+  *out_bits = bits;
+  if (bits & VVS_DEV_TIMEOUT) return VVS_ERR_DEVICE_TIMEOUT;
+  if (bits & (VVS_DEV_BAD_TOKEN | VVS_DEV_CACHE_OVERFLOW | VVS_DEV_BAD_NEIGHBOUR | VVS_DEV_BAD_ARG))
+    return VVS_ERR_DEVICE_BOUNDS;
+  return VVS_OK;
+}
+
+int vvs_last_launch_count(const vvs_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* vvs_strerror(int status) {
+  switch (status) {
+    case VVS_OK: return "ok";
+    case VVS_ERR_INVALID_ARG: return "invalid argument";
+    case VVS_ERR_SHAPE: return "shape outside the model description or its limits";
+    case VVS_ERR_ALIGN: return "device pointer not 16-byte aligned";
+    case VVS_ERR_CAPACITY: return "KV cache capacity exceeded";
+    case VVS_ERR_NOT_BOUND: return "weights or neighbour table not bound";
+    case VVS_ERR_CUDA: return "CUDA runtime error";
+    case VVS_ERR_DEVICE_TIMEOUT: return "bounded device-side wait ran out";
+    case VVS_ERR_DEVICE_BOUNDS: return "device-side index check failed";
+    case VVS_ERR_NOMEM: return "out of memory";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

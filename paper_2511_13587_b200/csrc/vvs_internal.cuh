@@ -1,0 +1,135 @@
+// Internal declarations of the verify-step library: context, scratch layout, launchers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vvs.h"
+
+#define VVS_CUDA_OK(expr)                         \
+  do {                                            \
+    cudaError_t e__ = (expr);                     \
+    if (e__ != cudaSuccess) return VVS_ERR_CUDA;  \
+  } while (0)
+
+namespace vvs {
+
+// Scratch memory of a context.  Row index m of an activation matrix is r * T + t with
+// r = c * B + b (cond sequences first).  "Decision rows" are (b, t) pairs: index b * T + t.
+struct Workspace {
+  float* x = nullptr;        // [M, d]   fp32 residual stream
+  void* xn = nullptr;        // [M, d]   T normalised activations (GEMM input)
+  float* qkv = nullptr;      // [M, 3d]  fp32 projections before RoPE
+  void* q = nullptr;         // [M, d]   T queries after RoPE
+  void* attn = nullptr;      // [M, d]   T attention output
+  float* gu = nullptr;       // [M, 2ff] fp32 gate | up
+  void* act = nullptr;       // [M, ff]  T silu(gate) * up
+  void* hid = nullptr;       // [M, d]   T features when the caller does not ask for them
+  float* logits_raw = nullptr;  // [M, V] fp32 per-sequence logits (generic path)
+  float* logits = nullptr;      // [B*T, V] fp32 guided logits / temperature (generic path)
+  float* part_m = nullptr;   // [n_tiles, B*T] per-tile running max
+  float* part_s = nullptr;   // [n_tiles, B*T] per-tile sum of exp(l - max)
+  float* stat_m = nullptr;   // [B*T] row max
+  float* stat_inv = nullptr; // [B*T] 1 / sum exp(l - max)
+  float* l_tok = nullptr;    // [B, K] guided logit of each drafted token
+  float* l_nbr = nullptr;    // [B, K, kmax] guided logits of its neighbours (entry 0 unused)
+  int32_t* sel_row = nullptr;   // [B] decision row (b*T + t) the next token is sampled from, -1 none
+  int32_t* sel_kind = nullptr;  // [B] 0 = residual of draft n, 1 = bonus
+  float* p_row = nullptr;    // [B, V] target probabilities of the selected row
+  double* r_part = nullptr;  // [B, n_chunks] per-chunk residual mass
+  double* p_part = nullptr;  // [B, n_chunks] per-chunk target mass (fallback when residual is 0)
+  float* rope_inv_freq = nullptr;  // [head_dim/2] angle per unit coordinate of each pair
+  int32_t* status = nullptr; // device status word
+};
+
+struct Layer {
+  const void *w_qkv, *w_o, *w_gate, *w_up, *w_down, *norm1, *norm2;
+};
+
+}  // namespace vvs
+
+struct vvs_ctx {
+  vvs_model_desc desc;
+  vvs::Workspace ws;
+  void* arena = nullptr;
+  size_t arena_bytes = 0;
+  bool weights_bound = false;
+  const void* tok_emb = nullptr;
+  const void* norm_f = nullptr;
+  const void* w_lm = nullptr;
+  vvs::Layer* layers = nullptr;  // host array [n_layers]
+  const int32_t* nbr_row_ptr = nullptr;
+  const int32_t* nbr_col = nullptr;
+  int64_t nbr_nnz = 0;
+  int device = 0;
+  int launches = 0;
+};
+
+namespace vvs {
+
+constexpr int kSampleChunk = 1024;  // codebook entries per residual-mass chunk
+
+// ---- generic kernels (any storage type), kernels_generic.cu ---------------------------------
+template <typename T>
+void launch_embed(const T* tok_emb, const int32_t* block, float* x, int n_images, int n_cfg,
+                  int t_len, int d, int tok_rows, int32_t* status, cudaStream_t s);
+template <typename T>
+void launch_rmsnorm(const float* x, const T* scale, T* out, int m, int d, float eps, cudaStream_t s);
+// c[m, n] (+)= sum_k a[m, k] * w[n, k]; c fp32 with leading dimension ldc
+template <typename T>
+void launch_gemm_nt(const T* a, const T* w, float* c, int m, int n, int k, int ldc, bool accumulate,
+                    cudaStream_t s);
+template <typename T>
+void launch_rope_append(const float* qkv, const float* inv_freq, T* q, T* kv_k, T* kv_v,
+                        const int32_t* cache_len, const vvs_model_desc& md, int layer, int kv_rows,
+                        int n_rows, int t_len, int32_t* status, cudaStream_t s);
+template <typename T>
+void launch_attention(const T* q, const T* kv_k, const T* kv_v, const int32_t* cache_len, T* out,
+                      const vvs_model_desc& md, int layer, int kv_rows, int n_rows, int t_len,
+                      cudaStream_t s);
+template <typename T>
+void launch_silu_mul(const float* gu, T* act, int m, int ff, cudaStream_t s);
+void launch_guide(const float* raw, float* logits, int n_images, int n_cfg, int rows_per_seq, int v,
+                  float cfg_scale, float inv_temp, cudaStream_t s);
+void launch_row_stats(const float* logits, float* part_m, float* part_s, int n_rows, int v,
+                      cudaStream_t s);
+
+// ---- decision stage, kernels_decide.cu -----------------------------------------------------
+struct DecideParams {
+  int n_images, n_cfg, rows_per_seq, first_row, n_draft_max, vocab, vocab_offset;
+  int mode, nbr_k, kmax;
+  float delta;
+  const int32_t* drafts;      // [B, drafts_ld] embedding ids
+  int drafts_ld;
+  const int32_t* n_draft;     // [B] or null
+  const float* draft_probs;   // [B, K, V]
+  const float* uniforms;      // [B, K+1]
+  const int32_t* row_ptr;
+  const int32_t* col;
+  const int32_t* cache_len;   // [R] or null (epilogue entry)
+  int n_forced;
+  int32_t* accept_len;
+  int32_t* next_token;
+  int32_t* new_len;
+  uint8_t* accept_mask;
+  float* margins;
+};
+void launch_finalize_stats(const Workspace& ws, int n_tiles, int n_rows, cudaStream_t s);
+void launch_gather_logits(const Workspace& ws, const DecideParams& p, cudaStream_t s);
+void launch_accept(const Workspace& ws, const DecideParams& p, cudaStream_t s);
+void launch_probs_from_logits(const float* logits, const Workspace& ws, float* probs, int n_rows,
+                              int v, cudaStream_t s);
+void launch_select_p_row(const Workspace& ws, int n_images, int v, cudaStream_t s);
+void launch_sample(const Workspace& ws, const DecideParams& p, cudaStream_t s);
+
+// ---- feature cache, kernels_fcache.cu ---------------------------------------------------------
+void launch_fcache_reset(const vvs_fcache& fc, cudaStream_t s);
+void launch_fcache_store(const vvs_fcache& fc, const void* hidden, int rows_per_seq, int d,
+                         int elem_bytes, const int32_t* base_pos, const int32_t* n_store,
+                         int32_t* status, cudaStream_t s);
+void launch_fcache_fetch(const vvs_fcache& fc, const uint8_t* skip_mask, int n_images,
+                         const int32_t* gamma, int gamma_max, int staleness, int d, int elem_bytes,
+                         void* out, int32_t* out_pos, int32_t* status, cudaStream_t s);
+
+}  // namespace vvs

@@ -1,0 +1,190 @@
+"""Parity of vvs_verify (through the C ABI) with the fp64 oracle on seeded inputs.
+
+Two regimes.  Decision replay: the oracle's decision stage re-run on the float32 target
+probabilities the GPU emitted must reproduce accept_len / accept_mask / next_token bit for bit
+(decisions within 1e-4 of their threshold excluded and counted).  End to end: probabilities
+within 2e-3 absolute (bf16) / 1e-5 (fp32), features within 1e-2 relative (bf16) / 1e-4 (fp32),
+appended K/V within the same relative bound, integer outputs equal unless the oracle's own
+margin is below the float error of the ratio."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import helpers as H
+from vvs_synth.configs import (B7_SMALL, CONFIGS, DTYPE_BF16, MODE_RELAXED, TINY, XL_SMALL)
+
+pytestmark = pytest.mark.gpu
+
+
+def _tols(ms):
+    if ms.dtype == DTYPE_BF16:
+        return dict(p_abs=2e-3, p_rel=6e-2, h_rel=1e-2, int_margin=6e-2)
+    return dict(p_abs=1e-5, p_rel=2e-4, h_rel=1e-4, int_margin=1e-4)
+
+
+def _check_end_to_end(case, gpu, ora):
+    ms = case["ms"]
+    tol = _tols(ms)
+    assert gpu["status"] == 0
+    assert gpu["launches"] > 0
+    assert H.rel_err_rows(gpu["hidden"], ora["hidden"]) < tol["h_rel"]
+    dp = np.abs(gpu["target_probs"] - ora["target_probs"])
+    assert dp.max() < tol["p_abs"]
+    assert (dp / ora["target_probs"]).max() < tol["p_rel"]
+    np.testing.assert_allclose(gpu["target_probs"].sum(-1), 1.0, atol=1e-4)
+    H.check_new_cache_rows(case, gpu, ora, tol["h_rel"])
+    # integer outputs against the oracle's own pipeline, classified by the oracle's margins
+    k = case["n_draft_max"]
+    real = 0
+    for b in range(case["n_images"]):
+        if gpu["accept_len"][b] != ora["accept_len"][b]:
+            n = min(gpu["accept_len"][b], ora["accept_len"][b])
+            ratio = max(ora["ratios"][b][n], 1e-30)
+            if ora["margins"][b][n] > tol["int_margin"] * max(ratio, 1e-3):
+                real += 1
+    assert real == 0
+    np.testing.assert_array_equal(
+        gpu["new_len"], case["cache_len"] + case["n_forced"] +
+        gpu["accept_len"][np.arange(len(gpu["new_len"])) % case["n_images"]])
+    return H.check_replay(case, gpu)
+
+
+def test_config0_tiny_fp32_strict():
+    """BASELINE configs[0]: 2 layers, d = 256, V = 1024, batch 1, no guidance, fill 64, K = 4."""
+    w = CONFIGS[0]
+    for trial in range(3):
+        case = H.build_case(w.shape, w.seed + trial, 1, 1, 1, 4, [64], cfg_scale=1.0,
+                            q_noise=0.7 if trial else 2.0, call_id=trial)
+        run = H.GpuRunner(w.shape, case["w"], 1, 5)
+        gpu = run.verify(case)
+        ora = H.run_oracle(case)
+        assert _check_end_to_end(case, gpu, ora) == 0
+        np.testing.assert_array_equal(gpu["accept_len"], ora["accept_len"])
+        np.testing.assert_array_equal(gpu["next_token"], ora["next_token"])
+        run.close()
+
+
+@pytest.mark.parametrize("n_images,fills", [(1, [288]), (3, [1, 575, 130])])
+def test_xl_shape_small_bf16_cfg(n_images, fills):
+    """LlamaGen-XL structure (2-D grid rope, 1 prefix token, guidance 2.0, K = 8) at reduced
+    width/depth; an extra unused cache row must stay untouched."""
+    ms = XL_SMALL
+    case = H.build_case(ms, 11 + n_images, n_images, 2, 1, 8, fills, kv_rows=2 * n_images + 1)
+    run = H.GpuRunner(ms, case["w"], 2 * n_images, 9)
+    gpu = run.verify(case)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    # outputs not requested are not needed for the decisions
+    gpu2 = run.verify(case, want_probs=False, want_hidden=False)
+    np.testing.assert_array_equal(gpu2["accept_len"], gpu["accept_len"])
+    np.testing.assert_array_equal(gpu2["next_token"], gpu["next_token"])
+    run.close()
+
+
+@pytest.mark.parametrize("delta", [float("inf"), 0.1, 0.0])
+def test_relaxed_acceptance_bf16(delta):
+    ms = XL_SMALL
+    case = H.build_case(ms, 23, 4, 2, 1, 8, [10, 200, 333, 574], mode=MODE_RELAXED, nbr_k=16,
+                        delta=delta, q_noise=1.5)
+    run = H.GpuRunner(ms, case["w"], 8, 9, max_nbr_k=16)
+    gpu = run.verify(case)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    if delta == 0.0:                                    # relaxed with delta = 0 is strict
+        strict = dict(case, mode=0, row_ptr=None, col=None)
+        gpu_s = run.verify(strict)
+        np.testing.assert_array_equal(gpu_s["accept_len"], gpu["accept_len"])
+        np.testing.assert_array_equal(gpu_s["next_token"], gpu["next_token"])
+    run.close()
+
+
+def test_7b_shape_small_bf16():
+    """7B structure: head_dim 128, 1-D rope, codebook inside a larger vocabulary."""
+    ms = B7_SMALL
+    case = H.build_case(ms, 31, 1, 2, 1, 8, [300])
+    run = H.GpuRunner(ms, case["w"], 2, 9)
+    gpu = run.verify(case)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    assert ((gpu["next_token"] >= ms.vocab_offset) & (gpu["next_token"] < ms.vocab_offset + ms.vocab)).all()
+    run.close()
+
+
+def test_ragged_drafts_forced_prefix_and_cache_edges():
+    """n_draft below K (including 0), two forced rows, an empty cache and a cache that the block
+    fills to capacity."""
+    ms = replace(XL_SMALL, s_max=64)
+    case = H.build_case(ms, 41, 4, 2, 2, 6, [0, 64 - 8, 5, 17], n_draft=[6, 3, 0, 1], q_noise=0.5)
+    run = H.GpuRunner(ms, case["w"], 8, 8)
+    gpu = run.verify(case)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    assert (gpu["accept_len"] <= case["n_draft"]).all()
+    assert gpu["accept_len"][2] == 0
+    run.close()
+
+
+def test_fp32_with_guidance_and_temperature():
+    ms = replace(TINY, vocab=1000, lm_rows=1000, tok_rows=1000)
+    case = H.build_case(ms, 51, 2, 2, 1, 4, [64, 9], cfg_scale=1.5, temperature=0.8, q_noise=0.6)
+    run = H.GpuRunner(ms, case["w"], 4, 5)
+    gpu = run.verify(case)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    run.close()
+
+
+def test_device_side_checks_report_instead_of_faulting():
+    import torch
+    ms = TINY
+    case = H.build_case(ms, 61, 1, 1, 1, 4, [64])
+    run = H.GpuRunner(ms, case["w"], 1, 5)
+    vb = run.vb
+    bad = dict(case, block=case["block"].copy())
+    bad["block"][0, 0] = ms.tok_rows + 5                 # forced token outside the embedding
+    assert run.verify(bad)["status"] & vb.VVS_DEV_BAD_TOKEN
+    over = dict(case, cache_len=np.array([ms.s_max - 2], np.int32))
+    res = run.verify(over)                               # block would overflow the cache
+    assert res["status"] & vb.VVS_DEV_CACHE_OVERFLOW
+    np.testing.assert_array_equal(res["kv_k"], H.O.widen(case["kv_k"]))   # nothing written
+    ok = run.verify(case)
+    assert ok["status"] == 0                             # context still usable
+    # host-side capacity check
+    a = dict(n_images=1, n_cfg=1, n_forced=1, n_draft_max=4, block=H.to_dev(case["block"]),
+             kv_k=H.to_dev(case["kv_k"]), kv_v=H.to_dev(case["kv_v"]), kv_rows=1,
+             cache_len=H.to_dev(over["cache_len"]), draft_probs=H.to_dev(case["draft_probs"]),
+             uniforms=H.to_dev(case["uniforms"]),
+             accept_len=torch.zeros(1, dtype=torch.int32, device="cuda"),
+             next_token=torch.zeros(1, dtype=torch.int32, device="cuda"),
+             new_len=torch.zeros(1, dtype=torch.int32, device="cuda"))
+    host_len = over["cache_len"].copy()
+    with pytest.raises(vb.VvsError) as e:
+        vb.vvs_verify(run.ctx, cache_len_host=host_len.ctypes.data, **a)
+    assert e.value.status == -4
+    with pytest.raises(vb.VvsError) as e:
+        vb.vvs_verify(run.ctx, **dict(a, n_draft_max=40))
+    assert e.value.status == -2
+    with pytest.raises(vb.VvsError) as e:
+        vb.vvs_verify(run.ctx, **dict(a, mode=1, nbr_k=4))
+    assert e.value.status == -2                          # nbr_k above max_nbr_k
+    with pytest.raises(vb.VvsError) as e:
+        vb.vvs_verify(run.ctx, **dict(a, temperature=0.0))
+    assert e.value.status == -1
+    with pytest.raises(vb.VvsError) as e:
+        vb.vvs_verify(run.ctx, **dict(a, draft_probs=H.to_dev(case["draft_probs"]).data_ptr() + 4))
+    assert e.value.status == -3
+    run.close()
+
+
+def test_deterministic_across_calls():
+    ms = XL_SMALL
+    case = H.build_case(ms, 71, 2, 2, 1, 8, [50, 400])
+    run = H.GpuRunner(ms, case["w"], 4, 9)
+    a = run.verify(case)
+    b = run.verify(case)
+    for key in ("accept_len", "next_token", "accept_mask", "new_len"):
+        np.testing.assert_array_equal(a[key], b[key])
+    np.testing.assert_array_equal(a["target_probs"], b["target_probs"])
+    np.testing.assert_array_equal(a["hidden"], b["hidden"])
+    run.close()
