@@ -1,0 +1,369 @@
+"""Benchmark of the verify step: `python bench.py --gpus N --steps K --warmup W`.
+
+One step = one pass of the whole hot path over one batch of synthetic input: vvs_verify
+(embedding .. acceptance .. residual sample, KV append) followed by the feature-cache store of
+the committed rows (and, for workload 2, the fetch for skip-masked images).  Prints ONE JSON
+line.  `--impl reference` times the fp64 CPU oracle instead, on a bounded sample.
+
+Multi-GPU: the step has no exchange between images, so N GPUs run N independent replicas
+(weak scaling, no collective on the data path); torch.distributed is used only for the barrier
+and the max-over-ranks of the device time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from vvs_synth import gen, philox  # noqa: E402
+from vvs_synth.configs import CONFIGS, MODE_RELAXED  # noqa: E402
+
+N_TRIALS = 32           # distinct (fill, block, draft) inputs cycled through the steps
+DRAFT_LOGIT_STD = 1.0   # target-independent drafter: q = softmax(N(0, std^2))
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------
+# synthetic inputs (host side, seeded)
+
+
+def host_trial(wl, trial: int) -> dict:
+    """Inputs of one verify call of workload `wl`: fills, block, draft distributions, uniforms."""
+    ms = wl.shape
+    b, k, f = wl.n_images, wl.n_draft_max, wl.n_forced
+    fills = gen.make_fills(wl.seed, b, wl.fill_lo, wl.fill_hi, trial)
+    q, drafts = gen.independent_draft(wl.seed, trial, b, k, ms.vocab, DRAFT_LOGIT_STD)
+    forced = gen.random_tokens(wl.seed, f"forced.{trial}", (b, f), ms.vocab_offset,
+                               ms.vocab_offset + ms.vocab)
+    block = np.concatenate([forced, drafts + ms.vocab_offset], axis=1).astype(np.int32)
+    return dict(cache_len=np.tile(fills, wl.n_cfg).astype(np.int32), block=block, draft_probs=q,
+                uniforms=philox.verify_uniforms(wl.seed, trial, b, k),
+                n_draft=np.full(b, k, np.int32),
+                skip_mask=(gen.rng_for(wl.seed, f"skip.{trial}").random(b) < 0.5).astype(np.uint8),
+                gamma=np.tile(gen.rng_for(wl.seed, f"gamma.{trial}").integers(1, 6, size=b), wl.n_cfg)
+                .astype(np.int32))
+
+
+def algorithmic_bytes(wl, trials) -> dict:
+    """Bytes a step must move: every streamed weight once plus the K/V rows attention reads."""
+    ms = wl.shape
+    weights = ms.streamed_params * 2
+    t_len = wl.block_len
+    per_pos = ms.n_layers * 2 * ms.d_model * 2                 # K and V, all layers, bf16
+    kv = float(np.mean([np.sum(t["cache_len"] + t_len) for t in trials])) * per_pos
+    return {"weights": weights, "kv": kv, "total": weights + kv}
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.proc.wait()
+            self.thread.join(timeout=1)
+
+    def summary(self) -> dict:
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        reasons = sorted({n for r in self.rows if len(r) >= 7 for n, v in zip(names, r[3:7])
+                          if v.lower().startswith("active")})
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": reasons, "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# the CUDA arm
+
+
+def run_ours(args) -> None:
+    import torch
+    import torch.distributed as dist
+    from paper_2511_13587_b200 import binding as vb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    wl = CONFIGS[args.workload]
+    ms = wl.shape
+    b, cfg, k, f = wl.n_images, wl.n_cfg, wl.n_draft_max, wl.n_forced
+    r, t_len = b * cfg, wl.block_len
+    relaxed = wl.mode == MODE_RELAXED
+    seed = wl.seed + 1000 * rank                                  # replicas draw their own inputs
+
+    def dev(a):
+        a = np.ascontiguousarray(a)
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        return torch.from_numpy(a).cuda()
+
+    # resident state: weights, KV cache, neighbour table, feature cache
+    hw = gen.make_weights(ms, seed)
+    wd = {n: dev(v) for n, v in hw.items() if n != "layers"}
+    wd["layers"] = [{n: dev(v) for n, v in hw["layers"][l].items()} for l in range(ms.n_layers)]
+    del hw
+    kv_k = torch.empty((ms.n_layers, r, ms.n_heads, ms.s_max, ms.head_dim), dtype=torch.bfloat16, device="cuda")
+    kv_v = torch.empty_like(kv_k)
+    for row in range(r):
+        hk, hv = gen.make_kv_row(ms, seed, row)
+        kv_k[:, row].copy_(dev(hk))
+        kv_v[:, row].copy_(dev(hv))
+    ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, wl.nbr_k))
+    vb.vvs_bind_weights(ctx, wd)
+    if relaxed:
+        rp, col = gen.neighbour_csr(gen.make_codebook(seed, ms.vocab, wl.latent_dim), wl.nbr_k)
+        rp_d, col_d = dev(rp), dev(col)
+        vb.vvs_bind_neighbors(ctx, rp_d, col_d)
+    cap = 5 + t_len
+    fc = vb.make_fcache(torch.zeros((r, cap, ms.d_model), dtype=torch.bfloat16, device="cuda"),
+                        torch.zeros((r, cap), dtype=torch.int32, device="cuda"),
+                        torch.zeros((r,), dtype=torch.int32, device="cuda"))
+    vb.vvs_feature_cache_reset(ctx, fc)
+
+    trials = [host_trial(wl, t) for t in range(N_TRIALS)]
+    keys = ("cache_len", "block", "draft_probs", "uniforms", "n_draft", "skip_mask", "gamma")
+    dtr = [{n: dev(t[n]) for n in keys} for t in trials]
+    out = dict(accept_len=torch.zeros(b, dtype=torch.int32, device="cuda"),
+               next_token=torch.zeros(b, dtype=torch.int32, device="cuda"),
+               new_len=torch.zeros(r, dtype=torch.int32, device="cuda"),
+               n_commit=torch.zeros(r, dtype=torch.int32, device="cuda"),
+               hidden=torch.zeros((r, t_len, ms.d_model), dtype=torch.bfloat16, device="cuda"))
+    fetch_out = torch.zeros((r, 5, ms.d_model), dtype=torch.bfloat16, device="cuda")
+    fetch_pos = torch.zeros((r, 5), dtype=torch.int32, device="cuda")
+    launches = [0]
+
+    def step(inp):
+        vb.vvs_verify(ctx, n_images=b, n_cfg=cfg, n_forced=f, n_draft_max=k, block=inp["block"],
+                      n_draft=inp["n_draft"], kv_k=kv_k, kv_v=kv_v, kv_rows=r, cache_len=inp["cache_len"],
+                      draft_probs=inp["draft_probs"], uniforms=inp["uniforms"], cfg_scale=wl.cfg_scale,
+                      temperature=wl.temperature, mode=wl.mode, nbr_k=wl.nbr_k, delta=wl.delta, **out)
+        vb.vvs_feature_cache_store(ctx, fc, out["hidden"], t_len, inp["cache_len"], out["n_commit"])
+        launches[0] += vb.vvs_last_launch_count(ctx) + 1
+        if relaxed:   # workload 2: skip-masked images reuse cached features
+            vb.vvs_feature_cache_fetch(ctx, fc, inp["skip_mask"], b, inp["gamma"], 5, 0, fetch_out, fetch_pos)
+            launches[0] += 1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ---------------------------------------------------------------
+    for i in range(max(args.warmup, 3)):
+        step(dtr[i % N_TRIALS])
+    barrier()
+    launches[0] = 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        barrier()
+        e0.record()
+        for i in range(args.steps):
+            step(dtr[i % N_TRIALS])
+        e1.record()
+        barrier()
+    ms_total = e0.elapsed_time(e1)
+    gpu_launches = launches[0]
+    status = vb.vvs_device_status(ctx)
+    drafts_per_step = float(np.mean([trials[i % N_TRIALS]["n_draft"].sum() for i in range(args.steps)]))
+
+    # ---- end to end: host buffers in, host results out, every step ------------------------------
+    pin = [{n: torch.from_numpy(np.ascontiguousarray(t[n])).pin_memory() for n in keys} for t in trials[:8]]
+    stage = {n: torch.empty_like(dtr[0][n]) for n in keys}
+    res_host = {n: torch.empty(out[n].shape, dtype=out[n].dtype).pin_memory()
+                for n in ("accept_len", "next_token", "new_len")}
+    h2d = sum(v.numel() * v.element_size() for v in pin[0].values())
+    d2h = sum(v.numel() * v.element_size() for v in res_host.values())
+
+    def step_e2e(i):
+        for n in keys:
+            stage[n].copy_(pin[i % len(pin)][n], non_blocking=True)
+        step(stage)
+        for n, h in res_host.items():
+            h.copy_(out[n], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for i in range(3):
+        step_e2e(i)
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    for i in range(args.steps):
+        step_e2e(i)
+    e3.record()
+    barrier()
+    ms_e2e = e2.elapsed_time(e3)
+
+    # ---- per-kernel-class timing for the roofline (separate pass, not the headline) -----------
+    vb.vvs_profile_enable(ctx, True)
+    n_prof = min(args.steps, 8)
+    for i in range(n_prof):
+        step(dtr[i % N_TRIALS])
+    cls_ms, cls_n = vb.vvs_profile_read(ctx)
+    vb.vvs_profile_enable(ctx, False)
+
+    # ---- reduce over ranks ----------------------------------------------------------------------
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = t.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    alg = algorithmic_bytes(wl, trials)
+    gemm_launch_ms = cls_ms[0] / max(cls_n[0], 1)
+    gemm_bytes_per_launch = alg["weights"] * n_prof / max(cls_n[0], 1)
+    achieved = gemm_bytes_per_launch / (gemm_launch_ms * 1e-3) / 1e9 if gemm_launch_ms > 0 else 0.0
+    ms_step = ms_total / args.steps
+    line = {
+        "metric": "verified draft tokens/sec (LlamaGen-XL-shaped verify step)",
+        "value": world * drafts_per_step * args.steps / (ms_total * 1e-3),
+        "unit": "drafts/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_step, "verify_latency_us": ms_step * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"configs[{args.workload}] {wl.name}", "n_images": b, "n_cfg": cfg,
+                   "n_draft": k, "block_rows": t_len, "fill": f"U[{wl.fill_lo},{wl.fill_hi}] per trial",
+                   "trials": N_TRIALS, "draft": f"independent softmax(N(0,{DRAFT_LOGIT_STD}^2))",
+                   "l2": "weights streamed per step (1.47 GB) exceed the 126 MB L2; no flush needed",
+                   "parallelism": "replicas only (no collective)"},
+        "step_hbm": {"algorithmic_bytes": alg["total"], "achieved_gbs": alg["total"] / (ms_step * 1e-3) / 1e9,
+                     "frac_of_measured": alg["total"] / (ms_step * 1e-3) / 1e9 / pk["hbm_gbs"],
+                     "frac_of_8tbs": alg["total"] / (ms_step * 1e-3) / 1e9 / 8000.0},
+        "roofline": {"kernel": "projection / LM-head GEMMs (weight streaming)", "bound": "hbm",
+                     "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / pk["hbm_gbs"], "peak_source": pk["source"],
+                     "traffic": None, "launches_per_step": cls_n[0] / n_prof,
+                     "class_ms_per_step": {"gemm": cls_ms[0] / n_prof, "attention": cls_ms[1] / n_prof,
+                                           "other": cls_ms[2] / n_prof}},
+        "e2e": {"value": world * drafts_per_step * args.steps / (ms_e2e * 1e-3), "unit": "drafts/s",
+                "ms_per_step": ms_e2e / args.steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": gpu_launches, "device_status": status, "clocks": clocks.summary(),
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, steps=args.cpu_steps)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------
+# the oracle arm (CPU)
+
+
+def cpu_baseline(wl, steps: int = 2) -> dict:
+    """The fp64 numpy oracle, as it stands, on the host cores: `steps` verify steps of one image
+    (its cond and uncond sequences) of the workload."""
+    from oracle import vvs_oracle as O
+    from threadpoolctl import threadpool_info
+    ms = wl.shape
+    w = gen.make_weights(ms, wl.seed)
+    rows = [gen.make_kv_row(ms, wl.seed, c * wl.n_images) for c in range(wl.n_cfg)]
+    kv_k = np.stack([x[0] for x in rows], axis=1)
+    kv_v = np.stack([x[1] for x in rows], axis=1)
+    row_ptr = col = None
+    if wl.mode == MODE_RELAXED:
+        row_ptr, col = gen.neighbour_csr(gen.make_codebook(wl.seed, ms.vocab, wl.latent_dim), wl.nbr_k)
+    times, drafts = [], 0
+    for s in range(steps):
+        t = host_trial(wl, s)
+        cl = np.array([t["cache_len"][c * wl.n_images] for c in range(wl.n_cfg)], np.int32)
+        t0 = time.perf_counter()
+        O.verify(ms, w, t["block"][:1], wl.n_forced, t["n_draft"][:1], kv_k, kv_v, cl,
+                 t["draft_probs"][:1], t["uniforms"][:1], wl.n_cfg, wl.cfg_scale, wl.temperature,
+                 wl.mode, row_ptr, col, wl.nbr_k, wl.delta)
+        times.append(time.perf_counter() - t0)
+        drafts += int(t["n_draft"][0])
+    cores = max([i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"] or [1])
+    return {"value": drafts / sum(times), "unit": "drafts/s", "cores": cores, "kind": "oracle",
+            "sample": f"{steps} verify steps of 1 image ({wl.n_cfg} sequences) of configs[{wl_index(wl)}], "
+                      f"numpy fp64, {sum(times):.1f} s", "s_per_step": sum(times) / steps}
+
+
+def wl_index(wl) -> int:
+    return [i for i, w in CONFIGS.items() if w is wl][0]
+
+
+def run_reference(args) -> None:
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    wl = CONFIGS[args.workload]
+    n = max(1, min(args.steps, 3))
+    base = cpu_baseline(wl, steps=n)
+    line = {"impl": "reference", "metric": "verified draft tokens/sec (LlamaGen-XL-shaped verify step)",
+            "value": base["value"], "unit": "drafts/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+            "steps": n, "warmup": 0, "ms_per_step": base["s_per_step"] * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"configs[{args.workload}] {wl.name}",
+                       "sample": base["sample"]},
+            "cpu_baseline": base,
+            "e2e": {"value": base["value"], "unit": "drafts/s", "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=1, choices=[1, 2])
+    ap.add_argument("--cpu-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

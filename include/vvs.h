@@ -175,6 +175,8 @@ typedef struct vvs_verify_out {
   int32_t* next_token;  /* [B] embedding-table id sampled from norm(max(0, p - q)) at the first
                            rejected position, or from the bonus row p_{T-1} if all accepted */
   int32_t* new_len;     /* [R] cache_len + F + accept_len: fill level after the step */
+  int32_t* n_commit;    /* optional [R] F + accept_len: block rows whose K/V and features are now
+                           committed (the n_store argument of vvs_feature_cache_store) */
   uint8_t* accept_mask; /* optional [B, K] */
   float* target_probs;  /* optional [B, T, V] float32 target distributions after guidance */
   void* hidden;         /* optional T [R, T, d_model] features (final-norm output) */
@@ -239,6 +241,16 @@ int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits);
 
 /* Number of kernels the last vvs_verify / vvs_epilogue call on this context launched. */
 int vvs_last_launch_count(const vvs_ctx* ctx);
+
+/* Per-kernel-class device timing for roofline reports.  While enabled, every launch of
+ * vvs_verify / vvs_epilogue is bracketed by CUDA events on the call's stream (this costs time:
+ * never enable it around a headline measurement).  Classes: 0 = projection / LM-head GEMMs,
+ * 1 = attention, 2 = everything else.  vvs_profile_read synchronises the stream, ADDS the
+ * milliseconds and launch counts recorded since the last read to ms[3] / launches[3] (host
+ * arrays) and forgets them.  Events are created by vvs_profile_enable, not on the verify path. */
+enum { VVS_PROF_GEMM = 0, VVS_PROF_ATTENTION = 1, VVS_PROF_OTHER = 2, VVS_PROF_CLASSES = 3 };
+int vvs_profile_enable(vvs_ctx* ctx, int on);
+int vvs_profile_read(vvs_ctx* ctx, void* stream, float* ms, int32_t* launches);
 
 const char* vvs_strerror(int status);
 

@@ -53,7 +53,7 @@ class vvs_verify_args(C.Structure):
 
 
 class vvs_verify_out(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("accept_len", "next_token", "new_len", "accept_mask",
+    _fields_ = [(n, C.c_void_p) for n in ("accept_len", "next_token", "new_len", "n_commit", "accept_mask",
                                           "target_probs", "hidden", "margins")]
 
 
@@ -77,12 +77,14 @@ lib.vvs_feature_cache_fetch.argtypes = [_P, C.POINTER(vvs_fcache), _P, C.c_int32
                                         C.c_int32, _P, _P, _P]
 lib.vvs_device_status.argtypes = [_P, _P, C.POINTER(C.c_int32)]
 lib.vvs_last_launch_count.argtypes = [_P]
+lib.vvs_profile_enable.argtypes = [_P, C.c_int]
+lib.vvs_profile_read.argtypes = [_P, _P, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
 lib.vvs_strerror.argtypes = [C.c_int]
 lib.vvs_strerror.restype = C.c_char_p
 for _n in ("vvs_create", "vvs_destroy", "vvs_workspace_bytes", "vvs_bind_weights",
            "vvs_bind_neighbors", "vvs_verify", "vvs_epilogue", "vvs_feature_cache_reset",
            "vvs_feature_cache_store", "vvs_feature_cache_fetch", "vvs_device_status",
-           "vvs_last_launch_count"):
+           "vvs_last_launch_count", "vvs_profile_enable", "vvs_profile_read"):
     getattr(lib, _n).restype = C.c_int
 
 
@@ -176,19 +178,19 @@ def _args(n_images, n_cfg, n_forced, n_draft_max, block, n_draft, kv_k, kv_v, kv
                            float(temperature), int(mode), int(nbr_k), float(delta))
 
 
-def _out(accept_len, next_token, new_len, accept_mask, target_probs, hidden, margins):
-    return vvs_verify_out(_ptr(accept_len), _ptr(next_token), _ptr(new_len), _ptr(accept_mask),
+def _out(accept_len, next_token, new_len, n_commit, accept_mask, target_probs, hidden, margins):
+    return vvs_verify_out(_ptr(accept_len), _ptr(next_token), _ptr(new_len), _ptr(n_commit), _ptr(accept_mask),
                           _ptr(target_probs), _ptr(hidden), _ptr(margins))
 
 
 def vvs_verify(ctx: int, *, n_images, n_cfg, n_forced, n_draft_max, block, kv_k, kv_v, kv_rows,
                cache_len, draft_probs, uniforms, accept_len, next_token, new_len, n_draft=None,
                cache_len_host=None, cfg_scale=1.0, temperature=1.0, mode=VVS_MODE_STRICT, nbr_k=1,
-               delta=float("inf"), accept_mask=None, target_probs=None, hidden=None, margins=None,
-               stream=None) -> None:
+               delta=float("inf"), n_commit=None, accept_mask=None, target_probs=None, hidden=None,
+               margins=None, stream=None) -> None:
     a = _args(n_images, n_cfg, n_forced, n_draft_max, block, n_draft, kv_k, kv_v, kv_rows, cache_len,
               cache_len_host, draft_probs, uniforms, cfg_scale, temperature, mode, nbr_k, delta)
-    o = _out(accept_len, next_token, new_len, accept_mask, target_probs, hidden, margins)
+    o = _out(accept_len, next_token, new_len, n_commit, accept_mask, target_probs, hidden, margins)
     _check(lib.vvs_verify(ctx, C.byref(a), C.byref(o), _stream(stream)), "vvs_verify")
 
 
@@ -198,7 +200,7 @@ def vvs_epilogue(ctx: int, *, hidden_in, n_rows_per_seq, first_row, drafts, n_im
                  accept_mask=None, target_probs=None, margins=None, stream=None) -> None:
     a = _args(n_images, n_cfg, 1, n_draft_max, None, n_draft, None, None, 0, None, None, draft_probs,
               uniforms, cfg_scale, temperature, mode, nbr_k, delta)
-    o = _out(accept_len, next_token, None, accept_mask, target_probs, None, margins)
+    o = _out(accept_len, next_token, None, None, accept_mask, target_probs, None, margins)
     _check(lib.vvs_epilogue(ctx, _ptr(hidden_in), int(n_rows_per_seq), int(first_row), _ptr(drafts),
                             C.byref(a), C.byref(o), _stream(stream)), "vvs_epilogue")
 
@@ -238,3 +240,16 @@ def vvs_device_status(ctx: int, stream=None, raise_on_error: bool = False) -> in
 
 def vvs_last_launch_count(ctx: int) -> int:
     return lib.vvs_last_launch_count(ctx)
+
+
+def vvs_profile_enable(ctx: int, on: bool) -> None:
+    _check(lib.vvs_profile_enable(ctx, 1 if on else 0), "vvs_profile_enable")
+
+
+def vvs_profile_read(ctx: int, stream=None):
+    """Returns ([ms per class], [launches per class]) accumulated since the last read;
+    classes: 0 GEMM, 1 attention, 2 other."""
+    ms = (C.c_float * 3)(0, 0, 0)
+    n = (C.c_int32 * 3)(0, 0, 0)
+    _check(lib.vvs_profile_read(ctx, _stream(stream), ms, n), "vvs_profile_read")
+    return list(ms), list(n)

@@ -164,6 +164,9 @@ __global__ void accept_kernel(Workspace ws, DecideParams p) {
       p.new_len[r] = p.cache_len[r] + p.n_forced + n;
     }
   }
+  if (p.n_commit) {
+    for (int c = 0; c < p.n_cfg; ++c) p.n_commit[c * p.n_images + b] = p.n_forced + n;
+  }
   int t_sel = p.first_row + n;
   ws.sel_row[b] = (t_sel < p.rows_per_seq) ? b * p.rows_per_seq + t_sel : -1;
   ws.sel_kind[b] = (n < nd) ? 0 : 1;
@@ -335,10 +338,14 @@ __global__ void sample_kernel(Workspace ws, DecideParams p, int n_chunks) {
   if (pick < 0 && threadIdx.x == 0) p.next_token[b] = -1;
 }
 
-void launch_sample(const Workspace& ws, const DecideParams& p, cudaStream_t s) {
+void launch_residual_mass(const Workspace& ws, const DecideParams& p, cudaStream_t s) {
   int n_chunks = (p.vocab + kSampleChunk - 1) / kSampleChunk;
   dim3 grid(n_chunks, p.n_images);
   residual_mass_kernel<<<grid, kSampleChunk / 4, 0, s>>>(ws, p, n_chunks);
+}
+
+void launch_sample(const Workspace& ws, const DecideParams& p, cudaStream_t s) {
+  int n_chunks = (p.vocab + kSampleChunk - 1) / kSampleChunk;
   sample_kernel<<<p.n_images, kSampleChunk, 0, s>>>(ws, p, n_chunks);
 }
 

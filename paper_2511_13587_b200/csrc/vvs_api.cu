@@ -79,10 +79,24 @@ int check_desc(const vvs_model_desc* d) {
   return VVS_OK;
 }
 
-struct Counter {
+// Brackets one kernel launch: counts it and, when profiling, records an event pair around it.
+struct Launch {
   vvs_ctx* ctx;
-  void operator()(int n = 1) const { ctx->launches += n; }
+  cudaStream_t s;
+  int slot = -1;
+  Launch(vvs_ctx* c, int cls, cudaStream_t st) : ctx(c), s(st) {
+    if (ctx->profiling && ctx->prof_used < ctx->prof_capacity) {
+      slot = ctx->prof_used++;
+      ctx->prof_class[slot] = cls;
+      cudaEventRecord(ctx->prof_events[2 * slot], s);
+    }
+  }
+  ~Launch() {
+    ctx->launches += 1;
+    if (slot >= 0) cudaEventRecord(ctx->prof_events[2 * slot + 1], s);
+  }
 };
+#define VVS_LAUNCH(cls, call) do { Launch l__(ctx, cls, s); call; } while (0)
 
 // LM head over the codebook rows, guidance, softmax statistics, decisions.  Generic path: the
 // per-sequence logits and the guided logits live in scratch.
@@ -92,7 +106,6 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
                   cudaStream_t s) {
   const vvs_model_desc& md = ctx->desc;
   Workspace& ws = ctx->ws;
-  Counter count{ctx};
   const int B = a->n_images, C = a->n_cfg, R = B * C;
   const int M = R * rows_per_seq, V = md.vocab, BT = B * rows_per_seq;
   const T* w_lm = static_cast<const T*>(ctx->w_lm) + (size_t)md.vocab_offset * md.d_model;
@@ -108,18 +121,21 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
   p.cache_len = with_cache ? a->cache_len : nullptr; p.n_forced = a->n_forced;
   p.accept_len = o->accept_len; p.next_token = o->next_token;
   p.new_len = with_cache ? o->new_len : nullptr;
+  p.n_commit = with_cache ? o->n_commit : nullptr;
   p.accept_mask = o->accept_mask; p.margins = o->margins;
 
-  launch_gemm_nt<T>(hid, w_lm, ws.logits_raw, M, V, md.d_model, V, false, s); count();
-  launch_guide(ws.logits_raw, ws.logits, B, C, rows_per_seq, V, a->cfg_scale, 1.f / a->temperature, s);
-  count();
-  launch_row_stats(ws.logits, ws.part_m, ws.part_s, BT, V, s); count();
-  launch_finalize_stats(ws, 1, BT, s); count();
-  if (p.n_draft_max > 0) { launch_gather_logits(ws, p, s); count(); }
-  launch_accept(ws, p, s); count();
-  if (o->target_probs) { launch_probs_from_logits(ws.logits, ws, o->target_probs, BT, V, s); count(); }
-  launch_select_p_row(ws, B, V, s); count();
-  launch_sample(ws, p, s); count(2);
+  VVS_LAUNCH(VVS_PROF_GEMM, launch_gemm_nt<T>(hid, w_lm, ws.logits_raw, M, V, md.d_model, V, false, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_guide(ws.logits_raw, ws.logits, B, C, rows_per_seq, V, a->cfg_scale,
+                                          1.f / a->temperature, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_row_stats(ws.logits, ws.part_m, ws.part_s, BT, V, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_finalize_stats(ws, 1, BT, s));
+  if (p.n_draft_max > 0) VVS_LAUNCH(VVS_PROF_OTHER, launch_gather_logits(ws, p, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_accept(ws, p, s));
+  if (o->target_probs)
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_probs_from_logits(ws.logits, ws, o->target_probs, BT, V, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_select_p_row(ws, B, V, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_residual_mass(ws, p, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_sample(ws, p, s));
   return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
 }
 
@@ -127,7 +143,6 @@ template <typename T>
 int run_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, cudaStream_t s) {
   const vvs_model_desc& md = ctx->desc;
   Workspace& ws = ctx->ws;
-  Counter count{ctx};
   const int B = a->n_images, C = a->n_cfg, R = B * C, Tn = a->n_forced + a->n_draft_max;
   const int M = R * Tn, d = md.d_model, ff = md.d_ff;
   T* kv_k = static_cast<T*>(a->kv_k);
@@ -138,25 +153,27 @@ int run_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, 
   T* act = static_cast<T*>(ws.act);
   T* hid = o->hidden ? static_cast<T*>(o->hidden) : static_cast<T*>(ws.hid);
 
-  launch_embed<T>(static_cast<const T*>(ctx->tok_emb), a->block, ws.x, B, C, Tn, d, md.tok_rows,
-                  ws.status, s);
-  count();
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_embed<T>(static_cast<const T*>(ctx->tok_emb), a->block, ws.x, B, C, Tn,
+                                             d, md.tok_rows, ws.status, s));
   for (int l = 0; l < md.n_layers; ++l) {
     const Layer& L = ctx->layers[l];
-    launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm1), xn, M, d, md.rms_eps, s); count();
-    launch_gemm_nt<T>(xn, static_cast<const T*>(L.w_qkv), ws.qkv, M, 3 * d, d, 3 * d, false, s); count();
-    launch_rope_append<T>(ws.qkv, ws.rope_inv_freq, q, kv_k, kv_v, a->cache_len, md, l, a->kv_rows, R,
-                          Tn, ws.status, s);
-    count();
-    launch_attention<T>(q, kv_k, kv_v, a->cache_len, attn, md, l, a->kv_rows, R, Tn, s); count();
-    launch_gemm_nt<T>(attn, static_cast<const T*>(L.w_o), ws.x, M, d, d, d, true, s); count();
-    launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm2), xn, M, d, md.rms_eps, s); count();
-    launch_gemm_nt<T>(xn, static_cast<const T*>(L.w_gate), ws.gu, M, ff, d, 2 * ff, false, s); count();
-    launch_gemm_nt<T>(xn, static_cast<const T*>(L.w_up), ws.gu + ff, M, ff, d, 2 * ff, false, s); count();
-    launch_silu_mul<T>(ws.gu, act, M, ff, s); count();
-    launch_gemm_nt<T>(act, static_cast<const T*>(L.w_down), ws.x, M, d, ff, d, true, s); count();
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm1), xn, M, d, md.rms_eps, s));
+    VVS_LAUNCH(VVS_PROF_GEMM,
+               launch_gemm_nt<T>(xn, static_cast<const T*>(L.w_qkv), ws.qkv, M, 3 * d, d, 3 * d, false, s));
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_append<T>(ws.qkv, ws.rope_inv_freq, q, kv_k, kv_v, a->cache_len, md,
+                                                     l, a->kv_rows, R, Tn, ws.status, s));
+    VVS_LAUNCH(VVS_PROF_ATTENTION,
+               launch_attention<T>(q, kv_k, kv_v, a->cache_len, attn, md, l, a->kv_rows, R, Tn, s));
+    VVS_LAUNCH(VVS_PROF_GEMM, launch_gemm_nt<T>(attn, static_cast<const T*>(L.w_o), ws.x, M, d, d, d, true, s));
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm2), xn, M, d, md.rms_eps, s));
+    VVS_LAUNCH(VVS_PROF_GEMM,
+               launch_gemm_nt<T>(xn, static_cast<const T*>(L.w_gate), ws.gu, M, ff, d, 2 * ff, false, s));
+    VVS_LAUNCH(VVS_PROF_GEMM,
+               launch_gemm_nt<T>(xn, static_cast<const T*>(L.w_up), ws.gu + ff, M, ff, d, 2 * ff, false, s));
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_silu_mul<T>(ws.gu, act, M, ff, s));
+    VVS_LAUNCH(VVS_PROF_GEMM, launch_gemm_nt<T>(act, static_cast<const T*>(L.w_down), ws.x, M, d, ff, d, true, s));
   }
-  launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s); count();
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
   if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
   return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
 }
@@ -241,6 +258,7 @@ int vvs_create(const vvs_model_desc* desc, vvs_ctx** out) {
 
 int vvs_destroy(vvs_ctx* ctx) {
   if (!ctx) return VVS_ERR_INVALID_ARG;
+  vvs_profile_enable(ctx, 0);
   if (ctx->arena) cudaFree(ctx->arena);
   delete[] ctx->layers;
   delete ctx;
@@ -383,6 +401,49 @@ int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits) {
 }
 
 int vvs_last_launch_count(const vvs_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int vvs_profile_enable(vvs_ctx* ctx, int on) {
+  if (!ctx) return VVS_ERR_INVALID_ARG;
+  if (!on) {
+    for (int i = 0; i < 2 * ctx->prof_capacity; ++i) cudaEventDestroy(ctx->prof_events[i]);
+    delete[] ctx->prof_events;
+    delete[] ctx->prof_class;
+    ctx->prof_events = nullptr;
+    ctx->prof_class = nullptr;
+    ctx->prof_capacity = ctx->prof_used = 0;
+    ctx->profiling = false;
+    return VVS_OK;
+  }
+  if (ctx->profiling) return VVS_OK;
+  const int cap = 16384;
+  ctx->prof_events = new (std::nothrow) cudaEvent_t[2 * cap];
+  ctx->prof_class = new (std::nothrow) int[cap];
+  if (!ctx->prof_events || !ctx->prof_class) return VVS_ERR_NOMEM;
+  for (int i = 0; i < 2 * cap; ++i) {
+    if (cudaEventCreate(&ctx->prof_events[i]) != cudaSuccess) {
+      ctx->prof_capacity = i / 2;
+      vvs_profile_enable(ctx, 0);
+      return VVS_ERR_CUDA;
+    }
+  }
+  ctx->prof_capacity = cap;
+  ctx->prof_used = 0;
+  ctx->profiling = true;
+  return VVS_OK;
+}
+
+int vvs_profile_read(vvs_ctx* ctx, void* stream, float* ms, int32_t* launches) {
+  if (!ctx || !ms || !launches) return VVS_ERR_INVALID_ARG;
+  VVS_CUDA_OK(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  for (int i = 0; i < ctx->prof_used; ++i) {
+    float t = 0.f;
+    VVS_CUDA_OK(cudaEventElapsedTime(&t, ctx->prof_events[2 * i], ctx->prof_events[2 * i + 1]));
+    ms[ctx->prof_class[i]] += t;
+    launches[ctx->prof_class[i]] += 1;
+  }
+  ctx->prof_used = 0;
+  return VVS_OK;
+}
 
 const char* vvs_strerror(int status) {
   switch (status) {

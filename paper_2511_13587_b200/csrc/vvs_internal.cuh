@@ -64,6 +64,12 @@ struct vvs_ctx {
   int64_t nbr_nnz = 0;
   int device = 0;
   int launches = 0;
+  // optional per-launch event timing (vvs_profile_enable)
+  bool profiling = false;
+  cudaEvent_t* prof_events = nullptr;  // pairs (start, stop)
+  int* prof_class = nullptr;           // class of each recorded pair
+  int prof_capacity = 0;               // pairs
+  int prof_used = 0;
 };
 
 namespace vvs {
@@ -112,6 +118,7 @@ struct DecideParams {
   int32_t* accept_len;
   int32_t* next_token;
   int32_t* new_len;
+  int32_t* n_commit;
   uint8_t* accept_mask;
   float* margins;
 };
@@ -121,6 +128,7 @@ void launch_accept(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_probs_from_logits(const float* logits, const Workspace& ws, float* probs, int n_rows,
                               int v, cudaStream_t s);
 void launch_select_p_row(const Workspace& ws, int n_images, int v, cudaStream_t s);
+void launch_residual_mass(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_sample(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 
 // ---- feature cache, kernels_fcache.cu ---------------------------------------------------------

@@ -104,12 +104,20 @@ def make_weights(ms: ModelShape, seed: int, layers=None, threads: int = 8, **kw)
 # KV cache, blocks, draft distributions
 
 
-def make_kv_cache(ms: ModelShape, seed: int, n_rows: int, std: float = 1.0):
+def make_kv_row(ms: ModelShape, seed: int, row: int, std: float = 1.0):
+    """K and V of one sequence: [n_layers][n_heads][s_max][head_dim] each, own Philox streams."""
+    shp = (ms.n_layers, ms.n_heads, ms.s_max, ms.head_dim)
+    return (store(_normal(seed, f"kv.k.{row}", shp, std), ms.dtype),
+            store(_normal(seed, f"kv.v.{row}", shp, std), ms.dtype))
+
+
+def make_kv_cache(ms: ModelShape, seed: int, n_rows: int, std: float = 1.0, threads: int = 8):
     """K and V caches, layout [n_layers][n_rows][n_heads][s_max][head_dim], all slots ~N(0,1)
     (slots at and beyond a row's fill level are garbage the step must ignore or overwrite)."""
-    shp = (ms.n_layers, n_rows, ms.n_heads, ms.s_max, ms.head_dim)
-    k = store(_normal(seed, "kv.k", shp, std), ms.dtype)
-    v = store(_normal(seed, "kv.v", shp, std), ms.dtype)
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        rows = list(ex.map(lambda r: make_kv_row(ms, seed, r, std), range(n_rows)))
+    k = np.stack([r[0] for r in rows], axis=1)
+    v = np.stack([r[1] for r in rows], axis=1)
     return k, v
 
 
