@@ -202,6 +202,15 @@ int vvs_epilogue(vvs_ctx* ctx, const void* hidden, int32_t n_rows_per_seq, int32
                  const int32_t* drafts, const vvs_verify_args* args, const vvs_verify_out* out,
                  void* stream);
 
+/* Verify(logits_t, C_t) alone (Alg. 2 line 10; Sec. 2): acceptance test, accepted prefix and
+ * residual / bonus sample on target probabilities the caller already holds (guidance and
+ * softmax already applied).  target_probs is device float32 [B, n_rows_per_seq, V]; rows,
+ * first_row and drafts as in vvs_epilogue.  args->n_cfg must be 1; cfg_scale and temperature are
+ * ignored; out->new_len, n_commit, hidden and target_probs must be NULL.  Needs no weights. */
+int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, int32_t first_row,
+               const int32_t* drafts, const vvs_verify_args* args, const vvs_verify_out* out,
+               void* stream);
+
 /* Token-level feature cache (Sec. 4.3): per sequence a ring of `cap` slots holding the most
  * recent features, addressed by absolute position (slot = pos mod cap).  All arrays are
  * device memory owned by the caller; vvs_feature_cache_reset marks every slot empty. */

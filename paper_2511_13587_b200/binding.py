@@ -71,6 +71,9 @@ lib.vvs_bind_neighbors.argtypes = [_P, _P, _P, C.c_int64]
 lib.vvs_verify.argtypes = [_P, C.POINTER(vvs_verify_args), C.POINTER(vvs_verify_out), _P]
 lib.vvs_epilogue.argtypes = [_P, _P, C.c_int32, C.c_int32, _P, C.POINTER(vvs_verify_args),
                              C.POINTER(vvs_verify_out), _P]
+lib.vvs_decide.argtypes = [_P, _P, C.c_int32, C.c_int32, _P, C.POINTER(vvs_verify_args),
+                           C.POINTER(vvs_verify_out), _P]
+lib.vvs_decide.restype = C.c_int
 lib.vvs_feature_cache_reset.argtypes = [_P, C.POINTER(vvs_fcache), _P]
 lib.vvs_feature_cache_store.argtypes = [_P, C.POINTER(vvs_fcache), _P, C.c_int32, _P, _P, _P]
 lib.vvs_feature_cache_fetch.argtypes = [_P, C.POINTER(vvs_fcache), _P, C.c_int32, _P, C.c_int32,
@@ -203,6 +206,16 @@ def vvs_epilogue(ctx: int, *, hidden_in, n_rows_per_seq, first_row, drafts, n_im
     o = _out(accept_len, next_token, None, None, accept_mask, target_probs, None, margins)
     _check(lib.vvs_epilogue(ctx, _ptr(hidden_in), int(n_rows_per_seq), int(first_row), _ptr(drafts),
                             C.byref(a), C.byref(o), _stream(stream)), "vvs_epilogue")
+
+
+def vvs_decide(ctx: int, *, target_probs, n_rows_per_seq, first_row, drafts, n_images, n_draft_max,
+               draft_probs, uniforms, accept_len, next_token, n_draft=None, mode=VVS_MODE_STRICT,
+               nbr_k=1, delta=float("inf"), accept_mask=None, margins=None, stream=None) -> None:
+    a = _args(n_images, 1, 1, n_draft_max, None, n_draft, None, None, 0, None, None, draft_probs,
+              uniforms, 1.0, 1.0, mode, nbr_k, delta)
+    o = _out(accept_len, next_token, None, None, accept_mask, None, None, margins)
+    _check(lib.vvs_decide(ctx, _ptr(target_probs), int(n_rows_per_seq), int(first_row), _ptr(drafts),
+                          C.byref(a), C.byref(o), _stream(stream)), "vvs_decide")
 
 
 def make_fcache(feat: torch.Tensor, fpos: torch.Tensor, newest: torch.Tensor) -> vvs_fcache:

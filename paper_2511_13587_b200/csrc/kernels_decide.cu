@@ -78,10 +78,10 @@ __global__ void gather_logits_kernel(const float* __restrict__ logits, float* __
   }
 }
 
-void launch_gather_logits(const Workspace& ws, const DecideParams& p, cudaStream_t s) {
+void launch_gather_logits(const float* logits, const Workspace& ws, const DecideParams& p, cudaStream_t s) {
   if (p.n_draft_max == 0) return;
   dim3 grid(p.n_draft_max, p.n_images);
-  gather_logits_kernel<<<grid, 128, 0, s>>>(ws.logits, ws.l_tok, ws.l_nbr, p, ws.status);
+  gather_logits_kernel<<<grid, 128, 0, s>>>(logits, ws.l_tok, ws.l_nbr, p, ws.status);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -106,8 +106,9 @@ __global__ void accept_kernel(Workspace ws, DecideParams p) {
         if (lane == 0) atomicOr(ws.status, VVS_DEV_BAD_TOKEN);
       } else {
         int drow = b * p.rows_per_seq + p.first_row + i;
-        float m = ws.stat_m[drow], inv = ws.stat_inv[drow];
-        double mass = (double)prob_of(ws.l_tok[b * K + i], m, inv);
+        const bool direct = p.direct_probs != nullptr;
+        float m = direct ? 0.f : ws.stat_m[drow], inv = direct ? 1.f : ws.stat_inv[drow];
+        double mass = (double)(direct ? ws.l_tok[b * K + i] : prob_of(ws.l_tok[b * K + i], m, inv));
         if (p.mode == VVS_MODE_RELAXED && p.nbr_k > 1) {
           int beg = p.row_ptr[x], len = p.row_ptr[x + 1] - beg;
           if (len < 1 && lane == 0) atomicOr(ws.status, VVS_DEV_BAD_NEIGHBOUR);
@@ -117,7 +118,7 @@ __global__ void accept_kernel(Workspace ws, DecideParams p) {
           bool stop = false;
           for (int j0 = 1; j0 < kk && !stop; j0 += 32) {
             int j = j0 + lane;
-            double pn = (j < kk) ? (double)prob_of(ln[j], m, inv) : 0.0;
+            double pn = (j < kk) ? (double)(direct ? ln[j] : prob_of(ln[j], m, inv)) : 0.0;
             double tot = cum + warp_incl_scan_d(pn, lane);
             unsigned over = __ballot_sync(0xffffffffu, (j < kk) && (tot > (double)p.delta));
             if (over) {
@@ -224,7 +225,9 @@ __global__ void residual_mass_kernel(Workspace ws, DecideParams p, int n_chunks)
   int kind = ws.sel_kind[b];
   int n = p.accept_len[b];
   const float* q_row = p.draft_probs + ((size_t)b * K + (kind == 0 ? n : 0)) * V;
-  const float* p_row = ws.p_row + (size_t)b * V;
+  const int sel = ws.sel_row[b];
+  if (sel < 0) return;  // no row to sample from: sample_kernel reports -1
+  const float* p_row = p.direct_probs ? p.direct_probs + (size_t)sel * V : ws.p_row + (size_t)b * V;
   double sr = 0.0, sp = 0.0;
   int end = min(V, (c + 1) * kSampleChunk);
   for (int j = c * kSampleChunk + threadIdx.x; j < end; j += blockDim.x) {
@@ -310,7 +313,8 @@ __global__ void sample_kernel(Workspace ws, DecideParams p, int n_chunks) {
   int n = p.accept_len[b];
   int eff_kind = s_use_p ? 1 : kind;
   const float* q_row = p.draft_probs + ((size_t)b * K + (eff_kind == 0 ? n : 0)) * V;
-  const float* p_row = ws.p_row + (size_t)b * V;
+  const float* p_row = p.direct_probs ? p.direct_probs + (size_t)ws.sel_row[b] * V
+                                      : ws.p_row + (size_t)b * V;
   int j = s_chunk * kSampleChunk + threadIdx.x;
   double val = 0.0;
   if (j < V) val = (double)residual_value(p_row[j], q_row, j, eff_kind);

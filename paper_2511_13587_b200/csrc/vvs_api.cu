@@ -98,6 +98,27 @@ struct Launch {
 };
 #define VVS_LAUNCH(cls, call) do { Launch l__(ctx, cls, s); call; } while (0)
 
+DecideParams decide_params(const vvs_ctx* ctx, int rows_per_seq, int first_row, const int32_t* drafts,
+                           int drafts_ld, const vvs_verify_args* a, const vvs_verify_out* o,
+                           bool with_cache) {
+  const vvs_model_desc& md = ctx->desc;
+  DecideParams p{};
+  p.n_images = a->n_images; p.n_cfg = a->n_cfg; p.rows_per_seq = rows_per_seq; p.first_row = first_row;
+  p.n_draft_max = a->n_draft_max; p.vocab = md.vocab; p.vocab_offset = md.vocab_offset;
+  p.mode = a->mode; p.nbr_k = a->mode == VVS_MODE_RELAXED ? a->nbr_k : 1; p.kmax = md.max_nbr_k;
+  p.delta = a->delta;
+  p.drafts = drafts; p.drafts_ld = drafts_ld; p.n_draft = a->n_draft;
+  p.draft_probs = a->draft_probs; p.uniforms = a->uniforms;
+  p.row_ptr = ctx->nbr_row_ptr; p.col = ctx->nbr_col;
+  p.direct_probs = nullptr;
+  p.cache_len = with_cache ? a->cache_len : nullptr; p.n_forced = a->n_forced;
+  p.accept_len = o->accept_len; p.next_token = o->next_token;
+  p.new_len = with_cache ? o->new_len : nullptr;
+  p.n_commit = with_cache ? o->n_commit : nullptr;
+  p.accept_mask = o->accept_mask; p.margins = o->margins;
+  return p;
+}
+
 // LM head over the codebook rows, guidance, softmax statistics, decisions.  Generic path: the
 // per-sequence logits and the guided logits live in scratch.
 template <typename T>
@@ -110,26 +131,15 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
   const int M = R * rows_per_seq, V = md.vocab, BT = B * rows_per_seq;
   const T* w_lm = static_cast<const T*>(ctx->w_lm) + (size_t)md.vocab_offset * md.d_model;
 
-  DecideParams p{};
-  p.n_images = B; p.n_cfg = C; p.rows_per_seq = rows_per_seq; p.first_row = first_row;
-  p.n_draft_max = a->n_draft_max; p.vocab = V; p.vocab_offset = md.vocab_offset;
-  p.mode = a->mode; p.nbr_k = a->mode == VVS_MODE_RELAXED ? a->nbr_k : 1; p.kmax = md.max_nbr_k;
-  p.delta = a->delta;
-  p.drafts = drafts; p.drafts_ld = drafts_ld; p.n_draft = a->n_draft;
-  p.draft_probs = a->draft_probs; p.uniforms = a->uniforms;
-  p.row_ptr = ctx->nbr_row_ptr; p.col = ctx->nbr_col;
-  p.cache_len = with_cache ? a->cache_len : nullptr; p.n_forced = a->n_forced;
-  p.accept_len = o->accept_len; p.next_token = o->next_token;
-  p.new_len = with_cache ? o->new_len : nullptr;
-  p.n_commit = with_cache ? o->n_commit : nullptr;
-  p.accept_mask = o->accept_mask; p.margins = o->margins;
+  DecideParams p = decide_params(ctx, rows_per_seq, first_row, drafts, drafts_ld, a, o, with_cache);
+
 
   VVS_LAUNCH(VVS_PROF_GEMM, launch_gemm_nt<T>(hid, w_lm, ws.logits_raw, M, V, md.d_model, V, false, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_guide(ws.logits_raw, ws.logits, B, C, rows_per_seq, V, a->cfg_scale,
                                           1.f / a->temperature, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_row_stats(ws.logits, ws.part_m, ws.part_s, BT, V, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_finalize_stats(ws, 1, BT, s));
-  if (p.n_draft_max > 0) VVS_LAUNCH(VVS_PROF_OTHER, launch_gather_logits(ws, p, s));
+  if (p.n_draft_max > 0) VVS_LAUNCH(VVS_PROF_OTHER, launch_gather_logits(ws.logits, ws, p, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_accept(ws, p, s));
   if (o->target_probs)
     VVS_LAUNCH(VVS_PROF_OTHER, launch_probs_from_logits(ws.logits, ws, o->target_probs, BT, V, s));
@@ -342,6 +352,31 @@ int vvs_epilogue(vvs_ctx* ctx, const void* hidden, int32_t n_rows_per_seq, int32
                                         first_row, drafts, a->n_draft_max, a, o, false, s);
   return run_decisions<float>(ctx, static_cast<const float*>(hidden), n_rows_per_seq, first_row, drafts,
                               a->n_draft_max, a, o, false, s);
+}
+
+int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, int32_t first_row,
+               const int32_t* drafts, const vvs_verify_args* a, const vvs_verify_out* o, void* stream) {
+  if (!ctx || !target_probs || !a || !o) return VVS_ERR_INVALID_ARG;
+  if (a->n_cfg != 1) return VVS_ERR_SHAPE;  // probabilities are already guided
+  const bool was_bound = ctx->weights_bound;
+  ctx->weights_bound = true;                // no weights are read on this path
+  int rc = check_decision_args(ctx, a, o, n_rows_per_seq);
+  ctx->weights_bound = was_bound;
+  if (rc != VVS_OK) return rc;
+  if (first_row < 0 || first_row + a->n_draft_max > n_rows_per_seq) return VVS_ERR_SHAPE;
+  if (a->n_draft_max > 0 && !drafts) return VVS_ERR_INVALID_ARG;
+  if (o->new_len || o->hidden || o->n_commit || o->target_probs) return VVS_ERR_INVALID_ARG;
+  if (!aligned16(target_probs)) return VVS_ERR_ALIGN;
+  ctx->launches = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  Workspace& ws = ctx->ws;
+  DecideParams p = decide_params(ctx, n_rows_per_seq, first_row, drafts, a->n_draft_max, a, o, false);
+  p.direct_probs = target_probs;
+  if (p.n_draft_max > 0) VVS_LAUNCH(VVS_PROF_OTHER, launch_gather_logits(target_probs, ws, p, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_accept(ws, p, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_residual_mass(ws, p, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_sample(ws, p, s));
+  return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
 }
 
 static int check_fcache(const vvs_ctx* ctx, const vvs_fcache* fc) {

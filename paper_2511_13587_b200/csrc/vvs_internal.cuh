@@ -113,6 +113,8 @@ struct DecideParams {
   const float* uniforms;      // [B, K+1]
   const int32_t* row_ptr;
   const int32_t* col;
+  const float* direct_probs;  // non-null: the gathered values and the sampled rows are target
+                              // probabilities [B*rows_per_seq, V] given by the caller, not logits
   const int32_t* cache_len;   // [R] or null (epilogue entry)
   int n_forced;
   int32_t* accept_len;
@@ -123,7 +125,7 @@ struct DecideParams {
   float* margins;
 };
 void launch_finalize_stats(const Workspace& ws, int n_tiles, int n_rows, cudaStream_t s);
-void launch_gather_logits(const Workspace& ws, const DecideParams& p, cudaStream_t s);
+void launch_gather_logits(const float* logits, const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_accept(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_probs_from_logits(const float* logits, const Workspace& ws, float* probs, int n_rows,
                               int v, cudaStream_t s);
