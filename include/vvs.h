@@ -211,6 +211,38 @@ int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, 
                const int32_t* drafts, const vvs_verify_args* args, const vvs_verify_out* out,
                void* stream);
 
+/* (No counterpart in the paper: this entry point exists for deployment reasons only.)
+ * vvs_decide without a context and without any allocation.  Some callers may not call
+ * cudaMalloc at all: code that runs inside a serving process whose allocator reserved the whole
+ * GPU at start-up, a plugin whose host forbids allocations, or a latency-critical loop that
+ * cannot afford the device-wide synchronisation an allocation implies.  For them the scratch of
+ * the decision kernels lives in one fixed array in device memory that is part of the library
+ * image: about 325 KB held on every GPU that loads the library, until the process exits.  The
+ * function calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ * Capacity (larger sizes return VVS_ERR_SHAPE): n_images <= 64, n_draft_max <= 16,
+ * nbr_k <= 64, vocab <= 65536.
+ *
+ * Arguments are those of vvs_decide, with what a context would carry passed explicitly: vocab,
+ * vocab_offset, and the CSR neighbour table (device int32, may be NULL in strict mode).
+ * status_bits: optional device int32 the VVS_DEV_* bits are OR-ed into (caller clears it);
+ * NULL = a private word inside the scratch array, cleared by each call and not readable.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current) and caches it; make that first call outside any stream capture.  All
+ * calls on a device share the one array, which still holds the previous call's values (each
+ * call rewrites what it reads): two calls whose kernels may overlap on the GPU (different
+ * streams without ordering, or several host threads) race on it and must be serialised. */
+#define VVS_NOALLOC_MAX_IMAGES 64
+#define VVS_NOALLOC_MAX_DRAFTS 16
+#define VVS_NOALLOC_MAX_NBR_K 64
+#define VVS_NOALLOC_MAX_VOCAB 65536
+int vvs_decide_noalloc(const float* target_probs, int32_t vocab, int32_t vocab_offset,
+                       int32_t n_rows_per_seq, int32_t first_row, const int32_t* drafts,
+                       const int32_t* nbr_row_ptr, const int32_t* nbr_col,
+                       const vvs_verify_args* args, const vvs_verify_out* out,
+                       int32_t* status_bits, void* stream);
+
 /* Token-level feature cache (Sec. 4.3): per sequence a ring of `cap` slots holding the most
  * recent features, addressed by absolute position (slot = pos mod cap).  All arrays are
  * device memory owned by the caller; vvs_feature_cache_reset marks every slot empty. */
