@@ -43,6 +43,15 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
     c.take(ws.gu, M * 2 * ff * 4);
     c.take(ws.act, M * ff * es);
     c.take(ws.hid, M * dm * es);
+    if (d.dtype == VVS_DTYPE_BF16) {
+      const size_t wide = 3 * dm > 2 * ff ? 3 * dm : 2 * ff;
+      const size_t tiles = (wide + 127) / 128, passes = (M + 255) / 256;
+      c.take(ws.slot_pos, M * 4);
+      c.take(ws.rope_cos, M * (size_t)(d.head_dim / 2) * 4);
+      c.take(ws.rope_sin, M * (size_t)(d.head_dim / 2) * 4);
+      c.take(ws.sk_scratch, M * wide * 4);
+      c.take(ws.sk_counters, tiles * passes * 4);
+    }
   }
   c.take(ws.logits_raw, M * V * 4);
   c.take(ws.logits, M * V * 4);
@@ -134,7 +143,21 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
   DecideParams p = decide_params(ctx, rows_per_seq, first_row, drafts, drafts_ld, a, o, with_cache);
 
 
-  VVS_LAUNCH(VVS_PROF_GEMM, launch_gemm_nt<T>(hid, w_lm, ws.logits_raw, M, V, md.d_model, V, false, s));
+  if (ctx->tensor_core_path) {
+    const GemmTcPlan plan = plan_gemm_tc(M, V, md.d_model, false, false, ctx->n_sms);
+    CUtensorMap tm_hid;
+    if (make_tmap_bf16_2d(&tm_hid, hid, (uint64_t)M, (uint64_t)md.d_model, (uint32_t)plan.nt) != VVS_OK)
+      return VVS_ERR_CUDA;
+    GemmTcArgs g{};
+    g.m = M; g.n = V; g.k = md.d_model;
+    g.tm_a = &ctx->lm_map; g.tm_b = &tm_hid; g.pdl = ctx->use_pdl; g.status = ws.status;
+    g.out = ws.logits_raw; g.ldo = V;
+    int rc = VVS_OK;
+    VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_STORE, plan, g, s));
+    if (rc != VVS_OK) return rc;
+  } else {
+    VVS_LAUNCH(VVS_PROF_GEMM, launch_gemm_nt<T>(hid, w_lm, ws.logits_raw, M, V, md.d_model, V, false, s));
+  }
   VVS_LAUNCH(VVS_PROF_OTHER, launch_guide(ws.logits_raw, ws.logits, B, C, rows_per_seq, V, a->cfg_scale,
                                           1.f / a->temperature, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_row_stats(ws.logits, ws.part_m, ws.part_s, BT, V, s));
@@ -183,6 +206,77 @@ int run_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, 
     VVS_LAUNCH(VVS_PROF_OTHER, launch_silu_mul<T>(ws.gu, act, M, ff, s));
     VVS_LAUNCH(VVS_PROF_GEMM, launch_gemm_nt<T>(act, static_cast<const T*>(L.w_down), ws.x, M, d, ff, d, true, s));
   }
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
+  if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
+  return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
+}
+
+// bf16 contexts: projections on the tensor cores (gemm_tc.cu), everything else as above.
+int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, cudaStream_t s) {
+  using T = __nv_bfloat16;
+  const vvs_model_desc& md = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const int B = a->n_images, C = a->n_cfg, R = B * C, Tn = a->n_forced + a->n_draft_max;
+  const int M = R * Tn, d = md.d_model, ff = md.d_ff;
+  T* kv_k = static_cast<T*>(a->kv_k);
+  T* kv_v = static_cast<T*>(a->kv_v);
+  T* xn = static_cast<T*>(ws.xn);
+  T* q = static_cast<T*>(ws.q);
+  T* attn = static_cast<T*>(ws.attn);
+  T* act = static_cast<T*>(ws.act);
+  T* hid = o->hidden ? static_cast<T*>(o->hidden) : static_cast<T*>(ws.hid);
+
+  const GemmTcPlan p_qkv = plan_gemm_tc(M, 3 * d, d, false, true, ctx->n_sms);
+  const GemmTcPlan p_o = plan_gemm_tc(M, d, d, false, true, ctx->n_sms);
+  const GemmTcPlan p_gu = plan_gemm_tc(M, ff, d, true, true, ctx->n_sms);
+  const GemmTcPlan p_down = plan_gemm_tc(M, d, ff, false, true, ctx->n_sms);
+  CUtensorMap tm_xn, tm_attn, tm_act;
+  if (make_tmap_bf16_2d(&tm_xn, xn, (uint64_t)M, (uint64_t)d, (uint32_t)p_qkv.nt) != VVS_OK ||
+      make_tmap_bf16_2d(&tm_attn, attn, (uint64_t)M, (uint64_t)d, (uint32_t)p_o.nt) != VVS_OK ||
+      make_tmap_bf16_2d(&tm_act, act, (uint64_t)M, (uint64_t)ff, (uint32_t)p_down.nt) != VVS_OK)
+    return VVS_ERR_CUDA;
+
+  GemmTcArgs base{};
+  base.m = M; base.pdl = ctx->use_pdl; base.status = ws.status;
+  base.scratch = ws.sk_scratch; base.counters = ws.sk_counters;
+  base.q = q; base.kv_k = kv_k; base.kv_v = kv_v; base.slot_pos = ws.slot_pos;
+  base.rope_cos = ws.rope_cos; base.rope_sin = ws.rope_sin;
+  base.d = d; base.n_heads = md.n_heads; base.hd = md.head_dim; base.s_max = md.s_max;
+  base.kv_rows = a->kv_rows; base.t_len = Tn; base.act = act; base.ff = ff;
+
+  int rc = VVS_OK;
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_embed<T>(static_cast<const T*>(ctx->tok_emb), a->block, ws.x, B, C, Tn,
+                                             d, md.tok_rows, ws.status, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, ws, md, R, Tn, s));
+  for (int l = 0; l < md.n_layers && rc == VVS_OK; ++l) {
+    const Layer& L = ctx->layers[l];
+    const LayerMaps& W = ctx->layer_maps[l];
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm1), xn, M, d, md.rms_eps, s));
+    {
+      GemmTcArgs g = base;
+      g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.ld_scratch = 3 * d; g.layer = l;
+      VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_QKV, p_qkv, g, s));
+    }
+    VVS_LAUNCH(VVS_PROF_ATTENTION,
+               launch_attention<T>(q, kv_k, kv_v, a->cache_len, attn, md, l, a->kv_rows, R, Tn, s));
+    if (rc == VVS_OK) {
+      GemmTcArgs g = base;
+      g.n = d; g.k = d; g.tm_a = &W.w_o; g.tm_b = &tm_attn; g.out = ws.x; g.ldo = d;
+      VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_o, g, s));
+    }
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm2), xn, M, d, md.rms_eps, s));
+    if (rc == VVS_OK) {
+      GemmTcArgs g = base;
+      g.n = ff; g.k = d; g.tm_a = &W.w_gate; g.tm_a2 = &W.w_up; g.tm_b = &tm_xn; g.ld_scratch = 2 * ff;
+      VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_SWIGLU, p_gu, g, s));
+    }
+    if (rc == VVS_OK) {
+      GemmTcArgs g = base;
+      g.n = d; g.k = ff; g.tm_a = &W.w_down; g.tm_b = &tm_act; g.out = ws.x; g.ldo = d;
+      VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_down, g, s));
+    }
+  }
+  if (rc != VVS_OK) return rc;
   VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
   if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
   return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
@@ -260,8 +354,16 @@ int vvs_create(const vvs_model_desc* desc, vvs_ctx** out) {
   }
   if (desc->n_layers > 0) {
     ctx->layers = new (std::nothrow) Layer[desc->n_layers]();
-    if (!ctx->layers) { vvs_destroy(ctx); return VVS_ERR_NOMEM; }
+    ctx->layer_maps = new (std::nothrow) LayerMaps[desc->n_layers]();
+    if (!ctx->layers || !ctx->layer_maps) { vvs_destroy(ctx); return VVS_ERR_NOMEM; }
   }
+  // Debug switches only: VVS_DEBUG_GENERIC runs bf16 contexts on the generic kernels,
+  // VVS_DEBUG_NO_PDL launches the tensor-core GEMMs without programmatic dependent launch.
+  ctx->tensor_core_path = desc->dtype == VVS_DTYPE_BF16 && !std::getenv("VVS_DEBUG_GENERIC");
+  ctx->use_pdl = !std::getenv("VVS_DEBUG_NO_PDL");
+  if (cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess ||
+      ctx->n_sms < 1)
+    ctx->n_sms = 148;
   *out = ctx;
   return VVS_OK;
 }
@@ -271,6 +373,7 @@ int vvs_destroy(vvs_ctx* ctx) {
   vvs_profile_enable(ctx, 0);
   if (ctx->arena) cudaFree(ctx->arena);
   delete[] ctx->layers;
+  delete[] ctx->layer_maps;
   delete ctx;
   return VVS_OK;
 }
@@ -295,6 +398,25 @@ int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w) {
       const vvs_layer_weights& s = w->layers[l];
       ctx->layers[l] = Layer{s.w_qkv, s.w_o, s.w_gate, s.w_up, s.w_down, s.norm1, s.norm2};
     }
+  }
+  if (ctx->tensor_core_path) {
+    const vvs_model_desc& md = ctx->desc;
+    const int d = md.d_model, ff = md.d_ff;
+    int rc = VVS_OK;
+    for (int l = 0; l < n && rc == VVS_OK; ++l) {
+      const vvs_layer_weights& s = w->layers[l];
+      LayerMaps& m = ctx->layer_maps[l];
+      rc = make_weight_tmap(&m.w_qkv, s.w_qkv, 3 * d, d);
+      if (rc == VVS_OK) rc = make_weight_tmap(&m.w_o, s.w_o, d, d);
+      if (rc == VVS_OK) rc = make_weight_tmap(&m.w_gate, s.w_gate, ff, d);
+      if (rc == VVS_OK) rc = make_weight_tmap(&m.w_up, s.w_up, ff, d);
+      if (rc == VVS_OK) rc = make_weight_tmap(&m.w_down, s.w_down, d, ff);
+    }
+    if (rc == VVS_OK)
+      rc = make_weight_tmap(&ctx->lm_map,
+                            static_cast<const __nv_bfloat16*>(w->w_lm) + (size_t)md.vocab_offset * d,
+                            md.vocab, d);
+    if (rc != VVS_OK) return rc;
   }
   ctx->tok_emb = w->tok_emb;
   ctx->norm_f = w->norm_f;
@@ -331,6 +453,7 @@ int vvs_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, 
   }
   ctx->launches = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (ctx->tensor_core_path) return run_verify_tc(ctx, a, o, s);
   return md.dtype == VVS_DTYPE_BF16 ? run_verify<__nv_bfloat16>(ctx, a, o, s)
                                     : run_verify<float>(ctx, a, o, s);
 }

@@ -1,6 +1,7 @@
 // Internal declarations of the verify-step library: context, scratch layout, launchers.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -40,11 +41,22 @@ struct Workspace {
   double* r_part = nullptr;  // [B, n_chunks] per-chunk residual mass
   double* p_part = nullptr;  // [B, n_chunks] per-chunk target mass (fallback when residual is 0)
   float* rope_inv_freq = nullptr;  // [head_dim/2] angle per unit coordinate of each pair
+  // tensor-core path
+  int32_t* slot_pos = nullptr;   // [M] cache slot of each block row, -1 if its sequence overflows
+  float* rope_cos = nullptr;     // [M, head_dim/2]
+  float* rope_sin = nullptr;     // [M, head_dim/2]
+  float* sk_scratch = nullptr;   // [M, max(3d, 2ff)] fp32 split-K sums; all zero between kernels
+  int* sk_counters = nullptr;    // [passes, tiles] split-K arrival counters; zero between kernels
   int32_t* status = nullptr; // device status word
 };
 
 struct Layer {
   const void *w_qkv, *w_o, *w_gate, *w_up, *w_down, *norm1, *norm2;
+};
+
+// TMA descriptors of one layer's projection matrices (bf16 contexts)
+struct LayerMaps {
+  CUtensorMap w_qkv, w_o, w_gate, w_up, w_down;
 };
 
 }  // namespace vvs
@@ -59,6 +71,11 @@ struct vvs_ctx {
   const void* norm_f = nullptr;
   const void* w_lm = nullptr;
   vvs::Layer* layers = nullptr;  // host array [n_layers]
+  bool tensor_core_path = false;     // bf16 contexts unless VVS_DEBUG_GENERIC is set
+  bool use_pdl = true;               // programmatic dependent launch of the tensor-core GEMMs
+  vvs::LayerMaps* layer_maps = nullptr;  // host array [n_layers]
+  CUtensorMap lm_map;
+  int n_sms = 148;
   const int32_t* nbr_row_ptr = nullptr;
   const int32_t* nbr_col = nullptr;
   int64_t nbr_nnz = 0;
@@ -100,6 +117,31 @@ void launch_guide(const float* raw, float* logits, int n_images, int n_cfg, int 
                   float cfg_scale, float inv_temp, cudaStream_t s);
 void launch_row_stats(const float* logits, float* part_m, float* part_s, int n_rows, int v,
                       cudaStream_t s);
+
+// ---- tensor-core projection GEMM, gemm_tc.cu ----------------------------------------------------
+enum { GEMM_EPI_STORE = 0, GEMM_EPI_ADD = 1, GEMM_EPI_QKV = 2, GEMM_EPI_SWIGLU = 3 };
+struct GemmTcPlan {
+  int nt, passes, tiles, kb_total, splits, stages, smem_bytes, tmem_cols;
+};
+struct GemmTcArgs {
+  int m, n, k;                 // tokens, weight rows (per matrix), reduction length
+  const CUtensorMap* tm_a;     // weights [n, k]
+  const CUtensorMap* tm_a2;    // second weight matrix (SWIGLU: up), else null
+  const CUtensorMap* tm_b;     // activations [m, k], box rows = plan.nt
+  bool pdl;
+  float* scratch; int ld_scratch; int* counters; int32_t* status;
+  float* out; int ldo;         // STORE / ADD
+  __nv_bfloat16* q; __nv_bfloat16* kv_k; __nv_bfloat16* kv_v;  // QKV
+  const int32_t* slot_pos; const float* rope_cos; const float* rope_sin;
+  int d, n_heads, hd, s_max, layer, kv_rows, t_len;
+  __nv_bfloat16* act; int ff;  // SWIGLU
+};
+int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+int make_weight_tmap(CUtensorMap* out, const void* w, int rows, int cols);
+GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_sms);
+int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStream_t s);
+void launch_rope_table(const int32_t* cache_len, const Workspace& ws, const vvs_model_desc& md, int n_rows,
+                       int t_len, cudaStream_t s);
 
 // ---- decision stage, kernels_decide.cu -----------------------------------------------------
 struct DecideParams {

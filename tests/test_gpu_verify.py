@@ -177,14 +177,47 @@ def test_device_side_checks_report_instead_of_faulting():
     run.close()
 
 
-def test_deterministic_across_calls():
+def test_repeatable_across_calls():
+    """Two calls on the same inputs: the float32 context is bitwise repeatable; the bf16 context
+    adds split-K partial sums with float atomics, so its low bits (and, through bf16 rounding of
+    activations, ~1e-2 of a probability) may move, but every decision must replay exactly on the
+    probabilities of its own call."""
     ms = XL_SMALL
     case = H.build_case(ms, 71, 2, 2, 1, 8, [50, 400])
     run = H.GpuRunner(ms, case["w"], 4, 9)
     a = run.verify(case)
     b = run.verify(case)
-    for key in ("accept_len", "next_token", "accept_mask", "new_len"):
-        np.testing.assert_array_equal(a[key], b[key])
-    np.testing.assert_array_equal(a["target_probs"], b["target_probs"])
-    np.testing.assert_array_equal(a["hidden"], b["hidden"])
+    np.testing.assert_allclose(a["target_probs"], b["target_probs"], rtol=5e-2, atol=1e-7)
+    assert H.rel_err_rows(a["hidden"], b["hidden"]) < 1e-2
+    H.check_replay(case, a)
+    H.check_replay(case, b)
     run.close()
+    w = CONFIGS[0]
+    case = H.build_case(w.shape, w.seed, 1, 1, 1, 4, [64], cfg_scale=1.0)
+    run = H.GpuRunner(w.shape, case["w"], 1, 5)
+    a = run.verify(case)
+    b = run.verify(case)
+    for key in ("accept_len", "next_token", "accept_mask", "new_len", "target_probs", "hidden"):
+        np.testing.assert_array_equal(a[key], b[key])
+    run.close()
+
+
+def test_tensor_core_path_agrees_with_generic_kernels(monkeypatch):
+    """The same bf16 step through the generic kernels (debug switch) and through the tensor-core
+    GEMMs: both within tolerance of the oracle and of each other."""
+    ms = XL_SMALL
+    case = H.build_case(ms, 81, 2, 2, 1, 8, [7, 222])
+    run = H.GpuRunner(ms, case["w"], 4, 9)
+    fast = run.verify(case)
+    run.close()
+    monkeypatch.setenv("VVS_DEBUG_GENERIC", "1")
+    run = H.GpuRunner(ms, case["w"], 4, 9)
+    slow = run.verify(case)
+    run.close()
+    monkeypatch.delenv("VVS_DEBUG_GENERIC")
+    assert slow["launches"] != fast["launches"]
+    assert H.rel_err_rows(fast["hidden"], slow["hidden"]) < 1e-2
+    np.testing.assert_allclose(fast["target_probs"], slow["target_probs"], rtol=6e-2, atol=1e-7)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, slow, ora)
+    _check_end_to_end(case, fast, ora)
