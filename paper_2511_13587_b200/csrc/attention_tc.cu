@@ -1,0 +1,339 @@
+// Block-vs-cache attention of the verify step on the 5th-generation tensor cores (bf16).
+//
+// Sequence r, head h: the T <= 32 block rows (queries) attend cache slots [0, L_r + t].  The key
+// range is cut into chunks of 128 keys, one CTA per (chunk, head, sequence) (flash-decoding
+// style split-KV), so a batch-1 step still fills the GPU and every CTA is a single shot:
+//   1. TMA stages the K chunk [128 keys x hd], the V chunk and the Q rows in 128-byte-swizzled
+//      shared memory (chunks that lie entirely in the old cache are requested before
+//      griddepcontrol.wait, i.e. while the QKV projection is still running).
+//   2. S^T = K Q^T  (tcgen05.mma, M = 128 keys, N = 16/32 queries) into TMEM.
+//   3. Each thread owns one key: scale, causal mask, per-query max / sum over the 128 keys by
+//      warp shuffles + shared memory, P = exp(S - max) written as bf16 into swizzled shared
+//      memory.  V rows of masked-out keys are zeroed so stale cache contents cannot leak.
+//   4. O = P V  (tcgen05.mma, M = 128 (rows >= T are don't-care), N = hd, V as MN-major operand).
+//   5. Query rows write (max, sum, O) partials; the CTA that arrives last for (r, h) merges the
+//      chunks (exact softmax re-normalisation) and writes the bf16 attention output.  No CTA
+//      waits for another.
+#include <math_constants.h>
+
+#include "tc_common.cuh"
+#include "vvs_internal.cuh"
+
+namespace vvs {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kChunkKeys = 128;
+
+struct AttnParams {
+  const int32_t* cache_len;
+  __nv_bfloat16* out;     // [M, d]
+  float* part_o;          // [R*H, n_chunks_max, T, hd]
+  float* part_ml;         // [R*H, n_chunks_max, T, 2]
+  int* counters;          // [R*H]
+  int32_t* status;
+  int d, n_heads, hd, s_max, layer, kv_rows, t_len, tq, n_chunks_max;
+  uint32_t tmem_cols;
+  float scale;
+};
+
+__device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity) { return mbar_wait(bar, parity); }
+
+// MN-major bf16 operand whose 64-element (128-byte) rows are 128-byte swizzled, one row per K
+// index: 8-row groups 1024 bytes apart (stride offset), 64-element column chunks lbo bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t saddr, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr >> 4) & 0x3FFF);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+
+__device__ __forceinline__ float warp_max_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(128)
+attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q,
+                    const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v) {
+  constexpr int NC = HD / 64;                       // 64-column chunks of the head dimension
+  constexpr uint32_t kKVBytes = kChunkKeys * 128;   // one 64-column chunk of a K or V tile
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_kq, bar_v, bar_s, bar_o;
+  __shared__ uint32_t tmem_slot;
+  __shared__ float red_max[4][32];
+  __shared__ float red_sum[4][32];
+  __shared__ int s_last;
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sK = smem;
+  uint8_t* sV = sK + NC * kKVBytes;
+  uint8_t* sP = sV + NC * kKVBytes;                 // 2 chunks of 64 keys: [128 rows x 128 B] each
+  uint8_t* sQ = sP + 2 * kKVBytes;                  // NC chunks: [tq rows x 128 B]
+  const uint32_t q_chunk_bytes = (uint32_t)p.tq * 128u;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int c = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
+  const int T = p.t_len;
+
+  if (tid == 0) {
+    mbar_init(&bar_kq, 1);
+    mbar_init(&bar_v, 1);
+    mbar_init(&bar_s, 1);
+    mbar_init(&bar_o, 1);
+    fence_barrier_init();
+    tma_prefetch_desc(&tm_q);
+    tma_prefetch_desc(&tm_k);
+    tma_prefetch_desc(&tm_v);
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_slot, p.tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
+  pdl_launch_dependents();
+
+  const int fill = p.cache_len[r];                  // written by earlier steps, not by the previous kernel
+  const bool ok = fill >= 0 && fill + T <= p.s_max;
+  const int n_keys = fill + T;
+  const int n_chunks = ok ? (n_keys + kChunkKeys - 1) / kChunkKeys : 0;
+  const int key0 = c * kChunkKeys;
+  bool active = ok && c < n_chunks;
+  const int row_base = ((p.layer * p.kv_rows + r) * p.n_heads + h) * p.s_max + key0;
+  const bool old_only = key0 + kChunkKeys <= fill;  // chunk holds no row written by this step
+
+  if (!ok && c == 0) {                              // overflowing sequence: defined (zero) output
+    pdl_wait();
+    for (int i = tid; i < T * HD; i += blockDim.x)
+      p.out[((size_t)r * T + i / HD) * p.d + (size_t)h * HD + i % HD] = __float2bfloat16_rn(0.f);
+  }
+
+  bool alive = active;
+  if (active && tid == 0) {
+    mbar_expect_tx(&bar_kq, NC * kKVBytes + NC * q_chunk_bytes);
+    mbar_expect_tx(&bar_v, NC * kKVBytes);
+    if (old_only) {
+      for (int j = 0; j < NC; ++j) tma_load_2d(sK + j * kKVBytes, &tm_k, &bar_kq, j * 64, row_base);
+      for (int j = 0; j < NC; ++j) tma_load_2d(sV + j * kKVBytes, &tm_v, &bar_v, j * 64, row_base);
+    }
+    pdl_wait();
+    for (int j = 0; j < NC; ++j) tma_load_2d(sQ + j * q_chunk_bytes, &tm_q, &bar_kq, h * HD + j * 64, r * T);
+    if (!old_only) {
+      for (int j = 0; j < NC; ++j) tma_load_2d(sK + j * kKVBytes, &tm_k, &bar_kq, j * 64, row_base);
+      for (int j = 0; j < NC; ++j) tma_load_2d(sV + j * kKVBytes, &tm_v, &bar_v, j * 64, row_base);
+    }
+  }
+  if (active && warp == 1 && lane == 0) {
+    // S^T[key, query] = sum_e K[key, e] Q[query, e]
+    if (wait_bounded(&bar_kq, 0)) {
+      tc_fence_after();
+      const uint32_t idesc = idesc_bf16_f32(128, (uint32_t)p.tq);
+#pragma unroll
+      for (int k16 = 0; k16 < HD / 16; ++k16) {
+        const uint32_t a = smem_u32(sK + (k16 / 4) * kKVBytes) + (k16 % 4) * 32;
+        const uint32_t b = smem_u32(sQ + (k16 / 4) * q_chunk_bytes) + (k16 % 4) * 32;
+        mma_bf16(tmem_base, smem_desc_sw128(a), smem_desc_sw128(b), idesc, k16 > 0 ? 1u : 0u);
+      }
+      mma_commit(&bar_s);
+    } else {
+      atomicOr(p.status, VVS_DEV_TIMEOUT);
+    }
+  }
+  __syncwarp();
+  pdl_wait();
+
+  if (active) {
+    const bool got = wait_bounded(&bar_s, 0);
+    if (__syncthreads_or(got ? 0 : 1)) {
+      if (tid == 0) atomicOr(p.status, VVS_DEV_TIMEOUT);
+      alive = false;
+    }
+  }
+  if (alive) {
+    tc_fence_after();
+    const int key = key0 + tid;
+    const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
+    float s[32];
+    tmem_ld16(t_row, s);
+    if (p.tq > 16) tmem_ld16(t_row + 16, s + 16);
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+      if (t < T) {
+        const bool valid = key <= fill + t;
+        s[t] = valid ? s[t] * p.scale : -CUDART_INF_F;
+        const float wm = warp_max_f(s[t]);
+        if (lane == 0) red_max[warp][t] = wm;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+      if (t < T) {
+        const float m = fmaxf(fmaxf(red_max[0][t], red_max[1][t]), fmaxf(red_max[2][t], red_max[3][t]));
+        const float e = (s[t] == -CUDART_INF_F) ? 0.f : expf(s[t] - m);
+        s[t] = e;
+        const float ws = warp_sum_f(e);
+        if (lane == 0) red_sum[warp][t] = ws;
+        // P[t, key] as bf16, K-major rows of 64 keys with the 128-byte swizzle
+        const uint32_t kk = (uint32_t)tid & 63u;
+        uint8_t* dst = sP + (tid >> 6) * kKVBytes + t * 128 + ((((kk >> 3) ^ ((uint32_t)t & 7u)) << 4) | ((kk & 7u) << 1));
+        *reinterpret_cast<__nv_bfloat16*>(dst) = __float2bfloat16_rn(e);
+      }
+    }
+    // V rows of keys that no query may see: cleared, so unwritten cache slots cannot inject NaN
+    if (!wait_bounded(&bar_v, 0)) atomicOr(p.status, VVS_DEV_TIMEOUT);
+    if (key >= n_keys) {
+#pragma unroll
+      for (int j = 0; j < NC; ++j) {
+        uint4* row = reinterpret_cast<uint4*>(sV + j * kKVBytes + tid * 128);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) row[i] = make_uint4(0, 0, 0, 0);
+      }
+    }
+    fence_proxy_async();      // generic-proxy writes of P and V visible to the tensor core
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1 && lane == 0) {
+      // O[query, e] = sum_key P[query, key] V[key, e]
+      const uint32_t idesc = idesc_bf16_f32(128, (uint32_t)HD) | (1u << 16);  // B is MN-major
+#pragma unroll
+      for (int k16 = 0; k16 < kChunkKeys / 16; ++k16) {
+        const uint32_t a = smem_u32(sP + (k16 / 4) * kKVBytes) + (k16 % 4) * 32;
+        const uint32_t b = smem_u32(sV) + k16 * 2048;
+        mma_bf16(tmem_base + 32, smem_desc_sw128(a), smem_desc_mn_sw128(b, kKVBytes), idesc, k16 > 0 ? 1u : 0u);
+      }
+      mma_commit(&bar_o);
+    }
+    __syncwarp();
+    const bool got = wait_bounded(&bar_o, 0);
+    if (__syncthreads_or(got ? 0 : 1)) {
+      if (tid == 0) atomicOr(p.status, VVS_DEV_TIMEOUT);
+      alive = false;
+    }
+  }
+  if (alive) {
+    tc_fence_after();
+    const size_t rh = (size_t)r * p.n_heads + h;
+    if (warp == 0) {                                  // TMEM lanes 0..31 = query rows
+      const uint32_t t_row = tmem_base + 32;
+      float* po = p.part_o + ((rh * p.n_chunks_max + c) * T + lane) * HD;
+      // chunk-wide max and sum of query `lane` (the four warps' reductions are still in place)
+      const float mine_max = fmaxf(fmaxf(red_max[0][lane], red_max[1][lane]), fmaxf(red_max[2][lane], red_max[3][lane]));
+      const float mine_sum = red_sum[0][lane] + red_sum[1][lane] + red_sum[2][lane] + red_sum[3][lane];
+      for (int e0 = 0; e0 < HD; e0 += 16) {
+        float o[16];
+        tmem_ld16(t_row + e0, o);
+        if (lane < T) {
+          if (n_chunks == 1) {
+            const float inv = 1.f / mine_sum;
+            __nv_bfloat16* dst = p.out + ((size_t)r * T + lane) * p.d + (size_t)h * HD + e0;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) dst[i] = __float2bfloat16_rn(o[i] * inv);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) po[e0 + i] = o[i];
+          }
+        }
+      }
+      if (lane < T && n_chunks > 1) {
+        float* ml = p.part_ml + ((rh * p.n_chunks_max + c) * T + lane) * 2;
+        ml[0] = mine_max;
+        ml[1] = mine_sum;
+      }
+    }
+    if (n_chunks > 1) {
+      __threadfence();
+      __syncthreads();
+      if (tid == 0) {
+        const int prev = atomicAdd(&p.counters[rh], 1);
+        s_last = (prev == n_chunks - 1) ? 1 : 0;
+      }
+      __syncthreads();
+      if (s_last) {
+        __threadfence();
+        for (int i = tid; i < T * HD; i += blockDim.x) {
+          const int t = i / HD, e = i - t * HD;
+          float m = -CUDART_INF_F;
+          for (int cc = 0; cc < n_chunks; ++cc)
+            m = fmaxf(m, __ldcg(p.part_ml + ((rh * p.n_chunks_max + cc) * T + t) * 2));
+          float num = 0.f, den = 0.f;
+          for (int cc = 0; cc < n_chunks; ++cc) {
+            const float* ml = p.part_ml + ((rh * p.n_chunks_max + cc) * T + t) * 2;
+            const float mc = __ldcg(ml);
+            const float w = (mc == -CUDART_INF_F) ? 0.f : expf(mc - m);
+            den += w * __ldcg(ml + 1);
+            num += w * __ldcg(p.part_o + ((rh * p.n_chunks_max + cc) * T + t) * HD + e);
+          }
+          p.out[((size_t)r * T + t) * p.d + (size_t)h * HD + e] = __float2bfloat16_rn(num / den);
+        }
+        if (tid == 0) p.counters[rh] = 0;
+      }
+    }
+  }
+  // ---- teardown ---------------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
+}
+
+}  // namespace
+
+int launch_attention_tc(const AttentionTcArgs& a, cudaStream_t s) {
+  AttnParams p{};
+  p.cache_len = a.cache_len; p.out = a.out; p.part_o = a.part_o; p.part_ml = a.part_ml;
+  p.counters = a.counters; p.status = a.status;
+  p.d = a.d; p.n_heads = a.n_heads; p.hd = a.hd; p.s_max = a.s_max; p.layer = a.layer;
+  p.kv_rows = a.kv_rows; p.t_len = a.t_len; p.tq = a.t_len <= 16 ? 16 : 32;
+  p.n_chunks_max = (a.s_max + kChunkKeys - 1) / kChunkKeys;
+  p.tmem_cols = a.hd == 64 ? 128u : 256u;
+  p.scale = 1.0f / sqrtf((float)a.hd);
+  const int nc = a.hd / 64;
+  const int smem = nc * 2 * kChunkKeys * 128 + 2 * kChunkKeys * 128 + nc * 32 * 128 + 1024;
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.n_chunks_max, a.n_heads, a.n_rows);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = a.pdl ? 1 : 0;
+  cudaError_t e;
+  static bool configured64 = false, configured128 = false;
+  if (a.hd == 64) {
+    if (!configured64) {
+      if (cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return VVS_ERR_CUDA;
+      configured64 = true;
+    }
+    e = cudaLaunchKernelEx(&cfg, attention_tc_kernel<64>, p, *a.tm_q, *a.tm_k, *a.tm_v);
+  } else {
+    if (!configured128) {
+      if (cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return VVS_ERR_CUDA;
+      configured128 = true;
+    }
+    e = cudaLaunchKernelEx(&cfg, attention_tc_kernel<128>, p, *a.tm_q, *a.tm_k, *a.tm_v);
+  }
+  return e == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+}
+
+}  // namespace vvs

@@ -51,6 +51,10 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
       c.take(ws.rope_sin, M * (size_t)(d.head_dim / 2) * 4);
       c.take(ws.sk_scratch, M * wide * 4);
       c.take(ws.sk_counters, tiles * passes * 4);
+      const size_t chunks = ((size_t)d.s_max + 127) / 128, rh = (size_t)d.max_rows * d.n_heads;
+      c.take(ws.attn_part_o, rh * chunks * d.max_block * d.head_dim * 4);
+      c.take(ws.attn_part_ml, rh * chunks * d.max_block * 2 * 4);
+      c.take(ws.attn_counters, rh * 4);
     }
   }
   c.take(ws.logits_raw, M * V * 4);
@@ -230,7 +234,17 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   const GemmTcPlan p_o = plan_gemm_tc(M, d, d, false, true, ctx->n_sms);
   const GemmTcPlan p_gu = plan_gemm_tc(M, ff, d, true, true, ctx->n_sms);
   const GemmTcPlan p_down = plan_gemm_tc(M, d, ff, false, true, ctx->n_sms);
-  CUtensorMap tm_xn, tm_attn, tm_act;
+  CUtensorMap tm_xn, tm_attn, tm_act, tm_q, tm_k, tm_v;
+  const uint64_t kv_total_rows = (uint64_t)md.n_layers * a->kv_rows * md.n_heads * md.s_max;
+  if (make_tmap_bf16_2d(&tm_q, q, (uint64_t)M, (uint64_t)d, Tn <= 16 ? 16u : 32u) != VVS_OK ||
+      make_tmap_bf16_2d(&tm_k, kv_k, kv_total_rows, (uint64_t)md.head_dim, 128u) != VVS_OK ||
+      make_tmap_bf16_2d(&tm_v, kv_v, kv_total_rows, (uint64_t)md.head_dim, 128u) != VVS_OK)
+    return VVS_ERR_CUDA;
+  AttentionTcArgs at{};
+  at.tm_q = &tm_q; at.tm_k = &tm_k; at.tm_v = &tm_v; at.cache_len = a->cache_len; at.out = attn;
+  at.part_o = ws.attn_part_o; at.part_ml = ws.attn_part_ml; at.counters = ws.attn_counters;
+  at.status = ws.status; at.d = d; at.n_heads = md.n_heads; at.hd = md.head_dim; at.s_max = md.s_max;
+  at.kv_rows = a->kv_rows; at.t_len = Tn; at.n_rows = R; at.pdl = ctx->use_pdl;
   if (make_tmap_bf16_2d(&tm_xn, xn, (uint64_t)M, (uint64_t)d, (uint32_t)p_qkv.nt) != VVS_OK ||
       make_tmap_bf16_2d(&tm_attn, attn, (uint64_t)M, (uint64_t)d, (uint32_t)p_o.nt) != VVS_OK ||
       make_tmap_bf16_2d(&tm_act, act, (uint64_t)M, (uint64_t)ff, (uint32_t)p_down.nt) != VVS_OK)
@@ -257,8 +271,10 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
       g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.ld_scratch = 3 * d; g.layer = l;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_QKV, p_qkv, g, s));
     }
-    VVS_LAUNCH(VVS_PROF_ATTENTION,
-               launch_attention<T>(q, kv_k, kv_v, a->cache_len, attn, md, l, a->kv_rows, R, Tn, s));
+    if (rc == VVS_OK) {
+      at.layer = l;
+      VVS_LAUNCH(VVS_PROF_ATTENTION, rc = launch_attention_tc(at, s));
+    }
     if (rc == VVS_OK) {
       GemmTcArgs g = base;
       g.n = d; g.k = d; g.tm_a = &W.w_o; g.tm_b = &tm_attn; g.out = ws.x; g.ldo = d;

@@ -47,6 +47,9 @@ struct Workspace {
   float* rope_sin = nullptr;     // [M, head_dim/2]
   float* sk_scratch = nullptr;   // [M, max(3d, 2ff)] fp32 split-K sums; all zero between kernels
   int* sk_counters = nullptr;    // [passes, tiles] split-K arrival counters; zero between kernels
+  float* attn_part_o = nullptr;  // [R*H, chunks, T, hd] un-normalised split-KV outputs
+  float* attn_part_ml = nullptr; // [R*H, chunks, T, 2] chunk max / sum
+  int* attn_counters = nullptr;  // [R*H] split-KV arrival counters; zero between kernels
   int32_t* status = nullptr; // device status word
 };
 
@@ -142,6 +145,19 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
 int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStream_t s);
 void launch_rope_table(const int32_t* cache_len, const Workspace& ws, const vvs_model_desc& md, int n_rows,
                        int t_len, cudaStream_t s);
+
+// ---- tensor-core attention, attention_tc.cu ----------------------------------------------------------
+struct AttentionTcArgs {
+  const CUtensorMap* tm_q;   // q [M, d], box {64, 16 or 32}
+  const CUtensorMap* tm_k;   // cache viewed as [layers*kv_rows*heads*s_max, hd], box {64, 128}
+  const CUtensorMap* tm_v;
+  const int32_t* cache_len;
+  __nv_bfloat16* out;
+  float* part_o; float* part_ml; int* counters; int32_t* status;
+  int d, n_heads, hd, s_max, layer, kv_rows, t_len, n_rows;
+  bool pdl;
+};
+int launch_attention_tc(const AttentionTcArgs& a, cudaStream_t s);
 
 // ---- decision stage, kernels_decide.cu -----------------------------------------------------
 struct DecideParams {
