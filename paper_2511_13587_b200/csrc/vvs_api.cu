@@ -298,6 +298,66 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
 }
 
+int enqueue_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, cudaStream_t s) {
+  if (ctx->tensor_core_path) return run_verify_tc(ctx, a, o, s);
+  return ctx->desc.dtype == VVS_DTYPE_BF16 ? run_verify<__nv_bfloat16>(ctx, a, o, s)
+                                           : run_verify<float>(ctx, a, o, s);
+}
+
+// The step is ~150-270 small kernels; launching them one by one costs more host time than the
+// GPU needs to run them.  Each distinct argument set is therefore captured once into a CUDA graph
+// (on a private stream, so the caller may use the legacy default stream) and replayed afterwards.
+int verify_via_graph(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, cudaStream_t s) {
+  vvs_verify_args ka = *a;
+  ka.cache_len_host = nullptr;  // host-side validation only, not part of the device work
+  std::vector<unsigned char> key(sizeof(ka) + sizeof(*o));
+  std::memcpy(key.data(), &ka, sizeof(ka));
+  std::memcpy(key.data() + sizeof(ka), o, sizeof(*o));
+  ++ctx->graph_clock;
+  for (auto& g : ctx->graphs) {
+    if (g.key == key) {
+      g.last_use = ctx->graph_clock;
+      ctx->launches = g.launches;
+      return cudaGraphLaunch(g.exec, s) == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+    }
+  }
+  cudaGraph_t graph = nullptr;
+  if (cudaStreamBeginCapture(ctx->capture_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    ctx->use_graph = false;
+    ctx->launches = 0;
+    return enqueue_verify(ctx, a, o, s);
+  }
+  ctx->launches = 0;
+  const int rc = enqueue_verify(ctx, a, o, ctx->capture_stream);
+  const cudaError_t e = cudaStreamEndCapture(ctx->capture_stream, &graph);
+  cudaGraphExec_t exec = nullptr;
+  if (rc != VVS_OK || e != cudaSuccess || !graph ||
+      cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) {
+    cudaGetLastError();
+    if (graph) cudaGraphDestroy(graph);
+    if (rc != VVS_OK) return rc;
+    ctx->use_graph = false;  // capture is not available here: fall back to plain launches
+    ctx->launches = 0;
+    return enqueue_verify(ctx, a, o, s);
+  }
+  cudaGraphDestroy(graph);
+  if (ctx->graphs.size() >= 64) {  // evict the least recently used entry
+    size_t victim = 0;
+    for (size_t i = 1; i < ctx->graphs.size(); ++i)
+      if (ctx->graphs[i].last_use < ctx->graphs[victim].last_use) victim = i;
+    cudaGraphExecDestroy(ctx->graphs[victim].exec);
+    ctx->graphs.erase(ctx->graphs.begin() + victim);
+  }
+  GraphEntry ge;
+  ge.key = std::move(key);
+  ge.exec = exec;
+  ge.launches = ctx->launches;
+  ge.last_use = ctx->graph_clock;
+  ctx->graphs.push_back(std::move(ge));
+  return cudaGraphLaunch(exec, s) == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+}
+
 int check_decision_args(const vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o,
                         int rows_per_seq) {
   const vvs_model_desc& md = ctx->desc;
@@ -377,6 +437,12 @@ int vvs_create(const vvs_model_desc* desc, vvs_ctx** out) {
   // VVS_DEBUG_NO_PDL launches the tensor-core GEMMs without programmatic dependent launch.
   ctx->tensor_core_path = desc->dtype == VVS_DTYPE_BF16 && !std::getenv("VVS_DEBUG_GENERIC");
   ctx->use_pdl = !std::getenv("VVS_DEBUG_NO_PDL");
+  ctx->use_graph = !std::getenv("VVS_DEBUG_NO_GRAPH");
+  if (cudaStreamCreateWithFlags(&ctx->capture_stream, cudaStreamNonBlocking) != cudaSuccess) {
+    cudaGetLastError();
+    ctx->capture_stream = nullptr;
+    ctx->use_graph = false;
+  }
   if (cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess ||
       ctx->n_sms < 1)
     ctx->n_sms = 148;
@@ -384,9 +450,17 @@ int vvs_create(const vvs_model_desc* desc, vvs_ctx** out) {
   return VVS_OK;
 }
 
+static void drop_graphs(vvs_ctx* ctx) {
+  for (auto& g : ctx->graphs)
+    if (g.exec) cudaGraphExecDestroy(g.exec);
+  ctx->graphs.clear();
+}
+
 int vvs_destroy(vvs_ctx* ctx) {
   if (!ctx) return VVS_ERR_INVALID_ARG;
   vvs_profile_enable(ctx, 0);
+  drop_graphs(ctx);
+  if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
   if (ctx->arena) cudaFree(ctx->arena);
   delete[] ctx->layers;
   delete[] ctx->layer_maps;
@@ -434,6 +508,7 @@ int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w) {
                             md.vocab, d);
     if (rc != VVS_OK) return rc;
   }
+  drop_graphs(ctx);  // captured steps hold the old pointers
   ctx->tok_emb = w->tok_emb;
   ctx->norm_f = w->norm_f;
   ctx->w_lm = w->w_lm;
@@ -444,6 +519,7 @@ int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w) {
 int vvs_bind_neighbors(vvs_ctx* ctx, const int32_t* row_ptr, const int32_t* col, int64_t nnz) {
   if (!ctx || !row_ptr || !col || nnz < 0) return VVS_ERR_INVALID_ARG;
   if (!aligned16(row_ptr) || !aligned16(col)) return VVS_ERR_ALIGN;
+  drop_graphs(ctx);
   ctx->nbr_row_ptr = row_ptr;
   ctx->nbr_col = col;
   ctx->nbr_nnz = nnz;
@@ -467,11 +543,13 @@ int vvs_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, 
     for (int r = 0; r < R; ++r)
       if (a->cache_len_host[r] < 0 || a->cache_len_host[r] + Tn > md.s_max) return VVS_ERR_CAPACITY;
   }
-  ctx->launches = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (ctx->tensor_core_path) return run_verify_tc(ctx, a, o, s);
-  return md.dtype == VVS_DTYPE_BF16 ? run_verify<__nv_bfloat16>(ctx, a, o, s)
-                                    : run_verify<float>(ctx, a, o, s);
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (ctx->use_graph && !ctx->profiling &&
+      cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone)
+    return verify_via_graph(ctx, a, o, s);
+  ctx->launches = 0;
+  return enqueue_verify(ctx, a, o, s);
 }
 
 int vvs_epilogue(vvs_ctx* ctx, const void* hidden, int32_t n_rows_per_seq, int32_t first_row,

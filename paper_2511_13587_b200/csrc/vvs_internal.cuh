@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "vvs.h"
 
 #define VVS_CUDA_OK(expr)                         \
@@ -64,6 +66,16 @@ struct LayerMaps {
 
 }  // namespace vvs
 
+namespace vvs {
+// One captured verify step: replayed whenever a call repeats the same arguments.
+struct GraphEntry {
+  std::vector<unsigned char> key;  // argument and output structs, byte for byte
+  cudaGraphExec_t exec = nullptr;
+  int launches = 0;
+  unsigned long long last_use = 0;
+};
+}  // namespace vvs
+
 struct vvs_ctx {
   vvs_model_desc desc;
   vvs::Workspace ws;
@@ -79,6 +91,11 @@ struct vvs_ctx {
   vvs::LayerMaps* layer_maps = nullptr;  // host array [n_layers]
   CUtensorMap lm_map;
   int n_sms = 148;
+  // CUDA-graph replay of vvs_verify (one graph per distinct argument set, small LRU cache)
+  bool use_graph = true;
+  cudaStream_t capture_stream = nullptr;
+  std::vector<vvs::GraphEntry> graphs;
+  unsigned long long graph_clock = 0;
   const int32_t* nbr_row_ptr = nullptr;
   const int32_t* nbr_col = nullptr;
   int64_t nbr_nnz = 0;
