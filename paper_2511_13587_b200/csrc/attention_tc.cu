@@ -41,18 +41,6 @@ struct AttnParams {
 
 __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity) { return mbar_wait(bar, parity); }
 
-// MN-major bf16 operand whose 64-element (128-byte) rows are 128-byte swizzled, one row per K
-// index: 8-row groups 1024 bytes apart (stride offset), 64-element column chunks lbo bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t saddr, uint32_t lbo_bytes) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((saddr >> 4) & 0x3FFF);
-  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFF) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
-
 __device__ __forceinline__ float warp_max_f(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));

@@ -55,6 +55,12 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
       c.take(ws.attn_part_o, rh * chunks * d.max_block * d.head_dim * 4);
       c.take(ws.attn_part_ml, rh * chunks * d.max_block * 2 * 4);
       c.take(ws.attn_counters, rh * 4);
+      c.take(ws.chain_wmaps, (size_t)d.n_layers * 5 * sizeof(CUtensorMap));
+      c.take(ws.chain_norms, (size_t)d.n_layers * 2 * sizeof(void*));
+      c.take(ws.chain_qkv, (size_t)2 * 32 * 3 * dm * 4);
+      c.take(ws.chain_gu, (size_t)2 * 32 * 2 * ff * 4);
+      c.take(ws.chain_ss, (size_t)2 * d.n_layers * 32 * 4);
+      c.take(ws.chain_sync, 256);
     }
   }
   c.take(ws.logits_raw, M * V * 4);
@@ -259,6 +265,24 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   base.kv_rows = a->kv_rows; base.t_len = Tn; base.act = act; base.ff = ff;
 
   int rc = VVS_OK;
+  if (ctx->use_chain && fused_chain_applicable(md, R, Tn)) {
+    // at most 32 tokens: the whole decoder chain runs as one persistent kernel
+    FusedChainArgs fc{};
+    fc.md = &md; fc.n_rows = R; fc.n_images = B; fc.t_len = Tn; fc.kv_rows = a->kv_rows; fc.n_sms = ctx->n_sms;
+    fc.wmaps = ws.chain_wmaps; fc.norms = ws.chain_norms;
+    fc.tok_emb = static_cast<const T*>(ctx->tok_emb); fc.block = a->block;
+    fc.x = ws.x; fc.qkv_acc = ws.chain_qkv; fc.gu_acc = ws.chain_gu; fc.ss = ws.chain_ss;
+    fc.cache_len = a->cache_len; fc.kv_k = kv_k; fc.kv_v = kv_v; fc.tm_k = &tm_k; fc.tm_v = &tm_v;
+    fc.slot_pos = ws.slot_pos; fc.rope_cos = ws.rope_cos; fc.rope_sin = ws.rope_sin;
+    fc.part_o = ws.attn_part_o; fc.part_ml = ws.attn_part_ml; fc.sync_words = ws.chain_sync;
+    fc.status = ws.status;
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, ws, md, R, Tn, s));
+    VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_fused_chain(fc, s));
+    if (rc != VVS_OK) return rc;
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
+    if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
+    return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
+  }
   VVS_LAUNCH(VVS_PROF_OTHER, launch_embed<T>(static_cast<const T*>(ctx->tok_emb), a->block, ws.x, B, C, Tn,
                                              d, md.tok_rows, ws.status, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, ws, md, R, Tn, s));
@@ -336,7 +360,6 @@ int verify_via_graph(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_ou
       cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) {
     cudaGetLastError();
     if (graph) cudaGraphDestroy(graph);
-    if (rc != VVS_OK) return rc;
     ctx->use_graph = false;  // capture is not available here: fall back to plain launches
     ctx->launches = 0;
     return enqueue_verify(ctx, a, o, s);
@@ -434,10 +457,12 @@ int vvs_create(const vvs_model_desc* desc, vvs_ctx** out) {
     if (!ctx->layers || !ctx->layer_maps) { vvs_destroy(ctx); return VVS_ERR_NOMEM; }
   }
   // Debug switches only: VVS_DEBUG_GENERIC runs bf16 contexts on the generic kernels,
-  // VVS_DEBUG_NO_PDL launches the tensor-core GEMMs without programmatic dependent launch.
+  // VVS_DEBUG_NO_PDL launches the tensor-core GEMMs without programmatic dependent launch,
+  // VVS_DEBUG_NO_CHAIN runs small calls through the per-projection kernels too.
   ctx->tensor_core_path = desc->dtype == VVS_DTYPE_BF16 && !std::getenv("VVS_DEBUG_GENERIC");
   ctx->use_pdl = !std::getenv("VVS_DEBUG_NO_PDL");
   ctx->use_graph = !std::getenv("VVS_DEBUG_NO_GRAPH");
+  ctx->use_chain = !std::getenv("VVS_DEBUG_NO_CHAIN");
   if (cudaStreamCreateWithFlags(&ctx->capture_stream, cudaStreamNonBlocking) != cudaSuccess) {
     cudaGetLastError();
     ctx->capture_stream = nullptr;
@@ -507,6 +532,20 @@ int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w) {
                             static_cast<const __nv_bfloat16*>(w->w_lm) + (size_t)md.vocab_offset * d,
                             md.vocab, d);
     if (rc != VVS_OK) return rc;
+    if (n > 0) {
+      // device copies for the whole-chain kernel, which walks all layers inside one launch
+      static_assert(sizeof(LayerMaps) == 5 * sizeof(CUtensorMap), "LayerMaps is five descriptors");
+      std::vector<const void*> norms(2 * (size_t)n);
+      for (int l = 0; l < n; ++l) {
+        norms[2 * l] = w->layers[l].norm1;
+        norms[2 * l + 1] = w->layers[l].norm2;
+      }
+      if (cudaMemcpy(ctx->ws.chain_wmaps, ctx->layer_maps, (size_t)n * sizeof(LayerMaps),
+                     cudaMemcpyHostToDevice) != cudaSuccess ||
+          cudaMemcpy(ctx->ws.chain_norms, norms.data(), norms.size() * sizeof(void*),
+                     cudaMemcpyHostToDevice) != cudaSuccess)
+        return VVS_ERR_CUDA;
+    }
   }
   drop_graphs(ctx);  // captured steps hold the old pointers
   ctx->tok_emb = w->tok_emb;
@@ -646,6 +685,12 @@ int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits) {
   VVS_CUDA_OK(cudaMemsetAsync(ctx->ws.status, 0, sizeof(bits), s));
   VVS_CUDA_OK(cudaStreamSynchronize(s));
   *out_bits = bits;
+  if ((bits & VVS_DEV_TIMEOUT) && ctx->ws.chain_sync) {
+    // a grid barrier of the whole-chain kernel gave up: its arrival counter is no longer a
+    // multiple of the grid size, start again from zero
+    VVS_CUDA_OK(cudaMemsetAsync(ctx->ws.chain_sync, 0, 16, s));
+    VVS_CUDA_OK(cudaStreamSynchronize(s));
+  }
   if (bits & VVS_DEV_TIMEOUT) return VVS_ERR_DEVICE_TIMEOUT;
   if (bits & (VVS_DEV_BAD_TOKEN | VVS_DEV_CACHE_OVERFLOW | VVS_DEV_BAD_NEIGHBOUR | VVS_DEV_BAD_ARG))
     return VVS_ERR_DEVICE_BOUNDS;

@@ -52,6 +52,13 @@ struct Workspace {
   float* attn_part_o = nullptr;  // [R*H, chunks, T, hd] un-normalised split-KV outputs
   float* attn_part_ml = nullptr; // [R*H, chunks, T, 2] chunk max / sum
   int* attn_counters = nullptr;  // [R*H] split-KV arrival counters; zero between kernels
+  // whole-chain kernel (at most 32 block tokens)
+  CUtensorMap* chain_wmaps = nullptr;          // [n_layers][5] weight descriptors, device copy
+  const __nv_bfloat16** chain_norms = nullptr; // [n_layers][2] norm-scale pointers, device copy
+  float* chain_qkv = nullptr;    // [2][32, 3d] fp32 split-K sums of the QKV projection (by layer parity)
+  float* chain_gu = nullptr;     // [2][32, 2ff] fp32 split-K sums of gate | up
+  float* chain_ss = nullptr;     // [2 * n_layers][32] sums of squares of the residual rows
+  unsigned* chain_sync = nullptr;  // [4] grid-barrier arrivals, epoch base, abort flag
   int32_t* status = nullptr; // device status word
 };
 
@@ -88,6 +95,7 @@ struct vvs_ctx {
   vvs::Layer* layers = nullptr;  // host array [n_layers]
   bool tensor_core_path = false;     // bf16 contexts unless VVS_DEBUG_GENERIC is set
   bool use_pdl = true;               // programmatic dependent launch of the tensor-core GEMMs
+  bool use_chain = true;             // whole-chain persistent kernel for calls of at most 32 tokens
   vvs::LayerMaps* layer_maps = nullptr;  // host array [n_layers]
   CUtensorMap lm_map;
   int n_sms = 148;
@@ -175,6 +183,28 @@ struct AttentionTcArgs {
   bool pdl;
 };
 int launch_attention_tc(const AttentionTcArgs& a, cudaStream_t s);
+
+// ---- whole-chain persistent kernel, fused_chain.cu ---------------------------------------------
+struct FusedChainArgs {
+  const vvs_model_desc* md;
+  int n_rows, n_images, t_len, kv_rows, n_sms;
+  const CUtensorMap* wmaps;             // device
+  const __nv_bfloat16* const* norms;    // device
+  const __nv_bfloat16* tok_emb;
+  const int32_t* block;
+  float* x; float* qkv_acc; float* gu_acc; float* ss;
+  const int32_t* cache_len;
+  __nv_bfloat16* kv_k; __nv_bfloat16* kv_v;
+  const CUtensorMap* tm_k;              // host copies of the cache descriptors (box {64, 128})
+  const CUtensorMap* tm_v;
+  const int32_t* slot_pos; const float* rope_cos; const float* rope_sin;
+  float* part_o; float* part_ml;
+  unsigned* sync_words;
+  int32_t* status;
+};
+bool fused_chain_applicable(const vvs_model_desc& md, int n_rows, int t_len);
+size_t fused_chain_smem_bytes(const vvs_model_desc& md, int t_len, int* w_stages);
+int launch_fused_chain(const FusedChainArgs& a, cudaStream_t s);
 
 // ---- decision stage, kernels_decide.cu -----------------------------------------------------
 struct DecideParams {
