@@ -30,6 +30,12 @@
 #include "tc_common.cuh"
 #include "vvs_internal.cuh"
 
+// Event trace hooks: empty unless a profiling build defines them before this point.
+#ifndef VVS_TRACE
+#define VVS_TRACE_DECL
+#define VVS_TRACE(tag) ((void)0)
+#endif
+
 namespace vvs {
 
 using namespace tc;
@@ -41,10 +47,11 @@ constexpr int kWorkers = 256;          // warps 2-9
 constexpr int kGroup = 128;
 constexpr int kSlabBytes = 16384;      // 128 weight rows x 64 bf16
 constexpr int kTokSlabBytes = 4096;    // 32 tokens x 64 bf16
-constexpr int kTokStages = 4;
+constexpr int kStageBytes = kSlabBytes + kTokSlabBytes;   // one ring stage: weight slab + token slab
 constexpr int kAccSlots = 4;           // TMEM accumulator slots of 64 columns
-constexpr int kMaxWStages = 12;
+constexpr int kMaxStages = 10;
 constexpr int kMaxSeq = 32;
+constexpr int kMaxLayers = 64;
 constexpr uint32_t kColS = 256, kColO = 320, kTmemCols = 512;
 constexpr uint32_t kGridSpinLimit = 1u << 21;
 enum { BAR_W = 1, BAR_E = 2, BAR_D = 3 };
@@ -53,10 +60,9 @@ enum { PH_QKV = 0, PH_O = 1, PH_GU = 2, PH_DOWN = 3 };
 struct ChainParams {
   int n_layers, d, n_heads, hd, ff, s_max, kv_rows;
   int m, t_len, tq, n_rows, n_images, tok_rows;
-  int w_stages, n_chunks_max;
+  int n_stages, n_chunks_max;
   float eps, scale;
   const CUtensorMap* wmaps;            // device [n_layers][5]: qkv, o, gate, up, down
-  const __nv_bfloat16* const* norms;   // device [n_layers][2]
   const __nv_bfloat16* tok_emb;
   const int32_t* block;
   float* x;                            // [m, d] residual stream
@@ -66,13 +72,13 @@ struct ChainParams {
   const int32_t* cache_len;
   __nv_bfloat16* kv_k;
   __nv_bfloat16* kv_v;
-  const int32_t* slot_pos;
   const float* rope_cos;
   const float* rope_sin;
   float* part_o;
   float* part_ml;
   unsigned* sync_words;                // [0] arrivals, [1] epoch base, [2] abort
   int32_t* status;
+  const __nv_bfloat16* norms[2 * kMaxLayers];   // norm scales, read through the constant bank
 };
 
 struct Phase {
@@ -95,15 +101,16 @@ __device__ __forceinline__ Phase phase_of(const ChainParams& p, int ph) {
 
 // Share of a projection owned by this CTA: a contiguous range of (tile, k-block) units in
 // tile-major order; the rotation moves the CTAs that get one unit more from phase to phase.
+// (tiles * k-blocks * grid stays far below 2^32 for every supported shape.)
 __device__ __forceinline__ void unit_range(const Phase& f, int layer, int ph, int& lo, int& hi) {
-  const int G = (int)gridDim.x, S = f.tiles * f.kbs;
-  const int v = (int)((blockIdx.x + (unsigned)(layer * 4 + ph) * 53u) % (unsigned)G);
-  lo = (int)(((long long)v * S) / G);
-  hi = (int)(((long long)(v + 1) * S) / G);
+  const unsigned G = gridDim.x, S = (unsigned)(f.tiles * f.kbs);
+  const unsigned v = (blockIdx.x + (unsigned)(layer * 4 + ph) * 53u) % G;
+  lo = (int)(v * S / G);
+  hi = (int)((v + 1) * S / G);
 }
 
 // Bounded wait; falls through at once when the CTA is in abort mode.
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* s_abort, int32_t* status) {
+__device__ __noinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* s_abort, int32_t* status) {
   if (*s_abort) return false;
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -162,29 +169,130 @@ __device__ __forceinline__ void rope8(const ChainParams& p, int tok, int e, floa
   }
 }
 
+// tcgen05.mma with an immediate accumulate flag
+__device__ __forceinline__ void mma_set(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+}
+__device__ __forceinline__ void mma_acc(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 1, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+}
+
+// Fast path of a wait: one poll, inline.
+__device__ __forceinline__ bool wait_fast(uint64_t* bar, uint32_t parity, volatile int* s_abort, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return wait_bar(bar, parity, s_abort, status);
+}
+
+// One round of token-operand building by the 256 worker threads: nb <= (1 << lg) units,
+// 256 >> lg threads per unit.  A unit's slab is m rows x 16 positions of 4 columns; thread j of
+// the unit takes positions j, j + tpu, ... so that consecutive lanes read consecutive 16 bytes
+// and every load of the round is in flight before the first use (MAXI = positions per thread).
+//   DOWN == false: slab = bf16(x * norm scale); the CTAs that own tile 0 also add the row sums
+//                  of squares into ss_out
+//   DOWN == true : slab = bf16(silu(gate / rms) * (up / rms)), rms from ss_in
+template <int MAXI, bool DOWN>
+__device__ __noinline__ void build_round(const ChainParams& p, uint8_t* ring, uint64_t* empty, volatile int* s_abort,
+                                         int tid_w, int nb, int lg, uint32_t it0, uint32_t per_unit, int s0, int kbs,
+                                         const float* src, const __nv_bfloat16* gsc, const float* ss_in,
+                                         float* ss_out) {
+  const uint32_t NS = (uint32_t)p.n_stages;
+  const int tpu = 256 >> lg, u = tid_w >> (8 - lg), j = tid_w & (tpu - 1);
+  if (u >= nb) return;                                   // uniform per warp (tpu >= 32)
+  const uint32_t it = it0 + (uint32_t)u * per_unit, st = it % NS, use = it / NS;
+  if (use > 0) wait_fast(&empty[st], (use - 1) & 1, s_abort, p.status);
+  const int s = s0 + u, tile = s / kbs, kb = s - tile * kbs;
+  const int m = p.m, ff = p.ff;
+  const int q = j & 15, row0 = j >> 4, rstep = tpu >> 4;  // this thread: column group q, rows row0 + k * rstep
+  const int col = kb * 64 + q * 4;
+  const int ld = DOWN ? 2 * ff : p.d;
+  const float* sp = src + (size_t)row0 * ld + col;
+  const size_t sstep = (size_t)rstep * ld;
+  const bool col_ok = !DOWN || col < ff;
+  float4 a[MAXI];
+  float4 b[DOWN ? MAXI : 1];
+  float sv[DOWN ? MAXI : 1];
+  uint2 g = make_uint2(0u, 0u);
+  if (!DOWN) g = __ldg(reinterpret_cast<const uint2*>(gsc + col));
+#pragma unroll
+  for (int k = 0; k < MAXI; ++k) {
+    a[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (DOWN) { b[k] = a[k]; sv[k] = 1.f; }
+    if (row0 + k * rstep < m) {
+      if (col_ok) {
+        a[k] = __ldcg(reinterpret_cast<const float4*>(sp));
+        if (DOWN) b[k] = __ldcg(reinterpret_cast<const float4*>(sp + ff));
+      }
+      if (DOWN) sv[k] = __ldcg(ss_in + row0 + k * rstep);
+    }
+    sp += sstep;
+  }
+  float gv[4] = {1.f, 1.f, 1.f, 1.f};
+  if (!DOWN) {
+    const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g.x));
+    const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g.y));
+    gv[0] = g01.x; gv[1] = g01.y; gv[2] = g23.x; gv[3] = g23.y;
+  }
+  const float inv_d = 1.f / (float)p.d, eps = p.eps;
+  uint8_t* out = ring + (size_t)st * kStageBytes + kSlabBytes + row0 * 128 + ((q & 1) << 3);
+  int row = row0;
+#pragma unroll
+  for (int k = 0; k < MAXI; ++k) {
+    float v[4] = {a[k].x, a[k].y, a[k].z, a[k].w};
+    if (DOWN) {
+      const float rinv = rsqrtf(fmaf(sv[k], inv_d, eps));
+      const float w[4] = {b[k].x, b[k].y, b[k].z, b[k].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float t = v[e] * rinv;
+        v[e] = __fdividef(t, 1.f + __expf(-t)) * (w[e] * rinv);
+      }
+    } else {
+      if (tile == 0) {                                   // uniform per warp
+        float ssq = v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, o);   // 16 lanes = one row
+        if (q == 0 && row < m) atomicAdd(ss_out + row, ssq);
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v[e] *= gv[e];
+    }
+    if (row < m) {
+      uint2 o;
+      *reinterpret_cast<__nv_bfloat162*>(&o.x) = __floats2bfloat162_rn(v[0], v[1]);
+      *reinterpret_cast<__nv_bfloat162*>(&o.y) = __floats2bfloat162_rn(v[2], v[3]);
+      *reinterpret_cast<uint2*>(out + ((((q >> 1) ^ row) & 7) << 4)) = o;
+    }
+    row += rstep;
+    out += rstep * 128;
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k,
+fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t w_full[kMaxWStages], w_empty[kMaxWStages];
-  __shared__ __align__(8) uint64_t b_full[kTokStages], b_empty[kTokStages];
+  __shared__ __align__(8) uint64_t full[kMaxStages], empty[kMaxStages];
   __shared__ __align__(8) uint64_t acc_full[kAccSlots], acc_empty[kAccSlots];
   __shared__ __align__(8) uint64_t att_kv_full, att_q_ready, att_s_full, att_p_ready, att_o_full;
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_abort;
   __shared__ int s_fill[kMaxSeq], s_nch[kMaxSeq], s_prefix[kMaxSeq + 1];
-  __shared__ float red_max[4][32], red_sum[4][32];
+  __shared__ float row_max[32], row_sum[32];
+  VVS_TRACE_DECL
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = (int)gridDim.x;
   const int NC = p.hd >> 6;                       // 64-column chunks of a head
-  const int NS = p.w_stages;
+  const uint32_t NS = (uint32_t)p.n_stages;
   const int T = p.t_len, H = p.n_heads, L = p.n_layers;
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* ring = smem;
-  uint8_t* tokring = ring + (size_t)NS * kSlabBytes;
-  uint8_t* sK = tokring + kTokStages * kTokSlabBytes;
+  uint8_t* ring = smem;                           // n_stages x [weight slab | token slab]
+  uint8_t* sK = ring + (size_t)NS * kStageBytes;
   uint8_t* sV = sK + NC * kSlabBytes;
   uint8_t* sP = sV + NC * kSlabBytes;             // 2 x [128 rows x 128 B]
   uint8_t* sQ = sP + 2 * kSlabBytes;              // NC x [tq rows x 128 B]
@@ -192,11 +300,10 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
 
   // ---- set-up ------------------------------------------------------------------------------------
   if (tid == 0) {
-    for (int i = 0; i < NS; ++i) { mbar_init(&w_full[i], 1); mbar_init(&w_empty[i], 1); }
-    for (int i = 0; i < kTokStages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
+    for (uint32_t i = 0; i < NS; ++i) { mbar_init(&full[i], 2); mbar_init(&empty[i], 1); }   // TMA + builders
     for (int i = 0; i < kAccSlots; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 1); }
     mbar_init(&att_kv_full, 1);
-    mbar_init(&att_q_ready, 1);
+    mbar_init(&att_q_ready, 2);   // the Q builders and the K / V row builders
     mbar_init(&att_s_full, 1);
     mbar_init(&att_p_ready, 1);
     mbar_init(&att_o_full, 1);
@@ -217,8 +324,9 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
     s_prefix[p.n_rows] = acc;
   }
   // token operands: rows of tokens that do not exist stay zero for the whole kernel
-  for (int i = tid; i < (kTokStages * kTokSlabBytes) / 16; i += kThreads)
-    reinterpret_cast<uint4*>(tokring)[i] = make_uint4(0, 0, 0, 0);
+  for (uint32_t i = tid; i < NS * (kTokSlabBytes / 16); i += kThreads)
+    reinterpret_cast<uint4*>(ring + (size_t)(i / (kTokSlabBytes / 16)) * kStageBytes + kSlabBytes)[i % (kTokSlabBytes / 16)] =
+        make_uint4(0, 0, 0, 0);
   for (int i = tid; i < (int)(NC * q_chunk_bytes) / 16; i += kThreads)
     reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
   if (warp == 1) {
@@ -232,7 +340,6 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
   const uint32_t tmem_base = tmem_slot;
   const unsigned epoch = *reinterpret_cast<volatile unsigned*>(p.sync_words + 1);
   const int n_items = s_prefix[p.n_rows] * H;     // attention items of one layer, all CTAs
-  const uint32_t idesc_gemm = idesc_bf16_f32(128, 32);
 
   auto decode_item = [&](int i, int& r, int& h, int& c) {
     const int rc = i / H;
@@ -248,44 +355,53 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
   if (warp == 0) {
     // =================================== weight producer ===========================================
     if (lane == 0) {
-      uint32_t it = 0;
+      uint32_t st = 0, round = 0;
       bool alive = true;
+#pragma unroll 1
       for (int l = 0; l < L && alive; ++l) {
+#pragma unroll 1
         for (int ph = 0; ph < 4 && alive; ++ph) {
           const Phase f = phase_of(p, ph);
           int lo, hi;
           unit_range(f, l, ph, lo, hi);
+          int tile = lo / f.kbs, kb = lo - tile * f.kbs;
+          const CUtensorMap* map = &p.wmaps[l * 5 + f.map0];
+#pragma unroll 1
           for (int s = lo; s < hi && alive; ++s) {
-            const int tile = s / f.kbs, kb = s - tile * f.kbs;
-            for (int j = 0; j <= f.dual; ++j, ++it) {
-              const uint32_t stage = it % NS, use = it / NS;
-              if (use > 0 && !wait_bar(&w_empty[stage], (use - 1) & 1, &s_abort, p.status)) { alive = false; break; }
-              mbar_expect_tx(&w_full[stage], kSlabBytes);
-              tma_load_2d(ring + (size_t)stage * kSlabBytes, &p.wmaps[l * 5 + f.map0 + j], &w_full[stage],
-                          kb * 64, tile * 128);
+            for (int j = 0; j <= f.dual; ++j) {
+              if (round > 0 && !wait_bar(&empty[st], (round - 1) & 1, &s_abort, p.status)) { alive = false; break; }
+              mbar_expect_tx(&full[st], kSlabBytes);
+              tma_load_2d(ring + (size_t)st * kStageBytes, map + j, &full[st], kb * 64, tile * 128);
+              VVS_TRACE(0x100 | (ph << 4) | (s - lo));
+              if (++st == NS) { st = 0; ++round; }
             }
+            if (++kb == f.kbs) { kb = 0; ++tile; }
           }
         }
       }
-      // every load that was issued must have landed before the CTA may exit
-      for (uint32_t stage = 0; stage < (uint32_t)NS; ++stage) {
-        if (it > stage) mbar_wait(&w_full[stage], ((it - 1 - stage) / NS) & 1);
-      }
+      // In abort mode loads may still be in flight with nobody waiting for them: let them land.
+      if (s_abort) __nanosleep(200000);
     }
   } else if (warp == 1) {
     // =================================== MMA issuer ==================================================
     if (lane == 0) {
-      uint32_t itw = 0, itb = 0, ita = 0, iatt = 0;
+      uint32_t st = 0, par = 0, ita = 0, iatt = 0;
       bool alive = true;
+      const uint32_t idesc_gemm = idesc_bf16_f32(128, 32);
+      const uint64_t desc0 = smem_desc_sw128(smem_u32(ring));   // + (byte offset >> 4) selects a slab
+#pragma unroll 1
       for (int l = 0; l < L && alive; ++l) {
+#pragma unroll 1
         for (int ph = 0; ph < 4 && alive; ++ph) {
           if (ph == PH_O) {
             // ---- attention products of this CTA's items ----
+#pragma unroll 1
             for (int i = blockIdx.x; i < n_items && alive; i += G, ++iatt) {
-              const uint32_t par = iatt & 1;
-              if (!wait_bar(&att_kv_full, par, &s_abort, p.status) ||
-                  !wait_bar(&att_q_ready, par, &s_abort, p.status)) { alive = false; break; }
+              const uint32_t apar = iatt & 1;
+              if (!wait_bar(&att_kv_full, apar, &s_abort, p.status) ||
+                  !wait_bar(&att_q_ready, apar, &s_abort, p.status)) { alive = false; break; }
               tc_fence_after();
+              VVS_TRACE(0x2A1);
               const uint32_t idesc_s = idesc_bf16_f32(128, (uint32_t)p.tq);
               for (int k16 = 0; k16 < p.hd / 16; ++k16) {
                 const uint32_t a = smem_u32(sK + (k16 >> 2) * kSlabBytes) + (k16 & 3) * 32;
@@ -293,8 +409,10 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
                 mma_bf16(tmem_base + kColS, smem_desc_sw128(a), smem_desc_sw128(b), idesc_s, k16 > 0 ? 1u : 0u);
               }
               mma_commit(&att_s_full);
-              if (!wait_bar(&att_p_ready, par, &s_abort, p.status)) { alive = false; break; }
+              VVS_TRACE(0x2A2);
+              if (!wait_bar(&att_p_ready, apar, &s_abort, p.status)) { alive = false; break; }
               tc_fence_after();
+              VVS_TRACE(0x2A3);
               const uint32_t idesc_o = idesc_bf16_f32(128, (uint32_t)p.hd) | (1u << 16);  // B is MN-major
               for (int k16 = 0; k16 < 8; ++k16) {
                 const uint32_t a = smem_u32(sP + (k16 >> 2) * kSlabBytes) + (k16 & 3) * 32;
@@ -303,47 +421,57 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
                          k16 > 0 ? 1u : 0u);
               }
               mma_commit(&att_o_full);
+              VVS_TRACE(0x2A4);
             }
             if (!alive) break;
           }
           const Phase f = phase_of(p, ph);
           int lo, hi;
           unit_range(f, l, ph, lo, hi);
-          int cur_tile = -1;
+          int kb = lo % f.kbs;
           uint32_t slot = 0;
-          for (int s = lo; s < hi; ++s, ++itb) {
-            const int tile = s / f.kbs;
-            const bool first = tile != cur_tile;
+#pragma unroll 1
+          for (int s = lo; s < hi; ++s) {
+            const bool first = (s == lo) || (kb == 0);
             if (first) {
-              if (cur_tile >= 0) mma_commit(&acc_full[slot]);
+              if (s != lo) mma_commit(&acc_full[slot]);
               slot = ita % kAccSlots;
               const uint32_t use = ita / kAccSlots;
               if (use > 0 && !wait_bar(&acc_empty[slot], (use - 1) & 1, &s_abort, p.status)) { alive = false; break; }
-              cur_tile = tile;
               ++ita;
             }
-            const uint32_t bst = itb % kTokStages, st = itw % NS, st2 = (itw + 1) % NS;
-            if (!wait_bar(&b_full[bst], (itb / kTokStages) & 1, &s_abort, p.status) ||
-                !wait_bar(&w_full[st], (itw / NS) & 1, &s_abort, p.status) ||
-                (f.dual && !wait_bar(&w_full[st2], ((itw + 1) / NS) & 1, &s_abort, p.status))) { alive = false; break; }
-            tc_fence_after();
-            const uint32_t a_addr = smem_u32(ring + (size_t)st * kSlabBytes);
-            const uint32_t a2_addr = smem_u32(ring + (size_t)st2 * kSlabBytes);
-            const uint32_t b_addr = smem_u32(tokring + bst * kTokSlabBytes);
-            const uint32_t acc = tmem_base + slot * 64;
-#pragma unroll
-            for (uint32_t k16 = 0; k16 < 4; ++k16) {
-              const uint32_t accum = (!first || k16 > 0) ? 1u : 0u;
-              const uint64_t bd = smem_desc_sw128(b_addr + k16 * 32);
-              mma_bf16(acc, smem_desc_sw128(a_addr + k16 * 32), bd, idesc_gemm, accum);
-              if (f.dual) mma_bf16(acc + 32, smem_desc_sw128(a2_addr + k16 * 32), bd, idesc_gemm, accum);
+            if (!wait_fast(&full[st], par, &s_abort, p.status)) { alive = false; break; }
+            const uint64_t a_desc = desc0 + (uint64_t)(st * (kStageBytes >> 4));
+            const uint64_t b_desc = a_desc + (kSlabBytes >> 4);
+            const uint32_t st_a = st;
+            if (++st == NS) { st = 0; par ^= 1; }
+            uint64_t a2_desc = 0;
+            uint32_t st_b = 0;
+            if (f.dual) {
+              if (!wait_fast(&full[st], par, &s_abort, p.status)) { alive = false; break; }
+              a2_desc = desc0 + (uint64_t)(st * (kStageBytes >> 4));
+              st_b = st;
+              if (++st == NS) { st = 0; par ^= 1; }
             }
-            mma_commit(&w_empty[st]);
-            if (f.dual) mma_commit(&w_empty[st2]);
-            mma_commit(&b_empty[bst]);
-            itw += 1 + f.dual;
+            tc_fence_after();
+            VVS_TRACE(0x200 | (ph << 4) | (s - lo));
+            const uint32_t acc = tmem_base + slot * 64;
+            if (first) mma_set(acc, a_desc, b_desc, idesc_gemm); else mma_acc(acc, a_desc, b_desc, idesc_gemm);
+            mma_acc(acc, a_desc + 2, b_desc + 2, idesc_gemm);
+            mma_acc(acc, a_desc + 4, b_desc + 4, idesc_gemm);
+            mma_acc(acc, a_desc + 6, b_desc + 6, idesc_gemm);
+            mma_commit(&empty[st_a]);
+            if (f.dual) {
+              if (first) mma_set(acc + 32, a2_desc, b_desc, idesc_gemm); else mma_acc(acc + 32, a2_desc, b_desc, idesc_gemm);
+              mma_acc(acc + 32, a2_desc + 2, b_desc + 2, idesc_gemm);
+              mma_acc(acc + 32, a2_desc + 4, b_desc + 4, idesc_gemm);
+              mma_acc(acc + 32, a2_desc + 6, b_desc + 6, idesc_gemm);
+              mma_commit(&empty[st_b]);
+            }
+            VVS_TRACE(0x280 | (ph << 4) | (s - lo));
+            if (++kb == f.kbs) kb = 0;
           }
-          if (alive && cur_tile >= 0) mma_commit(&acc_full[slot]);
+          if (alive && hi > lo) mma_commit(&acc_full[slot]);
         }
       }
     }
@@ -354,11 +482,13 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
     const int tid_g = grp_e ? tid - 64 : tid - 192;   // index inside the group of 128
     const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
     unsigned target = epoch;
-    uint32_t itb = 0, ita = 0, iatt = 0;
+    uint32_t it_slab = 0, ita = 0, iatt = 0;         // ring position at the start of the phase, items, att items
 
     auto grid_sync = [&]() {
+      if (tid_w == 0) VVS_TRACE(0x900);
       named_bar_sync(BAR_W, kWorkers);
       target += (unsigned)G;
+      if (tid_w == 0) VVS_TRACE(0x901);
       if (tid_w == 0 && !s_abort) {
         __threadfence();
         atomicAdd(p.sync_words, 1u);
@@ -372,6 +502,7 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
           *reinterpret_cast<volatile unsigned*>(p.sync_words + 2) = 1u;
           atomicOr(p.status, VVS_DEV_TIMEOUT);
         }
+        VVS_TRACE(0x902);
       }
       named_bar_sync(BAR_W, kWorkers);
     };
@@ -389,10 +520,14 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
       const int gtid = blockIdx.x * kWorkers + tid_w, gstride = G * kWorkers;
       const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
       const int nq = (2 * p.m * 3 * p.d) >> 2, ng = (2 * p.m * 2 * p.ff) >> 2, ns = (2 * L * 32) >> 2;
+#pragma unroll 1
       for (int i = gtid; i < nq; i += gstride) reinterpret_cast<float4*>(p.qkv_acc)[i] = z;
+#pragma unroll 1
       for (int i = gtid; i < ng; i += gstride) reinterpret_cast<float4*>(p.gu_acc)[i] = z;
+#pragma unroll 1
       for (int i = gtid; i < ns; i += gstride) reinterpret_cast<float4*>(p.ss)[i] = z;
       const int per_row = p.d >> 3;
+#pragma unroll 1
       for (int i = gtid; i < p.m * per_row; i += gstride) {
         const int tok = i / per_row, ch = i - tok * per_row;
         const int r = tok / T, t = tok - r * T, b = r % p.n_images;
@@ -409,53 +544,65 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
       grid_sync();
     }
 
-    // per-thread constants of the operand builders
+    // per-thread constants of the merge builders (128 threads per unit: token, 16 columns)
     const int b_tok = tid_g >> 2, b_qtr = tid_g & 3;
     const int b_r = b_tok / T, b_t = b_tok - b_r * T;
 
+#pragma unroll 1
     for (int l = 0; l < L; ++l) {
       const int par_l = l & 1;
       float* qkv = p.qkv_acc + (size_t)par_l * p.m * 3 * p.d;
       float* gu = p.gu_acc + (size_t)par_l * p.m * 2 * p.ff;
+#pragma unroll 1
       for (int ph = 0; ph < 4; ++ph) {
         if (ph == PH_O) {
           // ================================ attention ================================================
           int n_mine = 0;
+#pragma unroll 1
           for (int i = blockIdx.x; i < n_items; i += G, ++iatt, ++n_mine) {
             int r, h, c;
             decode_item(i, r, h, c);
             const uint32_t par = iatt & 1;
             const int fill = s_fill[r], n_keys = fill + T, key0 = c * 128;
             const int row_base = kv_row_base(l, r, h, c);
+            const int per_head = p.hd >> 3;
             if (!grp_e) {
               if (tid_g == 0 && n_mine > 0) issue_kv(l, i);   // the first item was requested a layer ahead
               // Q operand: q * (1/rms) rotated, bf16, K-major with the 128-byte swizzle
-              const int per_head = p.hd >> 3;
+#pragma unroll 1
               for (int idx = tid_g; idx < T * per_head; idx += kGroup) {
                 const int t = idx / per_head, ch = idx - t * per_head, e = ch << 3, tok = r * T + t;
-                const float rinv = rsqrtf(__ldcg(p.ss + (2 * l) * 32 + tok) / (float)p.d + p.eps);
+                const float ssv = __ldcg(p.ss + (2 * l) * 32 + tok);
                 float v[8];
                 ldcg8(qkv + (size_t)tok * 3 * p.d + h * p.hd + e, v);
+                const float rinv = rsqrtf(ssv / (float)p.d + p.eps);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) v[j] *= rinv;
                 rope8(p, tok, e, v);
                 uint8_t* dst = sQ + (e >> 6) * q_chunk_bytes + t * 128 + ((((e & 63) >> 3) ^ (t & 7)) << 4);
                 *reinterpret_cast<uint4*>(dst) = pack8(v);
               }
+              fence_proxy_async();
+              if (tid_g == 0) VVS_TRACE(0x3A1);
+              named_bar_sync(BAR_D, kGroup);
+              if (tid_g == 0) mbar_arrive(&att_q_ready);
+            } else {
               // the block's own K / V rows inside this chunk: cache append + patch of the staged tiles
               const int new_lo = fill > key0 ? fill : key0;
               const int new_hi = n_keys < key0 + 128 ? n_keys : key0 + 128;
               if (new_lo < new_hi) {
                 wait_bar(&att_kv_full, par, &s_abort, p.status);
                 const int n_new = new_hi - new_lo;
+#pragma unroll 1
                 for (int idx = tid_g; idx < n_new * per_head * 2; idx += kGroup) {
                   const int which = idx / (n_new * per_head);       // 0 = K, 1 = V
                   const int rem = idx - which * n_new * per_head;
                   const int kk = rem / per_head, ch = rem - kk * per_head, e = ch << 3;
                   const int key = new_lo + kk, t = key - fill, tok = r * T + t;
-                  const float rinv = rsqrtf(__ldcg(p.ss + (2 * l) * 32 + tok) / (float)p.d + p.eps);
+                  const float ssv = __ldcg(p.ss + (2 * l) * 32 + tok);
                   float v[8];
                   ldcg8(qkv + (size_t)tok * 3 * p.d + (which + 1) * p.d + h * p.hd + e, v);
+                  const float rinv = rsqrtf(ssv / (float)p.d + p.eps);
 #pragma unroll
                   for (int j = 0; j < 8; ++j) v[j] *= rinv;
                   if (which == 0) rope8(p, tok, e, v);
@@ -468,38 +615,58 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
                 }
               }
               fence_proxy_async();
-              named_bar_sync(BAR_D, kGroup);
+              if (tid_g == 0) VVS_TRACE(0x4A1);
+              named_bar_sync(BAR_E, kGroup);
               if (tid_g == 0) mbar_arrive(&att_q_ready);
-            } else {
               // scores: this thread owns key (quarter * 32 + lane) of the chunk
               wait_bar(&att_s_full, par, &s_abort, p.status);
               tc_fence_after();
-              const int kl = quarter * 32 + lane, key = key0 + kl;
+              if (tid_g == 0) VVS_TRACE(0x4A2);
+              const int kl = quarter * 32 + lane;
               const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + kColS;
-              float s[32];
-              tmem_ld16(t_row, s);
-              if (p.tq > 16) tmem_ld16(t_row + 16, s + 16);
+              {
+                // scores of this key for all queries -> shared memory, transposed ([query][key], fp32;
+                // kept in rows of the P tiles that belong to no query)
+                float sc[32];
+                tmem_ld16(t_row, sc);
+                if (p.tq > 16) tmem_ld16(t_row + 16, sc + 16);
 #pragma unroll
-              for (int t = 0; t < 32; ++t) {
-                if (t < T) {
-                  s[t] = (key <= fill + t) ? s[t] * p.scale : -CUDART_INF_F;
-                  const float wm = warp_max_f(s[t]);
-                  if (lane == 0) red_max[quarter][t] = wm;
-                }
+                for (int t = 0; t < 32; ++t)
+                  if (t < p.tq) reinterpret_cast<float*>(sP + (t >> 4) * kSlabBytes + 4096)[(t & 15) * 128 + kl] = sc[t];
               }
               named_bar_sync(BAR_E, kGroup);
+              // one warp per query row: mask, max, exp, sum; lane owns keys 4*lane .. 4*lane+3
+#pragma unroll 1
+              for (int t = quarter; t < T; t += 4) {
+                const float4 s4 = reinterpret_cast<const float4*>(sP + (t >> 4) * kSlabBytes + 4096)[(t & 15) * 32 + lane];
+                float sv[4] = {s4.x, s4.y, s4.z, s4.w};
+                float mx = -CUDART_INF_F;
 #pragma unroll
-              for (int t = 0; t < 32; ++t) {
-                if (t < T) {
-                  const float mx = fmaxf(fmaxf(red_max[0][t], red_max[1][t]), fmaxf(red_max[2][t], red_max[3][t]));
-                  const float e = (s[t] == -CUDART_INF_F) ? 0.f : expf(s[t] - mx);
-                  const float ws = warp_sum_f(e);
-                  if (lane == 0) red_sum[quarter][t] = ws;
-                  uint8_t* dst = sP + (kl >> 6) * kSlabBytes + t * 128 + (((((kl & 63) >> 3) ^ (t & 7)) << 4) | ((kl & 7) << 1));
-                  *reinterpret_cast<__nv_bfloat16*>(dst) = __float2bfloat16_rn(e);
+                for (int j = 0; j < 4; ++j) {
+                  sv[j] = (key0 + 4 * lane + j <= fill + t) ? sv[j] * p.scale : -CUDART_INF_F;
+                  mx = fmaxf(mx, sv[j]);
                 }
+                mx = warp_max_f(mx);
+                float sum = 0.f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  sv[j] = (sv[j] == -CUDART_INF_F) ? 0.f : __expf(sv[j] - mx);
+                  sum += sv[j];
+                }
+                sum = warp_sum_f(sum);
+                if (lane == 0) {
+                  row_max[t] = mx;
+                  row_sum[t] = sum;
+                }
+                // P[t, key] as bf16, K-major rows of 64 keys with the 128-byte swizzle
+                const int k4 = 4 * lane;
+                uint2 pk;
+                *reinterpret_cast<__nv_bfloat162*>(&pk.x) = __floats2bfloat162_rn(sv[0], sv[1]);
+                *reinterpret_cast<__nv_bfloat162*>(&pk.y) = __floats2bfloat162_rn(sv[2], sv[3]);
+                uint8_t* dst = sP + (k4 >> 6) * kSlabBytes + t * 128 + (((((k4 & 63) >> 3) ^ (t & 7)) << 4) | ((k4 & 7) << 1));
+                *reinterpret_cast<uint2*>(dst) = pk;
               }
-              if (key >= n_keys) {   // slots no query may see: cleared so stale contents cannot inject NaN
+              if (key0 + kl >= n_keys) {   // slots no query may see: cleared so stale contents cannot inject NaN
                 for (int j = 0; j < NC; ++j) {
                   uint4* row = reinterpret_cast<uint4*>(sV + j * kSlabBytes + kl * 128);
 #pragma unroll
@@ -508,14 +675,17 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
               }
               fence_proxy_async();
               tc_fence_before();
+              if (tid_g == 0) VVS_TRACE(0x4A3);
               named_bar_sync(BAR_E, kGroup);
               if (tid_g == 0) mbar_arrive(&att_p_ready);
             }
             wait_bar(&att_o_full, par, &s_abort, p.status);
             tc_fence_after();
+            if (tid_w == 0) VVS_TRACE(0x4A4);
             if (grp_e && quarter == 0) {                  // TMEM lanes 0..31 = query rows
               const size_t rh = (size_t)r * H + h;
               const size_t slot = (rh * p.n_chunks_max + c) * T + lane;
+#pragma unroll 1
               for (int e0 = 0; e0 < p.hd; e0 += 32) {
                 float o[32];
                 tmem_ld32(tmem_base + kColO + e0, o);
@@ -526,11 +696,12 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
                 }
               }
               if (lane < T) {
-                p.part_ml[slot * 2] = fmaxf(fmaxf(red_max[0][lane], red_max[1][lane]), fmaxf(red_max[2][lane], red_max[3][lane]));
-                p.part_ml[slot * 2 + 1] = red_sum[0][lane] + red_sum[1][lane] + red_sum[2][lane] + red_sum[3][lane];
+                p.part_ml[slot * 2] = row_max[lane];
+                p.part_ml[slot * 2 + 1] = row_sum[lane];
               }
             }
             tc_fence_before();
+            if (tid_w == 64) VVS_TRACE(0x4A5);
             named_bar_sync(BAR_W, kWorkers);
           }
           if (!grp_e && tid_g == 0 && l + 1 < L && (int)blockIdx.x < n_items) issue_kv(l + 1, blockIdx.x);
@@ -541,103 +712,135 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
         const Phase f = phase_of(p, ph);
         int lo, hi;
         unit_range(f, l, ph, lo, hi);
-        if (!grp_e) {
-          // ---- operand builders ----
-          for (int s = lo; s < hi; ++s, ++itb) {
-            const int tile = s / f.kbs, kb = s - tile * f.kbs;
-            const uint32_t bst = itb % kTokStages, use = itb / kTokStages;
-            if (use > 0) wait_bar(&b_empty[bst], (use - 1) & 1, &s_abort, p.status);
-            uint8_t* slab = tokring + bst * kTokSlabBytes;
-            const int k0 = kb * 64 + b_qtr * 16;
-            float v[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = 0.f;
-            float ssq = 0.f;
-            if (b_tok < p.m) {
-              if (ph == PH_QKV || ph == PH_GU) {
-                const int which = ph == PH_GU ? 1 : 0;
-                float xv[16], gv[16];
-                ldcg8(p.x + (size_t)b_tok * p.d + k0, xv);
-                ldcg8(p.x + (size_t)b_tok * p.d + k0 + 8, xv + 8);
-                const uint4* g = reinterpret_cast<const uint4*>(p.norms[l * 2 + which] + k0);
-                unpack8(__ldg(g), gv);
-                unpack8(__ldg(g + 1), gv + 8);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                  ssq = fmaf(xv[j], xv[j], ssq);
-                  v[j] = xv[j] * gv[j];
-                }
-              } else if (ph == PH_O) {
+        const int n_units = hi - lo;
+        const uint32_t per_unit = 1u + (uint32_t)f.dual;
+
+        // ---- token operands of this CTA's units, built by all eight worker warps at once ----
+        if (ph == PH_O) {
+          // merge of the split-KV attention partials: one group of 128 threads per unit
+          // (thread = token, 16 columns), two units per round
+#pragma unroll 1
+          for (int b0 = 0; b0 < n_units; b0 += 2) {
+            const int k = b0 + (grp_e ? 1 : 0);
+            if (k < n_units) {
+              const uint32_t it = it_slab + (uint32_t)k, st = it % NS, use = it / NS;
+              if (use > 0) wait_bar(&empty[st], (use - 1) & 1, &s_abort, p.status);
+              if (b_tok < p.m) {
+                const int kb = (lo + k) % f.kbs;
+                const int k0 = kb * 64 + b_qtr * 16;
                 const int h = k0 / p.hd, e = k0 - h * p.hd;
                 const int nch = s_nch[b_r];
                 const size_t base = (((size_t)b_r * H + h) * p.n_chunks_max) * T + b_t;
-                float mx = -CUDART_INF_F;
-                for (int c = 0; c < nch; ++c) mx = fmaxf(mx, __ldcg(p.part_ml + (base + (size_t)c * T) * 2));
-                float den = 0.f;
-                for (int c = 0; c < nch; ++c) {
-                  const size_t slot = base + (size_t)c * T;
-                  const float mc = __ldcg(p.part_ml + slot * 2);
-                  const float w = (mc == -CUDART_INF_F) ? 0.f : expf(mc - mx);
-                  den = fmaf(w, __ldcg(p.part_ml + slot * 2 + 1), den);
-                  float o[16];
-                  ldcg8(p.part_o + slot * p.hd + e, o);
-                  ldcg8(p.part_o + slot * p.hd + e + 8, o + 8);
+                float v[16];
 #pragma unroll
-                  for (int j = 0; j < 16; ++j) v[j] = fmaf(w, o[j], v[j]);
+                for (int j = 0; j < 16; ++j) v[j] = 0.f;
+                float mrun = -CUDART_INF_F, den = 0.f;
+#pragma unroll 1
+                for (int c0 = 0; c0 < nch; c0 += 4) {   // four chunks in flight at once
+                  float mc[4], lc[4], o[4][16];
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    if (c0 + j < nch) {
+                      const size_t slot = base + (size_t)(c0 + j) * T;
+                      const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + slot * 2));
+                      mc[j] = ml.x;
+                      lc[j] = ml.y;
+                      ldcg8(p.part_o + slot * p.hd + e, o[j]);
+                      ldcg8(p.part_o + slot * p.hd + e + 8, o[j] + 8);
+                    } else {
+                      mc[j] = -CUDART_INF_F;
+                      lc[j] = 0.f;
+#pragma unroll
+                      for (int q = 0; q < 16; ++q) o[j][q] = 0.f;
+                    }
+                  }
+                  const float mnew = fmaxf(fmaxf(mrun, mc[0]), fmaxf(fmaxf(mc[1], mc[2]), mc[3]));
+                  if (mnew == -CUDART_INF_F) continue;
+                  const float keep = (mrun == -CUDART_INF_F) ? 0.f : __expf(mrun - mnew);
+                  den *= keep;
+#pragma unroll
+                  for (int q = 0; q < 16; ++q) v[q] *= keep;
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    const float w = (mc[j] == -CUDART_INF_F) ? 0.f : __expf(mc[j] - mnew);
+                    den = fmaf(w, lc[j], den);
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) v[q] = fmaf(w, o[j][q], v[q]);
+                  }
+                  mrun = mnew;
                 }
                 const float inv = den > 0.f ? 1.f / den : 0.f;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] *= inv;
-              } else {
-                const float rinv = rsqrtf(__ldcg(p.ss + (2 * l + 1) * 32 + b_tok) / (float)p.d + p.eps);
-                const float* gp = gu + (size_t)b_tok * 2 * p.ff + k0;
-#pragma unroll
-                for (int c8 = 0; c8 < 2; ++c8) {
-                  if (k0 + c8 * 8 < p.ff) {
-                    float gt[8], up[8];
-                    ldcg8(gp + c8 * 8, gt);
-                    ldcg8(gp + p.ff + c8 * 8, up);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                      const float a = gt[j] * rinv;
-                      v[c8 * 8 + j] = a / (1.f + expf(-a)) * (up[j] * rinv);
-                    }
-                  }
-                }
+                for (int q = 0; q < 16; ++q) v[q] *= inv;
+                uint8_t* row = ring + (size_t)st * kStageBytes + kSlabBytes + b_tok * 128;
+                *reinterpret_cast<uint4*>(row + (((2 * b_qtr) ^ (b_tok & 7)) << 4)) = pack8(v);
+                *reinterpret_cast<uint4*>(row + (((2 * b_qtr + 1) ^ (b_tok & 7)) << 4)) = pack8(v + 8);
               }
-              uint8_t* row = slab + b_tok * 128;
-              *reinterpret_cast<uint4*>(row + (((2 * b_qtr) ^ (b_tok & 7)) << 4)) = pack8(v);
-              *reinterpret_cast<uint4*>(row + (((2 * b_qtr + 1) ^ (b_tok & 7)) << 4)) = pack8(v + 8);
-            }
-            if ((ph == PH_QKV || ph == PH_GU) && tile == 0) {
-              // sum of squares of the row, once per k-block (the CTAs that own tile 0)
-              ssq += __shfl_xor_sync(0xffffffffu, ssq, 1);
-              ssq += __shfl_xor_sync(0xffffffffu, ssq, 2);
-              if (b_qtr == 0 && b_tok < p.m) atomicAdd(p.ss + (2 * l + (ph == PH_GU ? 1 : 0)) * 32 + b_tok, ssq);
             }
             fence_proxy_async();
-            named_bar_sync(BAR_D, kGroup);
-            if (tid_g == 0) mbar_arrive(&b_full[bst]);
+            if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | b0);
+            named_bar_sync(BAR_W, kWorkers);
+            if (tid_w < 2 && b0 + tid_w < n_units) mbar_arrive(&full[(it_slab + (uint32_t)(b0 + tid_w)) % NS]);
           }
+        } else {
+          // x * norm scale (QKV, gate/up) or silu(gate) * up (down): up to four units per round
+          // (64 threads per unit), up to eight (32 threads per unit) for the norm operands
+          const int which = ph == PH_GU ? 1 : 0;
+          const __nv_bfloat16* gsc = p.norms[l * 2 + which];
+          int b0 = 0;
+#pragma unroll 1
+          while (b0 < n_units) {
+            const int left = n_units - b0;
+            const int cap = (ph != PH_DOWN && left > 4) ? 8 : 4;
+            const int nb = left < cap ? left : cap;
+            const int lg = nb <= 1 ? 0 : nb <= 2 ? 1 : nb <= 4 ? 2 : 3;
+            const uint32_t it0 = it_slab + (uint32_t)b0 * per_unit;
+            if (ph == PH_DOWN)
+              build_round<8, true>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, gu, nullptr,
+                                   p.ss + (2 * l + 1) * 32, nullptr);
+            else if (lg == 3)
+              build_round<16, false>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, p.x, gsc,
+                                     nullptr, p.ss + (2 * l + which) * 32);
+            else
+              build_round<8, false>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, p.x, gsc,
+                                    nullptr, p.ss + (2 * l + which) * 32);
+            fence_proxy_async();
+            if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | b0);
+            named_bar_sync(BAR_W, kWorkers);
+            if (tid_w < nb) {
+              const uint32_t it = it0 + (uint32_t)tid_w * per_unit;
+              mbar_arrive(&full[it % NS]);
+              if (f.dual) mbar_arrive(&full[(it + 1) % NS]);
+            }
+            b0 += nb;
+          }
+        }
+        it_slab += (uint32_t)n_units * per_unit;
+
+        if (!grp_e) {
           if (ph == PH_O && l + 1 < L) {
             // clear the accumulators the next layer adds into (last read one layer ago)
             const int gtid = blockIdx.x * kGroup + tid_g, gstride = G * kGroup;
             const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
             float4* q4 = reinterpret_cast<float4*>(p.qkv_acc + (size_t)(par_l ^ 1) * p.m * 3 * p.d);
             float4* g4 = reinterpret_cast<float4*>(p.gu_acc + (size_t)(par_l ^ 1) * p.m * 2 * p.ff);
+#pragma unroll 1
             for (int i = gtid; i < (p.m * 3 * p.d) >> 2; i += gstride) q4[i] = z;
+#pragma unroll 1
             for (int i = gtid; i < (p.m * 2 * p.ff) >> 2; i += gstride) g4[i] = z;
           }
         } else {
           // ---- epilogue: accumulators -> fp32 sums in L2 ----
           int s = lo;
+#pragma unroll 1
           while (s < hi) {
             const int tile = s / f.kbs;
             int next = (tile + 1) * f.kbs;
             s = next < hi ? next : hi;
             const uint32_t slot = ita % kAccSlots;
-            wait_bar(&acc_full[slot], (ita / kAccSlots) & 1, &s_abort, p.status);
+            wait_fast(&acc_full[slot], (ita / kAccSlots) & 1, &s_abort, p.status);
             tc_fence_after();
+            if (tid_g == 0) VVS_TRACE(0x400 | (ph << 4));
             const int n = tile * 128 + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + slot * 64;
             float* dst;
@@ -648,19 +851,26 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
             float v[32];
             tmem_ld32(taddr, v);
             if (n < nlim) {
+              float* ptr = dst + n;
 #pragma unroll
-              for (int tok = 0; tok < 32; ++tok)
-                if (tok < p.m) red_add_f32(dst + (size_t)tok * ld + n, v[tok]);
+              for (int tok = 0; tok < 32; ++tok) {
+                if (tok < p.m) red_add_f32(ptr, v[tok]);
+                ptr += ld;
+              }
             }
             if (f.dual) {
               tmem_ld32(taddr + 32, v);
               if (n < nlim) {
+                float* ptr = dst + p.ff + n;
 #pragma unroll
-                for (int tok = 0; tok < 32; ++tok)
-                  if (tok < p.m) red_add_f32(dst + (size_t)tok * ld + p.ff + n, v[tok]);
+                for (int tok = 0; tok < 32; ++tok) {
+                  if (tok < p.m) red_add_f32(ptr, v[tok]);
+                  ptr += ld;
+                }
               }
             }
             tc_fence_before();
+            if (tid_g == 0) VVS_TRACE(0x480 | (ph << 4));
             named_bar_sync(BAR_E, kGroup);
             if (tid_g == 0) mbar_arrive(&acc_empty[slot]);
             ++ita;
@@ -684,20 +894,19 @@ fused_chain_kernel(const ChainParams p, const __grid_constant__ CUtensorMap tm_k
 
 bool fused_chain_applicable(const vvs_model_desc& md, int n_rows, int t_len) {
   if (md.dtype != VVS_DTYPE_BF16 || md.n_layers < 1) return false;
-  if (n_rows * t_len > 32 || n_rows > kMaxSeq) return false;
+  if (n_rows * t_len > 32 || n_rows > kMaxSeq || md.n_layers > kMaxLayers) return false;
   if (md.d_model % 64 != 0 || md.d_ff % 8 != 0) return false;
   return true;
 }
 
-size_t fused_chain_smem_bytes(const vvs_model_desc& md, int t_len, int* w_stages) {
+size_t fused_chain_smem_bytes(const vvs_model_desc& md, int t_len, int* n_stages) {
   const int nc = md.head_dim / 64, tq = t_len <= 16 ? 16 : 32;
-  const size_t fixed = 1024 + (size_t)kTokStages * kTokSlabBytes + (size_t)2 * nc * kSlabBytes +
-                       2 * kSlabBytes + (size_t)nc * tq * 128;
+  const size_t fixed = 1024 + (size_t)2 * nc * kSlabBytes + 2 * kSlabBytes + (size_t)nc * tq * 128;
   const size_t budget = 226 * 1024;   // leaves room for the static barriers and tables
-  int stages = (int)((budget - fixed) / kSlabBytes);
-  if (stages > kMaxWStages) stages = kMaxWStages;
-  if (w_stages) *w_stages = stages;
-  return fixed + (size_t)stages * kSlabBytes;
+  int stages = (int)((budget - fixed) / kStageBytes);
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (n_stages) *n_stages = stages;
+  return fixed + (size_t)stages * kStageBytes;
 }
 
 int launch_fused_chain(const FusedChainArgs& a, cudaStream_t s) {
@@ -709,15 +918,16 @@ int launch_fused_chain(const FusedChainArgs& a, cudaStream_t s) {
   p.n_rows = a.n_rows; p.n_images = a.n_images; p.tok_rows = md.tok_rows;
   p.n_chunks_max = (md.s_max + 127) / 128;
   p.eps = md.rms_eps; p.scale = 1.0f / sqrtf((float)md.head_dim);
-  p.wmaps = a.wmaps; p.norms = a.norms; p.tok_emb = a.tok_emb; p.block = a.block;
+  p.wmaps = a.wmaps; p.tok_emb = a.tok_emb; p.block = a.block;
+  for (int i = 0; i < 2 * md.n_layers; ++i) p.norms[i] = a.norms_host[i];
   p.x = a.x; p.qkv_acc = a.qkv_acc; p.gu_acc = a.gu_acc; p.ss = a.ss;
   p.cache_len = a.cache_len; p.kv_k = a.kv_k; p.kv_v = a.kv_v;
-  p.slot_pos = a.slot_pos; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin;
+  p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin;
   p.part_o = a.part_o; p.part_ml = a.part_ml; p.sync_words = a.sync_words; p.status = a.status;
   int stages = 0;
   const size_t smem = fused_chain_smem_bytes(md, a.t_len, &stages);
   if (stages < 3) return VVS_ERR_SHAPE;
-  p.w_stages = stages;
+  p.n_stages = stages;
   static size_t configured = 0;
   if (configured < smem) {
     if (cudaFuncSetAttribute(fused_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)

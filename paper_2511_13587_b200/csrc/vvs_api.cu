@@ -56,7 +56,6 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
       c.take(ws.attn_part_ml, rh * chunks * d.max_block * 2 * 4);
       c.take(ws.attn_counters, rh * 4);
       c.take(ws.chain_wmaps, (size_t)d.n_layers * 5 * sizeof(CUtensorMap));
-      c.take(ws.chain_norms, (size_t)d.n_layers * 2 * sizeof(void*));
       c.take(ws.chain_qkv, (size_t)2 * 32 * 3 * dm * 4);
       c.take(ws.chain_gu, (size_t)2 * 32 * 2 * ff * 4);
       c.take(ws.chain_ss, (size_t)2 * d.n_layers * 32 * 4);
@@ -269,7 +268,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     // at most 32 tokens: the whole decoder chain runs as one persistent kernel
     FusedChainArgs fc{};
     fc.md = &md; fc.n_rows = R; fc.n_images = B; fc.t_len = Tn; fc.kv_rows = a->kv_rows; fc.n_sms = ctx->n_sms;
-    fc.wmaps = ws.chain_wmaps; fc.norms = ws.chain_norms;
+    fc.wmaps = ws.chain_wmaps; fc.norms_host = ctx->chain_norms.data();
     fc.tok_emb = static_cast<const T*>(ctx->tok_emb); fc.block = a->block;
     fc.x = ws.x; fc.qkv_acc = ws.chain_qkv; fc.gu_acc = ws.chain_gu; fc.ss = ws.chain_ss;
     fc.cache_len = a->cache_len; fc.kv_k = kv_k; fc.kv_v = kv_v; fc.tm_k = &tm_k; fc.tm_v = &tm_v;
@@ -535,14 +534,12 @@ int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w) {
     if (n > 0) {
       // device copies for the whole-chain kernel, which walks all layers inside one launch
       static_assert(sizeof(LayerMaps) == 5 * sizeof(CUtensorMap), "LayerMaps is five descriptors");
-      std::vector<const void*> norms(2 * (size_t)n);
+      ctx->chain_norms.resize(2 * (size_t)n);
       for (int l = 0; l < n; ++l) {
-        norms[2 * l] = w->layers[l].norm1;
-        norms[2 * l + 1] = w->layers[l].norm2;
+        ctx->chain_norms[2 * l] = static_cast<const __nv_bfloat16*>(w->layers[l].norm1);
+        ctx->chain_norms[2 * l + 1] = static_cast<const __nv_bfloat16*>(w->layers[l].norm2);
       }
       if (cudaMemcpy(ctx->ws.chain_wmaps, ctx->layer_maps, (size_t)n * sizeof(LayerMaps),
-                     cudaMemcpyHostToDevice) != cudaSuccess ||
-          cudaMemcpy(ctx->ws.chain_norms, norms.data(), norms.size() * sizeof(void*),
                      cudaMemcpyHostToDevice) != cudaSuccess)
         return VVS_ERR_CUDA;
     }

@@ -54,7 +54,6 @@ struct Workspace {
   int* attn_counters = nullptr;  // [R*H] split-KV arrival counters; zero between kernels
   // whole-chain kernel (at most 32 block tokens)
   CUtensorMap* chain_wmaps = nullptr;          // [n_layers][5] weight descriptors, device copy
-  const __nv_bfloat16** chain_norms = nullptr; // [n_layers][2] norm-scale pointers, device copy
   float* chain_qkv = nullptr;    // [2][32, 3d] fp32 split-K sums of the QKV projection (by layer parity)
   float* chain_gu = nullptr;     // [2][32, 2ff] fp32 split-K sums of gate | up
   float* chain_ss = nullptr;     // [2 * n_layers][32] sums of squares of the residual rows
@@ -97,6 +96,7 @@ struct vvs_ctx {
   bool use_pdl = true;               // programmatic dependent launch of the tensor-core GEMMs
   bool use_chain = true;             // whole-chain persistent kernel for calls of at most 32 tokens
   vvs::LayerMaps* layer_maps = nullptr;  // host array [n_layers]
+  std::vector<const __nv_bfloat16*> chain_norms;  // host [n_layers][2] norm-scale pointers
   CUtensorMap lm_map;
   int n_sms = 148;
   // CUDA-graph replay of vvs_verify (one graph per distinct argument set, small LRU cache)
@@ -189,7 +189,7 @@ struct FusedChainArgs {
   const vvs_model_desc* md;
   int n_rows, n_images, t_len, kv_rows, n_sms;
   const CUtensorMap* wmaps;             // device
-  const __nv_bfloat16* const* norms;    // device
+  const __nv_bfloat16* const* norms_host;  // HOST array [n_layers][2] of device pointers
   const __nv_bfloat16* tok_emb;
   const int32_t* block;
   float* x; float* qkv_acc; float* gu_acc; float* ss;
