@@ -286,10 +286,12 @@ int vvs_last_launch_count(const vvs_ctx* ctx);
 /* Per-kernel-class device timing for roofline reports.  While enabled, every launch of
  * vvs_verify / vvs_epilogue is bracketed by CUDA events on the call's stream (this costs time:
  * never enable it around a headline measurement).  Classes: 0 = projection / LM-head GEMMs,
- * 1 = attention, 2 = everything else.  vvs_profile_read synchronises the stream, ADDS the
- * milliseconds and launch counts recorded since the last read to ms[3] / launches[3] (host
- * arrays) and forgets them.  Events are created by vvs_profile_enable, not on the verify path. */
-enum { VVS_PROF_GEMM = 0, VVS_PROF_ATTENTION = 1, VVS_PROF_OTHER = 2, VVS_PROF_CLASSES = 3 };
+ * 1 = attention, 2 = everything else, 3 = the whole-chain kernel (embedding and every decoder
+ * layer in one launch; used by calls of at most 32 block tokens, which then have no class-0 / 1
+ * launches except the LM head).  vvs_profile_read synchronises the stream, ADDS the milliseconds
+ * and launch counts recorded since the last read to ms[4] / launches[4] (host arrays) and forgets
+ * them.  Events are created by vvs_profile_enable, not on the verify path. */
+enum { VVS_PROF_GEMM = 0, VVS_PROF_ATTENTION = 1, VVS_PROF_OTHER = 2, VVS_PROF_CHAIN = 3, VVS_PROF_CLASSES = 4 };
 int vvs_profile_enable(vvs_ctx* ctx, int on);
 int vvs_profile_read(vvs_ctx* ctx, void* stream, float* ms, int32_t* launches);
 

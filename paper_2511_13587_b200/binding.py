@@ -281,8 +281,8 @@ def vvs_profile_enable(ctx: int, on: bool) -> None:
 
 def vvs_profile_read(ctx: int, stream=None):
     """Returns ([ms per class], [launches per class]) accumulated since the last read;
-    classes: 0 GEMM, 1 attention, 2 other."""
-    ms = (C.c_float * 3)(0, 0, 0)
-    n = (C.c_int32 * 3)(0, 0, 0)
+    classes: 0 GEMM, 1 attention, 2 other, 3 whole-chain kernel."""
+    ms = (C.c_float * 4)(0, 0, 0, 0)
+    n = (C.c_int32 * 4)(0, 0, 0, 0)
     _check(lib.vvs_profile_read(ctx, _stream(stream), ms, n), "vvs_profile_read")
     return list(ms), list(n)

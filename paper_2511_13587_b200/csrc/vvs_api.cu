@@ -276,7 +276,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     fc.part_o = ws.attn_part_o; fc.part_ml = ws.attn_part_ml; fc.sync_words = ws.chain_sync;
     fc.status = ws.status;
     VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, ws, md, R, Tn, s));
-    VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_fused_chain(fc, s));
+    VVS_LAUNCH(VVS_PROF_CHAIN, rc = launch_fused_chain(fc, s));
     if (rc != VVS_OK) return rc;
     VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
     if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
