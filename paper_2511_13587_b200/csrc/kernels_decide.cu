@@ -8,11 +8,6 @@
 
 namespace vvs {
 
-// The one definition of a target probability from a guided logit and its row statistics; every
-// kernel that emits or compares probabilities calls it, so decisions and emitted values agree
-// bit for bit.
-__device__ __forceinline__ float prob_of(float l, float m, float inv) { return expf(l - m) * inv; }
-
 __device__ __forceinline__ double warp_sum_d(double v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -62,8 +62,13 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
       c.take(ws.chain_sync, 256);
     }
   }
-  c.take(ws.logits_raw, M * V * 4);
-  c.take(ws.logits, M * V * 4);
+  // full logits exist only on the generic path (float32 contexts, or bf16 ones forced onto it)
+  if (d.dtype != VVS_DTYPE_BF16 || std::getenv("VVS_DEBUG_GENERIC")) {
+    c.take(ws.logits_raw, M * V * 4);
+    c.take(ws.logits, M * V * 4);
+  } else {
+    c.take(ws.sel_hid, (size_t)d.max_rows * dm * es);
+  }
   c.take(ws.part_m, n_tiles * M * 4);
   c.take(ws.part_s, n_tiles * M * 4);
   c.take(ws.stat_m, M * 4);
@@ -153,20 +158,39 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
 
 
   if (ctx->tensor_core_path) {
-    const GemmTcPlan plan = plan_gemm_tc(M, V, md.d_model, false, false, ctx->n_sms);
-    CUtensorMap tm_hid;
-    if (make_tmap_bf16_2d(&tm_hid, hid, (uint64_t)M, (uint64_t)md.d_model, (uint32_t)plan.nt) != VVS_OK)
+    // LM head with guidance, softmax partials and gathers fused into its epilogue; the one row
+    // per image that sampling needs comes from a second pass over the selected rows
+    CUtensorMap tm_hid, tm_sel;
+    if (make_tmap_bf16_2d(&tm_hid, hid, (uint64_t)M, (uint64_t)md.d_model, (uint32_t)lmhead_box_rows(BT)) != VVS_OK ||
+        make_tmap_bf16_2d(&tm_sel, ws.sel_hid, (uint64_t)R, (uint64_t)md.d_model, (uint32_t)lmhead_box_rows(B)) != VVS_OK)
       return VVS_ERR_CUDA;
-    GemmTcArgs g{};
-    g.m = M; g.n = V; g.k = md.d_model;
-    g.tm_a = &ctx->lm_map; g.tm_b = &tm_hid; g.pdl = ctx->use_pdl; g.status = ws.status;
-    g.out = ws.logits_raw; g.ldo = V;
+    LmHeadArgs la{};
+    la.v = V; la.k = md.d_model; la.bt = BT; la.n_cfg = C; la.tm_a = &ctx->lm_map; la.tm_b = &tm_hid;
+    la.pdl = ctx->use_pdl; la.cfg_scale = a->cfg_scale; la.inv_temp = 1.f / a->temperature;
+    la.part_m = ws.part_m; la.part_s = ws.part_s; la.logits_out = o->target_probs; la.status = ws.status;
+    la.rows_per_seq = rows_per_seq; la.first_row = first_row; la.n_draft_max = p.n_draft_max;
+    la.vocab_offset = md.vocab_offset; la.relaxed = (p.mode == VVS_MODE_RELAXED && p.nbr_k > 1) ? 1 : 0;
+    la.nbr_k = p.nbr_k; la.kmax = p.kmax; la.drafts_ld = drafts_ld; la.drafts = drafts;
+    la.row_ptr = p.row_ptr; la.col = p.col; la.l_tok = ws.l_tok; la.l_nbr = ws.l_nbr;
     int rc = VVS_OK;
-    VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_STORE, plan, g, s));
+    VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_lmhead_tc(la, s));
     if (rc != VVS_OK) return rc;
-  } else {
-    VVS_LAUNCH(VVS_PROF_GEMM, launch_gemm_nt<T>(hid, w_lm, ws.logits_raw, M, V, md.d_model, V, false, s));
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_finalize_stats(ws, (V + 127) / 128, BT, s));
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_accept(ws, p, s));
+    if (o->target_probs)
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_probs_from_logits(o->target_probs, ws, o->target_probs, BT, V, s));
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_gather_sel_rows(hid, ws.sel_row, ws.sel_hid, B, C, BT, md.d_model, s));
+    LmHeadArgs lr{};
+    lr.v = V; lr.k = md.d_model; lr.bt = B; lr.n_cfg = C; lr.tm_a = &ctx->lm_map; lr.tm_b = &tm_sel;
+    lr.pdl = ctx->use_pdl; lr.cfg_scale = a->cfg_scale; lr.inv_temp = 1.f / a->temperature; lr.status = ws.status;
+    lr.row_mode = 1; lr.sel_row = ws.sel_row; lr.stat_m = ws.stat_m; lr.stat_inv = ws.stat_inv; lr.p_row = ws.p_row;
+    VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_lmhead_tc(lr, s));
+    if (rc != VVS_OK) return rc;
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_residual_mass(ws, p, s));
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_sample(ws, p, s));
+    return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
   }
+  VVS_LAUNCH(VVS_PROF_GEMM, launch_gemm_nt<T>(hid, w_lm, ws.logits_raw, M, V, md.d_model, V, false, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_guide(ws.logits_raw, ws.logits, B, C, rows_per_seq, V, a->cfg_scale,
                                           1.f / a->temperature, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_row_stats(ws.logits, ws.part_m, ws.part_s, BT, V, s));

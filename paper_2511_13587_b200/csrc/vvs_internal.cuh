@@ -40,6 +40,7 @@ struct Workspace {
   int32_t* sel_row = nullptr;   // [B] decision row (b*T + t) the next token is sampled from, -1 none
   int32_t* sel_kind = nullptr;  // [B] 0 = residual of draft n, 1 = bonus
   float* p_row = nullptr;    // [B, V] target probabilities of the selected row
+  void* sel_hid = nullptr;   // [n_cfg * B, d] features of the selected rows (tensor-core LM head, row mode)
   double* r_part = nullptr;  // [B, n_chunks] per-chunk residual mass
   double* p_part = nullptr;  // [B, n_chunks] per-chunk target mass (fallback when residual is 0)
   float* rope_inv_freq = nullptr;  // [head_dim/2] angle per unit coordinate of each pair
@@ -121,6 +122,11 @@ namespace vvs {
 
 constexpr int kSampleChunk = 1024;  // codebook entries per residual-mass chunk
 
+// The one definition of a target probability from a guided logit and its row statistics; every
+// kernel that emits or compares probabilities calls it, so decisions and emitted values agree
+// bit for bit.
+__device__ __forceinline__ float prob_of(float l, float m, float inv) { return expf(l - m) * inv; }
+
 // ---- generic kernels (any storage type), kernels_generic.cu ---------------------------------
 template <typename T>
 void launch_embed(const T* tok_emb, const int32_t* block, float* x, int n_images, int n_cfg,
@@ -183,6 +189,27 @@ struct AttentionTcArgs {
   bool pdl;
 };
 int launch_attention_tc(const AttentionTcArgs& a, cudaStream_t s);
+
+// ---- LM head with fused decision epilogue, lmhead_tc.cu -------------------------------------------
+struct LmHeadArgs {
+  int v, k, bt, n_cfg;           // codebook size, d_model, decision rows, 1 or 2 feature rows per decision row
+  const CUtensorMap* tm_a;       // codebook rows of w_lm [v, k]
+  const CUtensorMap* tm_b;       // features [n_cfg * bt, k] (cond rows, then uncond rows), box rows = lmhead_box_rows(bt)
+  bool pdl;
+  float cfg_scale, inv_temp;
+  float* part_m; float* part_s;  // [n_tiles, bt] softmax partials per 128-code tile
+  float* logits_out;             // optional [bt, v] guided logits
+  int32_t* status;
+  int rows_per_seq, first_row, n_draft_max, vocab_offset, relaxed, nbr_k, kmax, drafts_ld;
+  const int32_t* drafts; const int32_t* row_ptr; const int32_t* col;
+  float* l_tok; float* l_nbr;
+  int row_mode;                  // 1: bt = images, write probabilities of the selected rows to p_row
+  const int32_t* sel_row; const float* stat_m; const float* stat_inv; float* p_row;
+};
+int lmhead_box_rows(int bt);
+int launch_lmhead_tc(const LmHeadArgs& a, cudaStream_t s);
+void launch_gather_sel_rows(const void* hid, const int32_t* sel_row, void* out, int n_images, int n_cfg, int bt,
+                            int d, cudaStream_t s);
 
 // ---- whole-chain persistent kernel, fused_chain.cu ---------------------------------------------
 struct FusedChainArgs {
