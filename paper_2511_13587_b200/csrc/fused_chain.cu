@@ -460,13 +460,17 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             mma_acc(acc, a_desc + 2, b_desc + 2, idesc_gemm);
             mma_acc(acc, a_desc + 4, b_desc + 4, idesc_gemm);
             mma_acc(acc, a_desc + 6, b_desc + 6, idesc_gemm);
-            mma_commit(&empty[st_a]);
             if (f.dual) {
+              // the second weight slab multiplies the token slab of the FIRST stage: that stage is
+              // released only after these have been issued as well
               if (first) mma_set(acc + 32, a2_desc, b_desc, idesc_gemm); else mma_acc(acc + 32, a2_desc, b_desc, idesc_gemm);
               mma_acc(acc + 32, a2_desc + 2, b_desc + 2, idesc_gemm);
               mma_acc(acc + 32, a2_desc + 4, b_desc + 4, idesc_gemm);
               mma_acc(acc + 32, a2_desc + 6, b_desc + 6, idesc_gemm);
+              mma_commit(&empty[st_a]);
               mma_commit(&empty[st_b]);
+            } else {
+              mma_commit(&empty[st_a]);
             }
             VVS_TRACE(0x280 | (ph << 4) | (s - lo));
             if (++kb == f.kbs) kb = 0;
@@ -585,7 +589,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               fence_proxy_async();
               if (tid_g == 0) VVS_TRACE(0x3A1);
               named_bar_sync(BAR_D, kGroup);
-              if (tid_g == 0) mbar_arrive(&att_q_ready);
+              if (tid_g == 0 && !s_abort) mbar_arrive(&att_q_ready);
             } else {
               // the block's own K / V rows inside this chunk: cache append + patch of the staged tiles
               const int new_lo = fill > key0 ? fill : key0;
@@ -617,7 +621,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               fence_proxy_async();
               if (tid_g == 0) VVS_TRACE(0x4A1);
               named_bar_sync(BAR_E, kGroup);
-              if (tid_g == 0) mbar_arrive(&att_q_ready);
+              if (tid_g == 0 && !s_abort) mbar_arrive(&att_q_ready);
               // scores: this thread owns key (quarter * 32 + lane) of the chunk
               wait_bar(&att_s_full, par, &s_abort, p.status);
               tc_fence_after();
@@ -677,7 +681,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               tc_fence_before();
               if (tid_g == 0) VVS_TRACE(0x4A3);
               named_bar_sync(BAR_E, kGroup);
-              if (tid_g == 0) mbar_arrive(&att_p_ready);
+              if (tid_g == 0 && !s_abort) mbar_arrive(&att_p_ready);
             }
             wait_bar(&att_o_full, par, &s_abort, p.status);
             tc_fence_after();
@@ -780,7 +784,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             fence_proxy_async();
             if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | b0);
             named_bar_sync(BAR_W, kWorkers);
-            if (tid_w < 2 && b0 + tid_w < n_units) mbar_arrive(&full[(it_slab + (uint32_t)(b0 + tid_w)) % NS]);
+            if (tid_w < 2 && b0 + tid_w < n_units && !s_abort) mbar_arrive(&full[(it_slab + (uint32_t)(b0 + tid_w)) % NS]);
           }
         } else {
           // x * norm scale (QKV, gate/up) or silu(gate) * up (down): up to four units per round
@@ -791,7 +795,12 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
 #pragma unroll 1
           while (b0 < n_units) {
             const int left = n_units - b0;
-            const int cap = (ph != PH_DOWN && left > 4) ? 8 : 4;
+            // A round may not reach around the ring: its threads wait for the slot of their own
+            // unit to be free before any of them reports a unit of the round as built, so two
+            // units of one round must never share a slot.
+            const int ring_cap = ((int)NS + (int)per_unit - 1) / (int)per_unit;
+            int cap = (ph != PH_DOWN && left > 4) ? 8 : 4;
+            if (cap > ring_cap) cap = ring_cap;
             const int nb = left < cap ? left : cap;
             const int lg = nb <= 1 ? 0 : nb <= 2 ? 1 : nb <= 4 ? 2 : 3;
             const uint32_t it0 = it_slab + (uint32_t)b0 * per_unit;
@@ -807,10 +816,16 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             fence_proxy_async();
             if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | b0);
             named_bar_sync(BAR_W, kWorkers);
-            if (tid_w < nb) {
+            if (tid_w < nb && !s_abort) {
               const uint32_t it = it0 + (uint32_t)tid_w * per_unit;
               mbar_arrive(&full[it % NS]);
-              if (f.dual) mbar_arrive(&full[(it + 1) % NS]);
+              if (f.dual) {
+                // the second stage of the unit holds no token slab, but its barrier must be in the
+                // phase of this use before it takes the arrival
+                const uint32_t it2 = it + 1, use2 = it2 / NS;
+                if (use2 > 0) wait_fast(&empty[it2 % NS], (use2 - 1) & 1, &s_abort, p.status);
+                if (!s_abort) mbar_arrive(&full[it2 % NS]);
+              }
             }
             b0 += nb;
           }
@@ -872,7 +887,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             tc_fence_before();
             if (tid_g == 0) VVS_TRACE(0x480 | (ph << 4));
             named_bar_sync(BAR_E, kGroup);
-            if (tid_g == 0) mbar_arrive(&acc_empty[slot]);
+            if (tid_g == 0 && !s_abort) mbar_arrive(&acc_empty[slot]);
             ++ita;
           }
         }

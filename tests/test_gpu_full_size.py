@@ -1,0 +1,65 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+configs[1]: the whole LlamaGen-XL shape (36 layers, d = 1280, V = 16384), batch 1 with guidance,
+K = 8: the oracle finishes one such step in seconds, so every output is compared.
+configs[3] / configs[2]: full width, head_dim, vocabulary slice and batch, at reduced depth (the
+layers repeat the same kernels with other weights; depth is covered by configs[1])."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import helpers as H
+from test_gpu_verify import _check_end_to_end
+from vvs_synth.configs import B7, CONFIGS, MODE_RELAXED, XL
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config1_full_llamagen_xl_shape():
+    """Fill 477 needs four 128-key chunks per (sequence, head), i.e. more attention work items
+    than SMs, and the block's own rows straddle no chunk boundary; the small-shape tests cover
+    the other fills."""
+    wl, fill = CONFIGS[1], 477
+    case = H.build_case(wl.shape, wl.seed + fill, 1, 2, 1, 8, [fill], cfg_scale=wl.cfg_scale, q_noise=0.3)
+    run = H.GpuRunner(wl.shape, case["w"], 2, 9)
+    gpu = run.verify(case)
+    assert gpu["launches"] < 40            # the whole-chain kernel ran, not one kernel per projection
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    print("configs[1] full size: accept_len", gpu["accept_len"], "oracle", ora["accept_len"])
+    # The configuration the benchmark times does not ask for probabilities.  Split-K sums are
+    # added in L2 in arrival order, so two runs differ in the last bits of the logits: the accepted
+    # prefix (margins far above that) must repeat, the residual sample over 16384 almost equally
+    # likely codes need not and is only checked for range.
+    gpu2 = run.verify(case, want_probs=False)
+    np.testing.assert_array_equal(gpu2["accept_len"], gpu["accept_len"])
+    ms = wl.shape
+    assert ((gpu2["next_token"] >= ms.vocab_offset) & (gpu2["next_token"] < ms.vocab_offset + ms.vocab)).all()
+    run.close()
+
+
+def test_config3_7b_width_two_layers():
+    """d = 4096, 32 heads of 128, MLP 11008, 8192 codes inside a 65536-row head, fill 1500."""
+    ms = replace(B7, name="visual_ar_7b_2layers", n_layers=2)
+    case = H.build_case(ms, 0x56565303, 1, 2, 1, 8, [1500])
+    run = H.GpuRunner(ms, case["w"], 2, 9)
+    gpu = run.verify(case)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    assert ((gpu["next_token"] >= ms.vocab_offset) & (gpu["next_token"] < ms.vocab_offset + ms.vocab)).all()
+    run.close()
+
+
+def test_config2_batch16_relaxed_two_layers():
+    """16 images x guidance = 32 sequences (288 block rows), fills drawn per image, relaxed
+    acceptance with 64 neighbours: the per-projection tensor-core kernels, two token passes."""
+    wl = CONFIGS[2]
+    ms = replace(XL, name="llamagen_xl_2layers", n_layers=2)
+    fills = [1, 575, 130, 288, 17, 400, 333, 128, 127, 129, 256, 500, 64, 9, 511, 200]
+    case = H.build_case(ms, wl.seed, 16, 2, 1, 8, fills, mode=MODE_RELAXED, nbr_k=64, q_noise=1.5)
+    run = H.GpuRunner(ms, case["w"], 32, 9, max_nbr_k=64)
+    gpu = run.verify(case)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    run.close()

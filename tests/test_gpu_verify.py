@@ -18,8 +18,20 @@ pytestmark = pytest.mark.gpu
 
 
 def _tols(ms):
+    """Probabilities: 2e-3 absolute at every depth.  Features (and what follows from them in
+    relative terms): 1e-2 of the row norm up to 3 layers; every sublayer injects fresh bf16
+    rounding of its GEMM inputs, which adds up like a random walk over depth, so the bound grows
+    with sqrt(layers / 3).  At 36 layers the three bf16 implementations in this library (the
+    whole-chain kernel, the per-projection tensor-core kernels, the plain generic kernels) measure
+    2.0-3.1 % against the fp64 oracle and 3-4 % against one another on the random-init network."""
     if ms.dtype == DTYPE_BF16:
-        return dict(p_abs=2e-3, p_rel=6e-2, h_rel=1e-2, int_margin=6e-2)
+        depth = max(1.0, ms.n_layers / 3.0) ** 0.5
+        h_rel = 1e-2 * depth
+        # A feature error of h_rel of the row norm (~sqrt(d)) becomes a guided-logit error of
+        # h_rel * sqrt(d) * 0.02 (weight std) * sqrt(2^2 + 1^2) (guidance 2.0); the largest of the
+        # ~1e5 logits of a call sits near 5 sigma, and a logit error is a relative probability error.
+        p_rel = max(6e-2 * depth, h_rel * ms.d_model ** 0.5 * 0.02 * 5.0 ** 0.5 * 5.0)
+        return dict(p_abs=2e-3, p_rel=p_rel, h_rel=h_rel, int_margin=p_rel)
     return dict(p_abs=1e-5, p_rel=2e-4, h_rel=1e-4, int_margin=1e-4)
 
 
@@ -30,10 +42,14 @@ def _check_end_to_end(case, gpu, ora):
     assert gpu["launches"] > 0
     assert H.rel_err_rows(gpu["hidden"], ora["hidden"]) < tol["h_rel"]
     dp = np.abs(gpu["target_probs"] - ora["target_probs"])
-    assert dp.max() < tol["p_abs"]
+    # 2e-3 absolute, except where a single probability is so large (the 7B-width head has logits
+    # of std > 1) that its relative bound allows more
+    assert (dp < np.maximum(tol["p_abs"], tol["p_rel"] * ora["target_probs"])).all()
     assert (dp / ora["target_probs"]).max() < tol["p_rel"]
     np.testing.assert_allclose(gpu["target_probs"].sum(-1), 1.0, atol=1e-4)
-    H.check_new_cache_rows(case, gpu, ora, tol["h_rel"])
+    # appended K/V are compared per (layer, head, slot) row of head_dim elements: in a deep network
+    # the error of such a short row scatters around the feature error, hence twice the bound there
+    H.check_new_cache_rows(case, gpu, ora, tol["h_rel"] * (2.0 if ms.n_layers > 3 else 1.0))
     # integer outputs against the oracle's own pipeline, classified by the oracle's margins
     k = case["n_draft_max"]
     real = 0
