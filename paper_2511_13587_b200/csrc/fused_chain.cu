@@ -169,16 +169,25 @@ __device__ __forceinline__ void rope8(const ChainParams& p, int tok, int e, floa
   }
 }
 
-// tcgen05.mma with an immediate accumulate flag
-__device__ __forceinline__ void mma_set(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+// The MMA warp runs its loop with all 32 lanes (so that descriptors and addresses stay warp-uniform
+// values) and one elected lane issues; the election is inside the asm block, the same lane every time.
+__device__ __forceinline__ void mma_elect(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred pe, pa;\n\t"
+      "elect.sync _|pe, 0xffffffff;\n\t"
+      "setp.ne.b32 pa, %4, 0;\n\t"
+      "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pa;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
 }
-__device__ __forceinline__ void mma_acc(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 1, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+__device__ __forceinline__ void commit_elect(uint64_t* bar) {
+  asm volatile(
+      "{\n\t.reg .pred pe;\n\t"
+      "elect.sync _|pe, 0xffffffff;\n\t"
+      "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(smem_u32(bar))
+      : "memory");
 }
 
 // Fast path of a wait: one poll, inline.
@@ -372,7 +381,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               if (round > 0 && !wait_bar(&empty[st], (round - 1) & 1, &s_abort, p.status)) { alive = false; break; }
               mbar_expect_tx(&full[st], kSlabBytes);
               tma_load_2d(ring + (size_t)st * kStageBytes, map + j, &full[st], kb * 64, tile * 128);
-              VVS_TRACE(0x100 | (ph << 4) | (s - lo));
+              VVS_TRACE(0x100 | (ph << 4) | ((s - lo) & 15));
               if (++st == NS) { st = 0; ++round; }
             }
             if (++kb == f.kbs) { kb = 0; ++tile; }
@@ -384,7 +393,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
     }
   } else if (warp == 1) {
     // =================================== MMA issuer ==================================================
-    if (lane == 0) {
+    {
       uint32_t st = 0, par = 0, ita = 0, iatt = 0;
       bool alive = true;
       const uint32_t idesc_gemm = idesc_bf16_f32(128, 32);
@@ -400,28 +409,30 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               const uint32_t apar = iatt & 1;
               if (!wait_bar(&att_kv_full, apar, &s_abort, p.status) ||
                   !wait_bar(&att_q_ready, apar, &s_abort, p.status)) { alive = false; break; }
+              __syncwarp();
               tc_fence_after();
-              VVS_TRACE(0x2A1);
+              if (lane == 0) VVS_TRACE(0x2F1);
               const uint32_t idesc_s = idesc_bf16_f32(128, (uint32_t)p.tq);
               for (int k16 = 0; k16 < p.hd / 16; ++k16) {
                 const uint32_t a = smem_u32(sK + (k16 >> 2) * kSlabBytes) + (k16 & 3) * 32;
                 const uint32_t b = smem_u32(sQ + (k16 >> 2) * q_chunk_bytes) + (k16 & 3) * 32;
-                mma_bf16(tmem_base + kColS, smem_desc_sw128(a), smem_desc_sw128(b), idesc_s, k16 > 0 ? 1u : 0u);
+                mma_elect(tmem_base + kColS, smem_desc_sw128(a), smem_desc_sw128(b), idesc_s, k16 > 0 ? 1u : 0u);
               }
-              mma_commit(&att_s_full);
-              VVS_TRACE(0x2A2);
+              commit_elect(&att_s_full);
+              if (lane == 0) VVS_TRACE(0x2F2);
               if (!wait_bar(&att_p_ready, apar, &s_abort, p.status)) { alive = false; break; }
+              __syncwarp();
               tc_fence_after();
-              VVS_TRACE(0x2A3);
+              if (lane == 0) VVS_TRACE(0x2F3);
               const uint32_t idesc_o = idesc_bf16_f32(128, (uint32_t)p.hd) | (1u << 16);  // B is MN-major
               for (int k16 = 0; k16 < 8; ++k16) {
                 const uint32_t a = smem_u32(sP + (k16 >> 2) * kSlabBytes) + (k16 & 3) * 32;
                 const uint32_t b = smem_u32(sV) + k16 * 2048;
-                mma_bf16(tmem_base + kColO, smem_desc_sw128(a), smem_desc_mn_sw128(b, kSlabBytes), idesc_o,
+                mma_elect(tmem_base + kColO, smem_desc_sw128(a), smem_desc_mn_sw128(b, kSlabBytes), idesc_o,
                          k16 > 0 ? 1u : 0u);
               }
-              mma_commit(&att_o_full);
-              VVS_TRACE(0x2A4);
+              commit_elect(&att_o_full);
+              if (lane == 0) VVS_TRACE(0x2F4);
             }
             if (!alive) break;
           }
@@ -434,7 +445,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
           for (int s = lo; s < hi; ++s) {
             const bool first = (s == lo) || (kb == 0);
             if (first) {
-              if (s != lo) mma_commit(&acc_full[slot]);
+              if (s != lo) commit_elect(&acc_full[slot]);
               slot = ita % kAccSlots;
               const uint32_t use = ita / kAccSlots;
               if (use > 0 && !wait_bar(&acc_empty[slot], (use - 1) & 1, &s_abort, p.status)) { alive = false; break; }
@@ -453,29 +464,30 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               st_b = st;
               if (++st == NS) { st = 0; par ^= 1; }
             }
+            __syncwarp();
             tc_fence_after();
-            VVS_TRACE(0x200 | (ph << 4) | (s - lo));
+            if (lane == 0) VVS_TRACE(0x200 | (ph << 4) | ((s - lo) & 15));
             const uint32_t acc = tmem_base + slot * 64;
-            if (first) mma_set(acc, a_desc, b_desc, idesc_gemm); else mma_acc(acc, a_desc, b_desc, idesc_gemm);
-            mma_acc(acc, a_desc + 2, b_desc + 2, idesc_gemm);
-            mma_acc(acc, a_desc + 4, b_desc + 4, idesc_gemm);
-            mma_acc(acc, a_desc + 6, b_desc + 6, idesc_gemm);
+            mma_elect(acc, a_desc, b_desc, idesc_gemm, first ? 0u : 1u);
+            mma_elect(acc, a_desc + 2, b_desc + 2, idesc_gemm, 1u);
+            mma_elect(acc, a_desc + 4, b_desc + 4, idesc_gemm, 1u);
+            mma_elect(acc, a_desc + 6, b_desc + 6, idesc_gemm, 1u);
             if (f.dual) {
               // the second weight slab multiplies the token slab of the FIRST stage: that stage is
               // released only after these have been issued as well
-              if (first) mma_set(acc + 32, a2_desc, b_desc, idesc_gemm); else mma_acc(acc + 32, a2_desc, b_desc, idesc_gemm);
-              mma_acc(acc + 32, a2_desc + 2, b_desc + 2, idesc_gemm);
-              mma_acc(acc + 32, a2_desc + 4, b_desc + 4, idesc_gemm);
-              mma_acc(acc + 32, a2_desc + 6, b_desc + 6, idesc_gemm);
-              mma_commit(&empty[st_a]);
-              mma_commit(&empty[st_b]);
+              mma_elect(acc + 32, a2_desc, b_desc, idesc_gemm, first ? 0u : 1u);
+              mma_elect(acc + 32, a2_desc + 2, b_desc + 2, idesc_gemm, 1u);
+              mma_elect(acc + 32, a2_desc + 4, b_desc + 4, idesc_gemm, 1u);
+              mma_elect(acc + 32, a2_desc + 6, b_desc + 6, idesc_gemm, 1u);
+              commit_elect(&empty[st_a]);
+              commit_elect(&empty[st_b]);
             } else {
-              mma_commit(&empty[st_a]);
+              commit_elect(&empty[st_a]);
             }
-            VVS_TRACE(0x280 | (ph << 4) | (s - lo));
+            if (lane == 0) VVS_TRACE(0x280 | (ph << 4) | ((s - lo) & 15));
             if (++kb == f.kbs) kb = 0;
           }
-          if (alive && hi > lo) mma_commit(&acc_full[slot]);
+          if (alive && hi > lo) commit_elect(&acc_full[slot]);
         }
       }
     }
@@ -587,7 +599,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
                 *reinterpret_cast<uint4*>(dst) = pack8(v);
               }
               fence_proxy_async();
-              if (tid_g == 0) VVS_TRACE(0x3A1);
+              if (tid_g == 0) VVS_TRACE(0x3F1);
               named_bar_sync(BAR_D, kGroup);
               if (tid_g == 0 && !s_abort) mbar_arrive(&att_q_ready);
             } else {
@@ -619,13 +631,13 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
                 }
               }
               fence_proxy_async();
-              if (tid_g == 0) VVS_TRACE(0x4A1);
+              if (tid_g == 0) VVS_TRACE(0x4F1);
               named_bar_sync(BAR_E, kGroup);
               if (tid_g == 0 && !s_abort) mbar_arrive(&att_q_ready);
               // scores: this thread owns key (quarter * 32 + lane) of the chunk
               wait_bar(&att_s_full, par, &s_abort, p.status);
               tc_fence_after();
-              if (tid_g == 0) VVS_TRACE(0x4A2);
+              if (tid_g == 0) VVS_TRACE(0x4F2);
               const int kl = quarter * 32 + lane;
               const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + kColS;
               {
@@ -679,13 +691,13 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               }
               fence_proxy_async();
               tc_fence_before();
-              if (tid_g == 0) VVS_TRACE(0x4A3);
+              if (tid_g == 0) VVS_TRACE(0x4F3);
               named_bar_sync(BAR_E, kGroup);
               if (tid_g == 0 && !s_abort) mbar_arrive(&att_p_ready);
             }
             wait_bar(&att_o_full, par, &s_abort, p.status);
             tc_fence_after();
-            if (tid_w == 0) VVS_TRACE(0x4A4);
+            if (tid_w == 0) VVS_TRACE(0x4F4);
             if (grp_e && quarter == 0) {                  // TMEM lanes 0..31 = query rows
               const size_t rh = (size_t)r * H + h;
               const size_t slot = (rh * p.n_chunks_max + c) * T + lane;
@@ -705,7 +717,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               }
             }
             tc_fence_before();
-            if (tid_w == 64) VVS_TRACE(0x4A5);
+            if (tid_w == 64) VVS_TRACE(0x4F5);
             named_bar_sync(BAR_W, kWorkers);
           }
           if (!grp_e && tid_g == 0 && l + 1 < L && (int)blockIdx.x < n_items) issue_kv(l + 1, blockIdx.x);
@@ -782,7 +794,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               }
             }
             fence_proxy_async();
-            if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | b0);
+            if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | (b0 & 15));
             named_bar_sync(BAR_W, kWorkers);
             if (tid_w < 2 && b0 + tid_w < n_units && !s_abort) mbar_arrive(&full[(it_slab + (uint32_t)(b0 + tid_w)) % NS]);
           }
@@ -814,7 +826,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               build_round<8, false>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, p.x, gsc,
                                     nullptr, p.ss + (2 * l + which) * 32);
             fence_proxy_async();
-            if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | b0);
+            if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | (b0 & 15));
             named_bar_sync(BAR_W, kWorkers);
             if (tid_w < nb && !s_abort) {
               const uint32_t it = it0 + (uint32_t)tid_w * per_unit;
