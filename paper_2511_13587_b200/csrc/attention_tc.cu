@@ -156,32 +156,47 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
     tc_fence_after();
     const int key = key0 + tid;
     const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
-    float s[32];
-    tmem_ld16(t_row, s);
-    if (p.tq > 16) tmem_ld16(t_row + 16, s + 16);
+    {
+      // scores of this key for all queries -> shared memory, transposed ([query][key], fp32; kept in
+      // rows of the P tiles that belong to no query)
+      float sc[32];
+      tmem_ld16(t_row, sc);
+      if (p.tq > 16) tmem_ld16(t_row + 16, sc + 16);
 #pragma unroll
-    for (int t = 0; t < 32; ++t) {
-      if (t < T) {
-        const bool valid = key <= fill + t;
-        s[t] = valid ? s[t] * p.scale : -CUDART_INF_F;
-        const float wm = warp_max_f(s[t]);
-        if (lane == 0) red_max[warp][t] = wm;
-      }
+      for (int t = 0; t < 32; ++t)
+        if (t < p.tq) reinterpret_cast<float*>(sP + (t >> 4) * kKVBytes + 4096)[(t & 15) * 128 + tid] = sc[t];
     }
     __syncthreads();
+    // one warp per query row: mask, max, exp, sum; lane owns keys 4*lane .. 4*lane+3
+#pragma unroll 1
+    for (int t = warp; t < T; t += 4) {
+      const float4 s4 = reinterpret_cast<const float4*>(sP + (t >> 4) * kKVBytes + 4096)[(t & 15) * 32 + lane];
+      float sv[4] = {s4.x, s4.y, s4.z, s4.w};
+      float mx = -CUDART_INF_F;
 #pragma unroll
-    for (int t = 0; t < 32; ++t) {
-      if (t < T) {
-        const float m = fmaxf(fmaxf(red_max[0][t], red_max[1][t]), fmaxf(red_max[2][t], red_max[3][t]));
-        const float e = (s[t] == -CUDART_INF_F) ? 0.f : expf(s[t] - m);
-        s[t] = e;
-        const float ws = warp_sum_f(e);
-        if (lane == 0) red_sum[warp][t] = ws;
-        // P[t, key] as bf16, K-major rows of 64 keys with the 128-byte swizzle
-        const uint32_t kk = (uint32_t)tid & 63u;
-        uint8_t* dst = sP + (tid >> 6) * kKVBytes + t * 128 + ((((kk >> 3) ^ ((uint32_t)t & 7u)) << 4) | ((kk & 7u) << 1));
-        *reinterpret_cast<__nv_bfloat16*>(dst) = __float2bfloat16_rn(e);
+      for (int j = 0; j < 4; ++j) {
+        sv[j] = (key0 + 4 * lane + j <= fill + t) ? sv[j] * p.scale : -CUDART_INF_F;
+        mx = fmaxf(mx, sv[j]);
       }
+      mx = warp_max_f(mx);
+      float sum = 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        sv[j] = (sv[j] == -CUDART_INF_F) ? 0.f : __expf(sv[j] - mx);
+        sum += sv[j];
+      }
+      sum = warp_sum_f(sum);
+      if (lane == 0) {
+        red_max[0][t] = mx;
+        red_sum[0][t] = sum;
+      }
+      // P[t, key] as bf16, K-major rows of 64 keys with the 128-byte swizzle
+      const int k4 = 4 * lane;
+      uint2 pk;
+      *reinterpret_cast<__nv_bfloat162*>(&pk.x) = __floats2bfloat162_rn(sv[0], sv[1]);
+      *reinterpret_cast<__nv_bfloat162*>(&pk.y) = __floats2bfloat162_rn(sv[2], sv[3]);
+      uint8_t* dst = sP + (k4 >> 6) * kKVBytes + t * 128 + (((((k4 & 63) >> 3) ^ (t & 7)) << 4) | ((k4 & 7) << 1));
+      *reinterpret_cast<uint2*>(dst) = pk;
     }
     // V rows of keys that no query may see: cleared, so unwritten cache slots cannot inject NaN
     if (!wait_bounded(&bar_v, 0)) atomicOr(p.status, VVS_DEV_TIMEOUT);
@@ -222,8 +237,8 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
       const uint32_t t_row = tmem_base + 32;
       float* po = p.part_o + ((rh * p.n_chunks_max + c) * T + lane) * HD;
       // chunk-wide max and sum of query `lane` (the four warps' reductions are still in place)
-      const float mine_max = fmaxf(fmaxf(red_max[0][lane], red_max[1][lane]), fmaxf(red_max[2][lane], red_max[3][lane]));
-      const float mine_sum = red_sum[0][lane] + red_sum[1][lane] + red_sum[2][lane] + red_sum[3][lane];
+      const float mine_max = red_max[0][lane];
+      const float mine_sum = red_sum[0][lane];
       for (int e0 = 0; e0 < HD; e0 += 16) {
         float o[16];
         tmem_ld16(t_row + e0, o);

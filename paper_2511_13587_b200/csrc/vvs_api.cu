@@ -262,6 +262,8 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   const GemmTcPlan p_qkv = plan_gemm_tc(M, 3 * d, d, false, true, ctx->n_sms);
   const GemmTcPlan p_o = plan_gemm_tc(M, d, d, false, true, ctx->n_sms);
   const GemmTcPlan p_gu = plan_gemm_tc(M, ff, d, true, true, ctx->n_sms);
+  const GemmTcPlan p_g1 = plan_gemm_tc(M, ff, d, false, true, ctx->n_sms);   // gate and up as two launches
+  const bool wide = M > 64;
   const GemmTcPlan p_down = plan_gemm_tc(M, d, ff, false, true, ctx->n_sms);
   CUtensorMap tm_xn, tm_attn, tm_act, tm_q, tm_k, tm_v;
   const uint64_t kv_total_rows = (uint64_t)md.n_layers * a->kv_rows * md.n_heads * md.s_max;
@@ -313,7 +315,16 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     const Layer& L = ctx->layers[l];
     const LayerMaps& W = ctx->layer_maps[l];
     VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm1), xn, M, d, md.rms_eps, s));
-    {
+    if (wide) {
+      // many tokens: a per-thread epilogue over hundreds of tokens is slower than a plain split-K
+      // sum into fp32 followed by one thread per element for rotation, rounding and cache append
+      if (cudaMemsetAsync(ws.qkv, 0, (size_t)M * 3 * d * sizeof(float), s) != cudaSuccess) return VVS_ERR_CUDA;
+      GemmTcArgs g = base;
+      g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.out = ws.qkv; g.ldo = 3 * d;
+      VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_qkv, g, s));
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_append<T>(ws.qkv, ws.rope_inv_freq, q, kv_k, kv_v, a->cache_len, md,
+                                                       l, a->kv_rows, R, Tn, ws.status, s));
+    } else {
       GemmTcArgs g = base;
       g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.ld_scratch = 3 * d; g.layer = l;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_QKV, p_qkv, g, s));
@@ -328,7 +339,15 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_o, g, s));
     }
     VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm2), xn, M, d, md.rms_eps, s));
-    if (rc == VVS_OK) {
+    if (rc == VVS_OK && wide) {
+      if (cudaMemsetAsync(ws.gu, 0, (size_t)M * 2 * ff * sizeof(float), s) != cudaSuccess) return VVS_ERR_CUDA;
+      GemmTcArgs g = base;
+      g.n = ff; g.k = d; g.tm_a = &W.w_gate; g.tm_b = &tm_xn; g.out = ws.gu; g.ldo = 2 * ff;
+      VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_g1, g, s));
+      g.tm_a = &W.w_up; g.out = ws.gu + ff;
+      if (rc == VVS_OK) VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_g1, g, s));
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_silu_mul<T>(ws.gu, act, M, ff, s));
+    } else if (rc == VVS_OK) {
       GemmTcArgs g = base;
       g.n = ff; g.k = d; g.tm_a = &W.w_gate; g.tm_a2 = &W.w_up; g.tm_b = &tm_xn; g.ld_scratch = 2 * ff;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_SWIGLU, p_gu, g, s));
