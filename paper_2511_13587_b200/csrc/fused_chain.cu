@@ -796,6 +796,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             fence_proxy_async();
             if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | (b0 & 15));
             named_bar_sync(BAR_W, kWorkers);
+            if (tid_w == 0) VVS_TRACE(0x380 | (ph << 4) | (b0 & 15));
             if (tid_w < 2 && b0 + tid_w < n_units && !s_abort) mbar_arrive(&full[(it_slab + (uint32_t)(b0 + tid_w)) % NS]);
           }
         } else {
@@ -828,6 +829,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             fence_proxy_async();
             if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | (b0 & 15));
             named_bar_sync(BAR_W, kWorkers);
+            if (tid_w == 0) VVS_TRACE(0x380 | (ph << 4) | (b0 & 15));
             if (tid_w < nb && !s_abort) {
               const uint32_t it = it0 + (uint32_t)tid_w * per_unit;
               mbar_arrive(&full[it % NS]);
