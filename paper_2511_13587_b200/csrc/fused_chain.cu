@@ -54,6 +54,8 @@ constexpr int kMaxSeq = 32;
 constexpr int kMaxLayers = 64;
 constexpr uint32_t kColS = 256, kColO = 320, kTmemCols = 512;
 constexpr uint32_t kGridSpinLimit = 1u << 21;
+constexpr uint32_t kParkNs = 4000;          // a parked wait answers after at most this long
+constexpr uint32_t kParkedPolls = 1u << 19;  // ~2 s before a wait gives up
 enum { BAR_W = 1, BAR_E = 2, BAR_D = 3 };
 enum { PH_QKV = 0, PH_O = 1, PH_GU = 2, PH_DOWN = 3 };
 
@@ -112,9 +114,9 @@ __device__ __forceinline__ void unit_range(const Phase& f, int layer, int ph, in
 // Bounded wait; falls through at once when the CTA is in abort mode.
 __device__ __noinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* s_abort, int32_t* status) {
   if (*s_abort) return false;
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && *s_abort) return false;
+  for (uint32_t i = 0; i < kParkedPolls; ++i) {
+    if (mbar_try_wait_parked(bar, parity, kParkNs)) return true;
+    if ((i & 15u) == 15u && *s_abort) return false;
   }
   *s_abort = 1;
   atomicOr(status, VVS_DEV_TIMEOUT);
