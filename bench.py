@@ -386,17 +386,86 @@ def run_reference(args) -> None:
     print(json.dumps(line))
 
 
+# ---------------------------------------------------------------------------------------------
+# configs[4]: the acceptance epilogue in isolation (LM head + guidance + softmax + decisions)
+
+
+def run_epilogue_sweep(args) -> None:
+    """A few points of the configs[4] sweep through vvs_epilogue, inputs drawn on the device.
+    One JSON line; every point carries its time, the LM-head TFLOP/s (2 M d V over the whole call,
+    which runs the LM head, the decision kernels and the one-row-per-image second pass) and the
+    bytes-per-second of the codebook stream, each as a fraction of the measured peak."""
+    import torch
+    from paper_2511_13587_b200 import binding as vb
+    from vvs_synth.configs import ModelShape, MODE_STRICT
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    pk = peaks()
+    points = []
+    for d, v, b, k, c, mode, nbr_k in ((1280, 16384, 1, 8, 2, MODE_STRICT, 1), (1280, 16384, 16, 8, 2, MODE_RELAXED, 64),
+                                       (1280, 16384, 32, 8, 2, MODE_STRICT, 1), (4096, 16384, 32, 8, 2, MODE_STRICT, 1),
+                                       (4096, 65536, 8, 8, 2, MODE_STRICT, 1), (4096, 65536, 64, 16, 2, MODE_STRICT, 1),
+                                       (4096, 65536, 64, 16, 1, MODE_STRICT, 1), (1280, 4096, 64, 16, 2, MODE_RELAXED, 64)):
+        ms = ModelShape("epilogue", 0, d, 0, 0, 0, v)
+        rows = k + 1
+        ctx = vb.vvs_create(vb.make_desc(ms, b * c, rows, max(1, nbr_k)))
+        g = torch.Generator(device="cuda").manual_seed(0x56565304)
+        w_lm = (torch.randn((v, d), generator=g, device="cuda") * (2.0 / d ** 0.5)).to(torch.bfloat16)
+        vb.vvs_bind_weights(ctx, {"w_lm": w_lm, "layers": []})
+        if mode == MODE_RELAXED:
+            rp, col = gen.neighbour_csr(gen.make_codebook(0x56565304, v), nbr_k)
+            rp_d, col_d = torch.from_numpy(rp).cuda(), torch.from_numpy(col).cuda()
+            vb.vvs_bind_neighbors(ctx, rp_d, col_d)
+        hidden = torch.randn((b * c, rows, d), generator=g, device="cuda").to(torch.bfloat16)
+        q = torch.softmax(torch.randn((b, k, v), generator=g, device="cuda"), -1).contiguous()
+        drafts = torch.randint(0, v, (b, k), generator=g, device="cuda", dtype=torch.int32)
+        u = torch.rand((b, k + 1), generator=g, device="cuda").clamp_(1e-6, 1 - 1e-6)
+        nd = torch.full((b,), k, dtype=torch.int32, device="cuda")
+        o = dict(accept_len=torch.zeros(b, dtype=torch.int32, device="cuda"),
+                 next_token=torch.zeros(b, dtype=torch.int32, device="cuda"))
+
+        def call():
+            vb.vvs_epilogue(ctx, hidden_in=hidden, n_rows_per_seq=rows, first_row=0, drafts=drafts, n_images=b,
+                            n_cfg=c, n_draft_max=k, n_draft=nd, draft_probs=q, uniforms=u, cfg_scale=2.0,
+                            temperature=1.0, mode=mode, nbr_k=nbr_k, delta=float("inf"), **o)
+
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        ms_call = e0.elapsed_time(e1) / args.steps
+        m_rows = b * c * rows
+        flops, byts = 2.0 * m_rows * d * v, d * v * 2 + m_rows * d * 2 + b * v * 4
+        points.append({"d": d, "V": v, "B": b, "K": k, "C": c, "M": m_rows, "relaxed_k": nbr_k if mode else 0,
+                       "us": ms_call * 1e3, "tflops": flops / ms_call / 1e9,
+                       "frac_tensor": flops / ms_call / 1e9 / pk["bf16_tflops"],
+                       "gbs": byts / ms_call / 1e6, "frac_hbm": byts / ms_call / 1e6 / pk["hbm_gbs"],
+                       "device_status": vb.vvs_device_status(ctx)})
+        vb.vvs_destroy(ctx)
+    print(json.dumps({"metric": "acceptance epilogue in isolation (configs[4] sweep points)", "unit": "us per call",
+                      "steps": args.steps, "dtype": "bf16", "data": "synthetic", "peak_source": pk["source"],
+                      "points": points}))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3])
-    ap.add_argument("--cpu-steps", type=int, default=2)
+    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3, 4])
+    ap.add_argument("--cpu-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload == 4:
+        run_epilogue_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
