@@ -76,6 +76,12 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
   const int c = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
   const int T = p.t_len;
 
+  {
+    // chunks beyond this sequence's keys have nothing to do: leave before any set-up (the grid is
+    // sized for the longest possible sequence)
+    const int fill0 = p.cache_len[r];
+    if (fill0 >= 0 && fill0 + T <= p.s_max && c * kChunkKeys >= fill0 + T) return;
+  }
   if (tid == 0) {
     mbar_init(&bar_kq, 1);
     mbar_init(&bar_v, 1);

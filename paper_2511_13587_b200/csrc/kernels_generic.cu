@@ -289,19 +289,24 @@ void launch_attention(const T* q, const T* kv_k, const T* kv_v, const int32_t* c
 }
 
 // ---------------------------------------------------------------------------------------------
+// act[m, j] = silu(gate[m, j]) * up[m, j]; grid (column chunks of 1024, rows), 4 columns per thread
 template <typename T>
 __global__ void silu_mul_kernel(const float* __restrict__ gu, T* __restrict__ act, int ff) {
-  const float* row = gu + (size_t)blockIdx.x * 2 * ff;
-  T* o = act + (size_t)blockIdx.x * ff;
-  for (int j = threadIdx.x; j < ff; j += blockDim.x) {
-    float g = row[j];
-    o[j] = from_f<T>(g / (1.f + expf(-g)) * row[ff + j]);
-  }
+  const float* row = gu + (size_t)blockIdx.y * 2 * ff;
+  T* o = act + (size_t)blockIdx.y * ff;
+  const int j = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (j >= ff) return;                       // ff is a multiple of 8
+  const float4 g = *reinterpret_cast<const float4*>(row + j);
+  const float4 u = *reinterpret_cast<const float4*>(row + ff + j);
+  o[j] = from_f<T>(g.x / (1.f + expf(-g.x)) * u.x);
+  o[j + 1] = from_f<T>(g.y / (1.f + expf(-g.y)) * u.y);
+  o[j + 2] = from_f<T>(g.z / (1.f + expf(-g.z)) * u.z);
+  o[j + 3] = from_f<T>(g.w / (1.f + expf(-g.w)) * u.w);
 }
 
 template <typename T>
 void launch_silu_mul(const float* gu, T* act, int m, int ff, cudaStream_t s) {
-  silu_mul_kernel<T><<<m, 256, 0, s>>>(gu, act, ff);
+  silu_mul_kernel<T><<<dim3((ff + 1023) / 1024, m), 256, 0, s>>>(gu, act, ff);
 }
 
 // ---------------------------------------------------------------------------------------------
