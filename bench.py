@@ -39,6 +39,26 @@ def metric_name(wl) -> str:
     return f"verified draft tokens/sec ({shape}-shaped verify step)"
 
 
+def replica_seed(seed: int, rank: int) -> int:
+    """Replicas draw their own inputs: rank r of a multi-GPU run uses its own seed."""
+    return seed + 1000 * rank
+
+
+def max_over_ranks(values, world: int, device="cpu"):
+    """Element-wise maximum of `values` (floats) over all ranks; the identity for one rank."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_value(world: int, drafts_per_step: float, steps: int, ms_total: float) -> float:
+    """Whole-job throughput: every replica verifies its own drafts in the (max over ranks) time."""
+    return world * drafts_per_step * steps / (ms_total * 1e-3)
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -142,7 +162,7 @@ def run_ours(args) -> None:
     b, cfg, k, f = wl.n_images, wl.n_cfg, wl.n_draft_max, wl.n_forced
     r, t_len = b * cfg, wl.block_len
     relaxed = wl.mode == MODE_RELAXED
-    seed = wl.seed + 1000 * rank                                  # replicas draw their own inputs
+    seed = replica_seed(wl.seed, rank)
 
     def dev(a):
         a = np.ascontiguousarray(a)
@@ -273,10 +293,7 @@ def run_ours(args) -> None:
     vb.vvs_profile_enable(ctx, False)
 
     # ---- reduce over ranks ----------------------------------------------------------------------
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = t.tolist()
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -300,7 +317,7 @@ def run_ours(args) -> None:
     ms_step = ms_total / args.steps
     line = {
         "metric": metric_name(wl),
-        "value": world * drafts_per_step * args.steps / (ms_total * 1e-3),
+        "value": aggregate_value(world, drafts_per_step, args.steps, ms_total),
         "unit": "drafts/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_step, "verify_latency_us": ms_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -320,7 +337,7 @@ def run_ours(args) -> None:
                      "traffic": NCU_TRAFFIC.get(args.workload), "launches_per_step": dom_launches,
                      "class_ms_per_step": {"gemm": cls_ms[0] / n_prof, "attention": cls_ms[1] / n_prof,
                                            "other": cls_ms[2] / n_prof, "chain": cls_ms[3] / n_prof}},
-        "e2e": {"value": world * drafts_per_step * args.steps / (ms_e2e * 1e-3), "unit": "drafts/s",
+        "e2e": {"value": aggregate_value(world, drafts_per_step, args.steps, ms_e2e), "unit": "drafts/s",
                 "ms_per_step": ms_e2e / args.steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": gpu_launches, "device_status": status, "clocks": clocks.summary(),
     }
