@@ -34,6 +34,8 @@
 #ifndef VVS_TRACE
 #define VVS_TRACE_DECL
 #define VVS_TRACE(tag) ((void)0)
+#define VVS_TRACE_MMA(tag) ((void)0)   // inside the MMA warp's layer loop (layer index `l` in scope)
+#define VVS_TRACE_END ((void)0)
 #endif
 
 namespace vvs {
@@ -413,7 +415,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
                   !wait_bar(&att_q_ready, apar, &s_abort, p.status)) { alive = false; break; }
               __syncwarp();
               tc_fence_after();
-              if (lane == 0) VVS_TRACE(0x2F1);
+              VVS_TRACE_MMA(0x2F1);
               const uint32_t idesc_s = idesc_bf16_f32(128, (uint32_t)p.tq);
               for (int k16 = 0; k16 < p.hd / 16; ++k16) {
                 const uint32_t a = smem_u32(sK + (k16 >> 2) * kSlabBytes) + (k16 & 3) * 32;
@@ -421,11 +423,11 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
                 mma_elect(tmem_base + kColS, smem_desc_sw128(a), smem_desc_sw128(b), idesc_s, k16 > 0 ? 1u : 0u);
               }
               commit_elect(&att_s_full);
-              if (lane == 0) VVS_TRACE(0x2F2);
+              VVS_TRACE_MMA(0x2F2);
               if (!wait_bar(&att_p_ready, apar, &s_abort, p.status)) { alive = false; break; }
               __syncwarp();
               tc_fence_after();
-              if (lane == 0) VVS_TRACE(0x2F3);
+              VVS_TRACE_MMA(0x2F3);
               const uint32_t idesc_o = idesc_bf16_f32(128, (uint32_t)p.hd) | (1u << 16);  // B is MN-major
               for (int k16 = 0; k16 < 8; ++k16) {
                 const uint32_t a = smem_u32(sP + (k16 >> 2) * kSlabBytes) + (k16 & 3) * 32;
@@ -434,7 +436,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
                          k16 > 0 ? 1u : 0u);
               }
               commit_elect(&att_o_full);
-              if (lane == 0) VVS_TRACE(0x2F4);
+              VVS_TRACE_MMA(0x2F4);
             }
             if (!alive) break;
           }
@@ -468,7 +470,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             }
             __syncwarp();
             tc_fence_after();
-            if (lane == 0) VVS_TRACE(0x200 | (ph << 4) | ((s - lo) & 15));
+            VVS_TRACE_MMA(0x200 | (ph << 4) | ((s - lo) & 15));
             const uint32_t acc = tmem_base + slot * 64;
             mma_elect(acc, a_desc, b_desc, idesc_gemm, first ? 0u : 1u);
             mma_elect(acc, a_desc + 2, b_desc + 2, idesc_gemm, 1u);
@@ -486,7 +488,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             } else {
               commit_elect(&empty[st_a]);
             }
-            if (lane == 0) VVS_TRACE(0x280 | (ph << 4) | ((s - lo) & 15));
+            VVS_TRACE_MMA(0x280 | (ph << 4) | ((s - lo) & 15));
             if (++kb == f.kbs) kb = 0;
           }
           if (alive && hi > lo) commit_elect(&acc_full[slot]);
@@ -915,6 +917,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
   }
 
   // ---- teardown ---------------------------------------------------------------------------------
+  VVS_TRACE_END;
   __syncwarp();
   tc_fence_before();
   __syncthreads();
