@@ -377,3 +377,55 @@ class FeatureCache:
                     out[r, j] = self.feat[r, pos % self.cap]
                     out_pos[r, j] = pos
         return out, out_pos
+
+
+# ---------------------------------------------------------------------------------------
+# Dynamic verification skipping (Sec. 4.4 "Fine-grained Skipped Step Scheduling", Eq. 2, Alg. 1)
+#
+# What the paper fixes: skip only if the last step was verified; the candidate paths are
+# down-sampled with stride 2; S_bar = sum_l w_l S^(l), w_l = alpha^l / sum_k alpha^k, S^(l) the
+# cosine similarity of the latent codebook embeddings of the tokens at depth l; skip iff
+# S_bar >= T_sim.  Readings where it is silent (**parity unpinned** by the paper): S^(l) is the
+# mean cosine over all unordered pairs of the kept paths; the depth L is the shortest kept path
+# (deeper tokens are ignored); an embedding of norm 0 has cosine 0 with everything; fewer than
+# two kept paths, or depth 0, give S_bar = 1 resp. 0.
+
+
+def downsample_paths(n_paths: int, stride: int) -> list:
+    """Alg. 1, Downsample(C, stride): every stride-th candidate path, starting with the first."""
+    return list(range(0, n_paths, stride))
+
+
+def path_similarity(paths: np.ndarray, path_len: np.ndarray, codebook: np.ndarray, alpha: float,
+                    stride: int = 2) -> float:
+    """Eq. 2 on the down-sampled paths.  paths int [N, Lmax] codebook indices, path_len int [N],
+    codebook float [V, dim] (latent embeddings E)."""
+    keep = downsample_paths(len(paths), stride)
+    depth = int(min(path_len[i] for i in keep)) if keep else 0
+    if depth <= 0:
+        return 0.0
+    if len(keep) < 2:
+        return 1.0
+    e = np.asarray(codebook, dtype=np.float64)
+    w = np.array([alpha ** l for l in range(depth)], dtype=np.float64)
+    w = w / w.sum()
+    s_bar = 0.0
+    for l in range(depth):
+        total, pairs = 0.0, 0
+        for a in range(len(keep)):
+            for b in range(a + 1, len(keep)):
+                x, y = e[paths[keep[a], l]], e[paths[keep[b], l]]
+                nx, ny = np.sqrt(np.dot(x, x)), np.sqrt(np.dot(y, y))
+                total += np.dot(x, y) / (nx * ny) if nx > 0.0 and ny > 0.0 else 0.0
+                pairs += 1
+        s_bar += w[l] * (total / pairs)
+    return float(s_bar)
+
+
+def skip_decision(paths, path_len, codebook, alpha: float, threshold: float, last_verified: bool,
+                  stride: int = 2):
+    """Alg. 1: (bypass verification?, S_bar).  Never two skipped steps in a row."""
+    if not last_verified:
+        return False, 0.0
+    s_bar = path_similarity(np.asarray(paths), np.asarray(path_len), codebook, alpha, stride)
+    return bool(s_bar >= threshold), s_bar
