@@ -465,7 +465,30 @@ def run_epilogue_sweep(args) -> None:
                        "gbs": byts / ms_call / 1e6, "frac_hbm": byts / ms_call / 1e6 / pk["hbm_gbs"],
                        "device_status": vb.vvs_device_status(ctx)})
         vb.vvs_destroy(ctx)
+    # the dynamic skip decision (Alg. 1 / Eq. 2): 16 images, 24 candidate paths of depth 5 each,
+    # the 8-dim latent codebook of 16384 codes; latency-bound (one CTA per image, a few hundred
+    # dependent-load-limited cosine terms), reported as time per call
+    ms = ModelShape("skip", 0, 64, 0, 0, 0, 128)
+    ctx = vb.vvs_create(vb.make_desc(ms, 1, 1, 1))
+    g = torch.Generator(device="cuda").manual_seed(7)
+    cb = torch.randn((16384, 8), generator=g, device="cuda")
+    paths = torch.randint(0, 16384, (16, 24, 5), generator=g, device="cuda", dtype=torch.int32)
+    dec = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    sim = torch.zeros(16, dtype=torch.float32, device="cuda")
+    for _ in range(3):
+        vb.vvs_skip_decide(ctx, paths, None, cb, None, 2, 0.8, 0.65, dec, sim)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(100):
+        vb.vvs_skip_decide(ctx, paths, None, cb, None, 2, 0.8, 0.65, dec, sim)
+    e1.record()
+    torch.cuda.synchronize()
+    skip_us = e0.elapsed_time(e1) * 10.0
+    vb.vvs_destroy(ctx)
     print(json.dumps({"metric": "acceptance epilogue in isolation (configs[4] sweep points)", "unit": "us per call",
+                      "skip_decide": {"images": 16, "paths": 24, "depth": 5, "codebook": [16384, 8], "stride": 2,
+                                      "us_per_call": skip_us, "bound": "latency (launch + one chain of L2 loads)"},
                       "steps": args.steps, "dtype": "bf16", "data": "synthetic", "peak_source": pk["source"],
                       "points": points}))
 

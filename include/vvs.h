@@ -276,6 +276,27 @@ int vvs_feature_cache_fetch(vvs_ctx* ctx, const vvs_fcache* fc, const uint8_t* s
                             int32_t n_images, const int32_t* gamma, int32_t gamma_max,
                             int32_t staleness, void* out, int32_t* out_pos, void* stream);
 
+/* Dynamic verification skipping (Sec. 4.4 "Fine-grained Skipped Step Scheduling", Eq. 2,
+ * Algorithm 1): for every image, decide whether the next step may bypass target verification.
+ *   paths          device int32 [n_images, n_paths, max_len] candidate token paths of the draft
+ *                  tree as codebook indices (0 .. vocab-1); path i of an image has path_len[i] tokens
+ *   path_len       device int32 [n_images, n_paths], or NULL = every path has max_len tokens
+ *   codebook       device float32 [vocab, dim] latent embeddings E of the VQ codebook
+ *   last_verified  device uint8 [n_images] (V_last), or NULL = every image's last step was verified
+ * Alg. 1: an image whose last step was not verified never skips (decision 0, similarity 0).
+ * Otherwise the paths are down-sampled (every stride-th path, the paper uses 2), and
+ * S_bar = sum_l w_l S^(l), w_l = alpha^l / sum_k alpha^k (Eq. 2), is compared with the threshold:
+ * decision[b] = 1 (skip) iff S_bar >= threshold; similarity[b] = S_bar.  Where the paper is silent:
+ * S^(l) is the mean cosine similarity over all unordered pairs of kept paths of the embeddings of
+ * their tokens at depth l; the depth is the shortest kept path; a zero embedding has cosine 0; a
+ * single kept path gives S_bar = 1, depth 0 gives 0.  Limits (VVS_ERR_SHAPE beyond): 64 kept
+ * paths, max_len 16.  A token outside the codebook sets VVS_DEV_BAD_TOKEN and counts as cosine 0.
+ * Sums are taken in float64 in a fixed order: the same inputs give the same bits. */
+int vvs_skip_decide(vvs_ctx* ctx, const int32_t* paths, const int32_t* path_len, int32_t n_images,
+                    int32_t n_paths, int32_t max_len, const float* codebook, int32_t vocab, int32_t dim,
+                    const uint8_t* last_verified, int32_t stride, float alpha, float threshold,
+                    uint8_t* decision, float* similarity, void* stream);
+
 /* Synchronise `stream`, copy the device status word to *out_bits (VVS_DEV_* bits) and clear
  * it.  Returns VVS_ERR_DEVICE_TIMEOUT / VVS_ERR_DEVICE_BOUNDS if such a bit was set. */
 int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits);

@@ -35,6 +35,11 @@ is silent or garbled:
   block row, addressed by (row, absolute position) in a ring of `cap` slots; fetch(gamma, s)
   returns positions newest-s-gamma+1 .. newest-s.  **parity unpinned** for the choice of
   post-norm features and ring addressing; the index arithmetic itself is pinned.
+* dynamic skip decision (Sec. 4.4, Eq. 2, Alg. 1): S^(l) = mean cosine over all unordered pairs
+  of the paths kept by the stride-2 down-sampling, depth = shortest kept path, zero embedding =
+  cosine 0.  **parity unpinned** for the pair-mean and the depth rule (the paper says only
+  "cosine similarity of token representations at each position"); the depth weights, the
+  no-two-skips guard, the threshold rule and the cosine itself are pinned.
 * decisions are taken on the float32 target probabilities the step emits: ratios, pooled
   masses and the sampling CDF accumulate in float64 in ascending / distance order.
 """

@@ -81,6 +81,9 @@ lib.vvs_feature_cache_reset.argtypes = [_P, C.POINTER(vvs_fcache), _P]
 lib.vvs_feature_cache_store.argtypes = [_P, C.POINTER(vvs_fcache), _P, C.c_int32, _P, _P, _P]
 lib.vvs_feature_cache_fetch.argtypes = [_P, C.POINTER(vvs_fcache), _P, C.c_int32, _P, C.c_int32,
                                         C.c_int32, _P, _P, _P]
+lib.vvs_skip_decide.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_int32, C.c_int32, _P,
+                                C.c_int32, C.c_float, C.c_float, _P, _P, _P]
+lib.vvs_skip_decide.restype = C.c_int
 lib.vvs_device_status.argtypes = [_P, _P, C.POINTER(C.c_int32)]
 lib.vvs_last_launch_count.argtypes = [_P]
 lib.vvs_profile_enable.argtypes = [_P, C.c_int]
@@ -261,6 +264,18 @@ def vvs_feature_cache_fetch(ctx: int, fc: vvs_fcache, skip_mask, n_images, gamma
     _check(lib.vvs_feature_cache_fetch(ctx, C.byref(fc), _ptr(skip_mask), int(n_images), _ptr(gamma),
                                        int(gamma_max), int(staleness), _ptr(out), _ptr(out_pos),
                                        _stream(stream)), "vvs_feature_cache_fetch")
+
+
+def vvs_skip_decide(ctx: int, paths, path_len, codebook, last_verified, stride: int, alpha: float,
+                    threshold: float, decision, similarity, stream=None) -> None:
+    """Alg. 1 / Eq. 2 of the paper: paths int32 [B, N, L], path_len int32 [B, N] or None,
+    codebook float32 [V, dim], last_verified uint8 [B] or None -> decision uint8 [B], similarity
+    float32 [B]."""
+    b, n, l = paths.shape
+    v, dim = codebook.shape
+    _check(lib.vvs_skip_decide(ctx, _ptr(paths), _ptr(path_len), int(b), int(n), int(l), _ptr(codebook), int(v),
+                               int(dim), _ptr(last_verified), int(stride), float(alpha), float(threshold),
+                               _ptr(decision), _ptr(similarity), _stream(stream)), "vvs_skip_decide")
 
 
 def vvs_device_status(ctx: int, stream=None, raise_on_error: bool = False) -> int:

@@ -717,6 +717,18 @@ int vvs_feature_cache_fetch(vvs_ctx* ctx, const vvs_fcache* fc, const uint8_t* s
   return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
 }
 
+int vvs_skip_decide(vvs_ctx* ctx, const int32_t* paths, const int32_t* path_len, int32_t n_images,
+                    int32_t n_paths, int32_t max_len, const float* codebook, int32_t vocab, int32_t dim,
+                    const uint8_t* last_verified, int32_t stride, float alpha, float threshold,
+                    uint8_t* decision, float* similarity, void* stream) {
+  if (!ctx || !paths || !codebook || !decision || !similarity) return VVS_ERR_INVALID_ARG;
+  if (n_images < 1 || n_paths < 1 || max_len < 1 || vocab < 1 || dim < 1 || stride < 1) return VVS_ERR_SHAPE;
+  if (!(alpha > 0.f) || !std::isfinite(alpha) || std::isnan(threshold)) return VVS_ERR_INVALID_ARG;
+  return launch_skip_decide(paths, path_len, codebook, last_verified, n_images, n_paths, max_len, vocab, dim,
+                            stride, alpha, threshold, decision, similarity, ctx->ws.status,
+                            static_cast<cudaStream_t>(stream));
+}
+
 int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits) {
   if (!ctx || !out_bits) return VVS_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -265,6 +265,12 @@ void launch_select_p_row(const Workspace& ws, int n_images, int v, cudaStream_t 
 void launch_residual_mass(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_sample(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 
+// ---- dynamic skip decision, kernels_skip.cu -----------------------------------------------------
+int launch_skip_decide(const int32_t* paths, const int32_t* path_len, const float* codebook,
+                       const uint8_t* last_verified, int n_images, int n_paths, int max_len, int vocab, int dim,
+                       int stride, float alpha, float threshold, uint8_t* decision, float* sim, int32_t* status,
+                       cudaStream_t s);
+
 // ---- feature cache, kernels_fcache.cu ---------------------------------------------------------
 void launch_fcache_reset(const vvs_fcache& fc, cudaStream_t s);
 void launch_fcache_store(const vvs_fcache& fc, const void* hidden, int rows_per_seq, int d,
