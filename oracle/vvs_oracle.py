@@ -434,3 +434,19 @@ def skip_decision(paths, path_len, codebook, alpha: float, threshold: float, las
         return False, 0.0
     s_bar = path_similarity(np.asarray(paths), np.asarray(path_len), codebook, alpha, stride)
     return bool(s_bar >= threshold), s_bar
+
+
+# ---------------------------------------------------------------------------------------
+# Unverified token selection with truncation (Sec. 4.2, Eq. 3; Alg. 2 "UniformSample")
+#
+# The paper fixes: a verification-free step draws one candidate path uniformly at random and keeps
+# its first gamma = min(L_s, floor(L_bar)) tokens, L_s the length of the drawn path, L_bar the mean
+# length over all paths of the pruned tree.  Reading: path index = floor(u * N) for u in (0, 1).
+
+
+def select_unverified(paths: np.ndarray, path_len: np.ndarray, u: float):
+    """Returns (path index, gamma, the gamma kept tokens)."""
+    n = len(paths)
+    idx = min(n - 1, int(np.floor(float(u) * n)))
+    gamma = min(int(path_len[idx]), int(np.floor(np.sum(path_len, dtype=np.int64) / n)))
+    return idx, gamma, np.asarray(paths[idx][:gamma])

@@ -70,3 +70,20 @@ def test_guard_threshold_and_degenerate_inputs():
     cb0 = cb.copy(); cb0[1] = 0.0                                                          # zero embedding: cosine 0
     assert abs(O.path_similarity(paths, np.full(3, 2), cb0, 1.0) - 0.5) < 1e-15
     assert O.downsample_paths(7, 2) == [0, 2, 4, 6] and O.downsample_paths(4, 3) == [0, 3]
+
+
+def test_uniform_path_selection_and_truncation():
+    """Sec. 4.2 / Eq. 3: every path is drawn on an interval of width 1/N; gamma = min(L_s, floor(mean))."""
+    paths = np.arange(5 * 6).reshape(5, 6)
+    lens = np.array([6, 2, 5, 3, 4])                        # mean 4.0
+    hits = np.zeros(5, int)
+    for k in range(1000):
+        i, g, toks = O.select_unverified(paths, lens, (k + 0.5) / 1000)
+        hits[i] += 1
+        assert g == min(lens[i], 4) and list(toks) == list(paths[i][:g])
+    assert (hits == 200).all()
+    assert O.select_unverified(paths, lens, 0.999999)[0] == 4 and O.select_unverified(paths, lens, 1e-9)[0] == 0
+    # the floor: lengths 3, 4 -> mean 3.5 -> at most 3 tokens even from the longer path
+    assert O.select_unverified(paths[:2], np.array([3, 4]), 0.75)[1] == 3
+    assert O.select_unverified(paths[:2], np.array([1, 6]), 0.75)[1] == 3     # mean 3.5, L_s = 6
+    assert O.select_unverified(paths[:2], np.array([1, 6]), 0.25)[1] == 1     # L_s = 1
