@@ -297,6 +297,18 @@ int vvs_skip_decide(vvs_ctx* ctx, const int32_t* paths, const int32_t* path_len,
                     const uint8_t* last_verified, int32_t stride, float alpha, float threshold,
                     uint8_t* decision, float* similarity, void* stream);
 
+/* Unverified token selection with truncation (Sec. 4.2, Eq. 3; "UniformSample" in Algorithm 2): the
+ * tokens a verification-free step accepts.  For every image one candidate path is drawn uniformly,
+ * index floor(uniforms[b] * n_paths) with uniforms device float32 [n_images] in (0, 1), and cut to
+ * its first gamma = min(L_s, floor(L_bar)) tokens, L_s its own length and L_bar the mean length of
+ * all n_paths paths of the image.  paths / path_len as in vvs_skip_decide (path_len NULL = max_len).
+ * Outputs (device int32): out_path [n_images] the drawn index, out_gamma [n_images],
+ * out_tokens [n_images, max_len] the kept tokens followed by -1.  A length outside 0..max_len is
+ * clamped and sets VVS_DEV_BAD_ARG. */
+int vvs_select_unverified(vvs_ctx* ctx, const int32_t* paths, const int32_t* path_len, int32_t n_images,
+                          int32_t n_paths, int32_t max_len, const float* uniforms, int32_t* out_path,
+                          int32_t* out_gamma, int32_t* out_tokens, void* stream);
+
 /* Synchronise `stream`, copy the device status word to *out_bits (VVS_DEV_* bits) and clear
  * it.  Returns VVS_ERR_DEVICE_TIMEOUT / VVS_ERR_DEVICE_BOUNDS if such a bit was set. */
 int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits);

@@ -84,6 +84,8 @@ lib.vvs_feature_cache_fetch.argtypes = [_P, C.POINTER(vvs_fcache), _P, C.c_int32
 lib.vvs_skip_decide.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_int32, C.c_int32, _P,
                                 C.c_int32, C.c_float, C.c_float, _P, _P, _P]
 lib.vvs_skip_decide.restype = C.c_int
+lib.vvs_select_unverified.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P, _P, _P]
+lib.vvs_select_unverified.restype = C.c_int
 lib.vvs_device_status.argtypes = [_P, _P, C.POINTER(C.c_int32)]
 lib.vvs_last_launch_count.argtypes = [_P]
 lib.vvs_profile_enable.argtypes = [_P, C.c_int]
@@ -276,6 +278,14 @@ def vvs_skip_decide(ctx: int, paths, path_len, codebook, last_verified, stride: 
     _check(lib.vvs_skip_decide(ctx, _ptr(paths), _ptr(path_len), int(b), int(n), int(l), _ptr(codebook), int(v),
                                int(dim), _ptr(last_verified), int(stride), float(alpha), float(threshold),
                                _ptr(decision), _ptr(similarity), _stream(stream)), "vvs_skip_decide")
+
+
+def vvs_select_unverified(ctx: int, paths, path_len, uniforms, out_path, out_gamma, out_tokens, stream=None) -> None:
+    """Sec. 4.2 / Eq. 3: uniform draw of one candidate path per image, cut to gamma tokens."""
+    b, n, l = paths.shape
+    _check(lib.vvs_select_unverified(ctx, _ptr(paths), _ptr(path_len), int(b), int(n), int(l), _ptr(uniforms),
+                                     _ptr(out_path), _ptr(out_gamma), _ptr(out_tokens), _stream(stream)),
+           "vvs_select_unverified")
 
 
 def vvs_device_status(ctx: int, stream=None, raise_on_error: bool = False) -> int:

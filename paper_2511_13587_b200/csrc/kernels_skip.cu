@@ -101,7 +101,44 @@ skip_decide_kernel(const int32_t* __restrict__ paths, const int32_t* __restrict_
   }
 }
 
+// Unverified token selection with truncation (Sec. 4.2, Eq. 3): one warp per image.
+__global__ void select_unverified_kernel(const int32_t* __restrict__ paths, const int32_t* __restrict__ path_len,
+                                         const float* __restrict__ uniforms, int n_paths, int max_len,
+                                         int32_t* __restrict__ out_path, int32_t* __restrict__ out_gamma,
+                                         int32_t* __restrict__ out_tokens, int32_t* status) {
+  const int b = blockIdx.x, lane = threadIdx.x;
+  long long total = 0;
+  bool bad = false;
+  for (int i = lane; i < n_paths; i += 32) {
+    const int len = path_len ? path_len[(size_t)b * n_paths + i] : max_len;
+    bad |= len < 0 || len > max_len;
+    total += len < 0 ? 0 : (len > max_len ? max_len : len);
+  }
+  for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, VVS_DEV_BAD_ARG);
+  int idx = (int)floorf(uniforms[b] * (float)n_paths);
+  idx = idx < 0 ? 0 : (idx > n_paths - 1 ? n_paths - 1 : idx);
+  int len_s = path_len ? path_len[(size_t)b * n_paths + idx] : max_len;
+  len_s = len_s < 0 ? 0 : (len_s > max_len ? max_len : len_s);
+  const int mean_floor = (int)(total / n_paths);
+  const int gamma = len_s < mean_floor ? len_s : mean_floor;
+  if (lane == 0) {
+    out_path[b] = idx;
+    out_gamma[b] = gamma;
+  }
+  for (int t = lane; t < max_len; t += 32)
+    out_tokens[(size_t)b * max_len + t] = t < gamma ? paths[((size_t)b * n_paths + idx) * max_len + t] : -1;
+}
+
 }  // namespace
+
+int launch_select_unverified(const int32_t* paths, const int32_t* path_len, const float* uniforms, int n_images,
+                             int n_paths, int max_len, int32_t* out_path, int32_t* out_gamma, int32_t* out_tokens,
+                             int32_t* status, cudaStream_t s) {
+  select_unverified_kernel<<<n_images, 32, 0, s>>>(paths, path_len, uniforms, n_paths, max_len, out_path, out_gamma,
+                                                   out_tokens, status);
+  return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+}
 
 int launch_skip_decide(const int32_t* paths, const int32_t* path_len, const float* codebook,
                        const uint8_t* last_verified, int n_images, int n_paths, int max_len, int vocab, int dim,

@@ -729,6 +729,15 @@ int vvs_skip_decide(vvs_ctx* ctx, const int32_t* paths, const int32_t* path_len,
                             static_cast<cudaStream_t>(stream));
 }
 
+int vvs_select_unverified(vvs_ctx* ctx, const int32_t* paths, const int32_t* path_len, int32_t n_images,
+                          int32_t n_paths, int32_t max_len, const float* uniforms, int32_t* out_path,
+                          int32_t* out_gamma, int32_t* out_tokens, void* stream) {
+  if (!ctx || !paths || !uniforms || !out_path || !out_gamma || !out_tokens) return VVS_ERR_INVALID_ARG;
+  if (n_images < 1 || n_paths < 1 || max_len < 1) return VVS_ERR_SHAPE;
+  return launch_select_unverified(paths, path_len, uniforms, n_images, n_paths, max_len, out_path, out_gamma,
+                                  out_tokens, ctx->ws.status, static_cast<cudaStream_t>(stream));
+}
+
 int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits) {
   if (!ctx || !out_bits) return VVS_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -271,6 +271,10 @@ int launch_skip_decide(const int32_t* paths, const int32_t* path_len, const floa
                        int stride, float alpha, float threshold, uint8_t* decision, float* sim, int32_t* status,
                        cudaStream_t s);
 
+int launch_select_unverified(const int32_t* paths, const int32_t* path_len, const float* uniforms, int n_images,
+                             int n_paths, int max_len, int32_t* out_path, int32_t* out_gamma, int32_t* out_tokens,
+                             int32_t* status, cudaStream_t s);
+
 // ---- feature cache, kernels_fcache.cu ---------------------------------------------------------
 void launch_fcache_reset(const vvs_fcache& fc, cudaStream_t s);
 void launch_fcache_store(const vvs_fcache& fc, const void* hidden, int rows_per_seq, int d,

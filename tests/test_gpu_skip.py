@@ -85,3 +85,27 @@ def test_skip_decision_edge_cases_and_errors():
     with pytest.raises(vb.VvsError):
         vb.vvs_skip_decide(ctx, big, None, cb, None, 2, 0.5, 0.9, dec, sim)
     vb.vvs_destroy(ctx)
+
+
+def test_unverified_selection_is_bit_exact_with_oracle():
+    """Sec. 4.2 / Eq. 3 through the C ABI: drawn path, gamma and kept tokens equal the oracle's."""
+    ctx = _ctx()
+    rng = gen.rng_for(23, "select")
+    for b, n, l in ((1, 1, 1), (16, 24, 5), (9, 61, 16), (3, 7, 4)):
+        paths = rng.integers(0, 16384, size=(b, n, l)).astype(np.int32)
+        plen = rng.integers(0, l + 1, size=(b, n)).astype(np.int32)
+        u = rng.random(b).astype(np.float32).clip(1e-6, 1 - 1e-6)
+        u[0] = np.float32(1 - 1e-6)
+        op = torch.full((b,), -9, dtype=torch.int32, device="cuda")
+        og = torch.full((b,), -9, dtype=torch.int32, device="cuda")
+        ot = torch.full((b, l), -9, dtype=torch.int32, device="cuda")
+        for use_len in (True, False):
+            vb.vvs_select_unverified(ctx, torch.from_numpy(paths).cuda(), torch.from_numpy(plen).cuda() if use_len else None,
+                                     torch.from_numpy(u).cuda(), op, og, ot)
+            assert vb.vvs_device_status(ctx) == 0
+            for i in range(b):
+                # both sides take floor(u * N) on the float32 product
+                idx, g, toks = O.select_unverified(paths[i], plen[i] if use_len else np.full(n, l), np.float32(u[i]) * np.float32(n) / n)
+                assert int(op[i]) == idx and int(og[i]) == g
+                assert ot[i].tolist() == list(toks) + [-1] * (l - g)
+    vb.vvs_destroy(ctx)
