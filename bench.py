@@ -497,23 +497,20 @@ def run_epilogue_sweep(args) -> None:
 # Algorithm 2 of the paper as a loop over the library's entry points (one image)
 
 
-def run_generation_loop(args) -> None:
-    """VVS decoding loop (Alg. 2) on the LlamaGen-XL shape with a synthetic stand-in drafter: per
+def decoding_loops(ms, seed: int, runs, n_tokens: int = 576, k: int = 8, cfg_scale: float = 2.0,
+                   latent_dim: int = 8, warm: bool = True):
+    """VVS decoding loop (Alg. 2) on model shape `ms` with a synthetic stand-in drafter: per
     iteration a skip decision (vvs_skip_decide), then either a target verification of the K drafts
     behind the still unverified tokens (vvs_verify with n_forced = 1 + gamma: post verification,
     Sec. 4.1; feature-cache store) or a verification-free step (vvs_select_unverified; feature-cache
-    fetch of gamma stale features).  Reports generated tokens/s and TPF = tokens per target forward.
-    The drafter is synthetic (q = softmax(N(0,1)), a random candidate tree whose paths share a stem
-    and latent-space neighbours), so TPF here says nothing about image quality or real drafters."""
+    fetch of gamma stale features).  `runs` = [(name, threshold)].  Returns (device status,
+    {name: statistics incl. the per-iteration log}).  The drafter is synthetic (q = softmax(N(0,1)),
+    a random candidate tree whose paths share a stem), so tokens per forward says nothing about
+    image quality or real drafters."""
     import torch
     from paper_2511_13587_b200 import binding as vb
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-    if int(os.environ.get("RANK", "0")) != 0:
-        return
-    wl = CONFIGS[1]
-    ms = wl.shape
-    k, n_paths, depth, t_max = wl.n_draft_max, 12, 5, 1 + 5 + wl.n_draft_max
-    rng = gen.rng_for(wl.seed, "loop")
+    n_paths, depth, t_max = 12, 5, 1 + 5 + k
+    rng = gen.rng_for(seed, "loop")
 
     def dev(a):
         a = np.ascontiguousarray(a)
@@ -521,7 +518,7 @@ def run_generation_loop(args) -> None:
             return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
         return torch.from_numpy(a).cuda()
 
-    hw = gen.make_weights(ms, wl.seed)
+    hw = gen.make_weights(ms, seed)
     wd = {n: dev(v) for n, v in hw.items() if n != "layers"}
     wd["layers"] = [{n: dev(v) for n, v in hw["layers"][l].items()} for l in range(ms.n_layers)]
     del hw
@@ -529,12 +526,12 @@ def run_generation_loop(args) -> None:
     kv_v = torch.randn_like(kv_k)
     ctx = vb.vvs_create(vb.make_desc(ms, 2, t_max, 1))
     vb.vvs_bind_weights(ctx, wd)
-    codebook_h = gen.make_codebook(wl.seed, ms.vocab, wl.latent_dim).astype(np.float32)
+    codebook_h = gen.make_codebook(seed, ms.vocab, latent_dim).astype(np.float32)
     codebook = dev(codebook_h)
     fc = vb.make_fcache(torch.zeros((2, 5 + t_max, ms.d_model), dtype=torch.bfloat16, device="cuda"),
                         torch.zeros((2, 5 + t_max), dtype=torch.int32, device="cuda"),
                         torch.zeros((2,), dtype=torch.int32, device="cuda"))
-    q_all, d_all = gen.independent_draft(wl.seed, 0, 16, k, ms.vocab, DRAFT_LOGIT_STD)   # 16 draft sets, cycled
+    q_all, d_all = gen.independent_draft(seed, 0, 16, k, ms.vocab, DRAFT_LOGIT_STD)   # 16 draft sets, cycled
     q_dev = [dev(q_all[i:i + 1]) for i in range(16)]
     out = dict(accept_len=torch.zeros(1, dtype=torch.int32, device="cuda"),
                next_token=torch.zeros(1, dtype=torch.int32, device="cuda"),
@@ -564,8 +561,9 @@ def run_generation_loop(args) -> None:
         vb.vvs_feature_cache_reset(ctx, fc)
         fill, generated, forwards, skips, it, stored = 1, 0, 0, 0, 0, 0
         pending = []                                   # tokens accepted without verification, K/V not cached yet
-        last_tok, v_last = int(rng.integers(0, ms.vocab)), False      # Alg. 2 line 3
-        while generated < 576 and fill + t_max <= ms.s_max:
+        last_tok, v_last = ms.vocab_offset + int(rng.integers(0, ms.vocab)), False      # Alg. 2 line 3
+        log = []
+        while generated < n_tokens and fill + t_max <= ms.s_max:
             drafts = d_all[it % 16]
             stem = int(rng.integers(1, depth + 1))     # synthetic tree: shared stem, then latent-space neighbours or noise
             paths = np.tile(drafts[None, :depth], (n_paths, 1)).astype(np.int32)
@@ -578,19 +576,21 @@ def run_generation_loop(args) -> None:
             if not skip:
                 f = 1 + len(pending)
                 t_len = f + k
-                block_buf[:t_len].copy_(torch.tensor([last_tok] + pending + [int(x) for x in drafts], dtype=torch.int32))
+                block_buf[:t_len].copy_(torch.tensor([last_tok] + pending + [ms.vocab_offset + int(x) for x in drafts],
+                                                     dtype=torch.int32))
                 cl_buf.fill_(fill)
-                u_buf.copy_(torch.from_numpy(philox.verify_uniforms(wl.seed, it, 1, k)))
+                u_buf.copy_(torch.from_numpy(philox.verify_uniforms(seed, it, 1, k)))
                 q_buf.copy_(q_dev[it % 16])
                 o = dict(out, hidden=hid_buf[t_len])
                 vb.vvs_verify(ctx, n_images=1, n_cfg=2, n_forced=f, n_draft_max=k, block=block_buf, n_draft=None,
                               kv_k=kv_k, kv_v=kv_v, kv_rows=2, cache_len=cl_buf, draft_probs=q_buf, uniforms=u_buf,
-                              cfg_scale=wl.cfg_scale, temperature=1.0, mode=0, nbr_k=1, delta=float("inf"), **o)
+                              cfg_scale=cfg_scale, temperature=1.0, mode=0, nbr_k=1, delta=float("inf"), **o)
                 vb.vvs_feature_cache_store(ctx, fc, hid_buf[t_len], t_len, cl_buf, out["n_commit"])
                 n_acc, nxt = int(out["accept_len"].item()), int(out["next_token"].item())
                 fill += f + n_acc
                 stored += f + n_acc
                 generated += n_acc + 1
+                log.append(("verify", f, n_acc, int(out["new_len"][0].item())))
                 last_tok, pending, v_last = nxt, [], True
                 forwards += 1
             else:
@@ -600,23 +600,41 @@ def run_generation_loop(args) -> None:
                 if min(gamma, stored) > 0:               # the first steps have fewer cached features than gamma
                     gam_buf.fill_(min(gamma, 5, stored))
                     vb.vvs_feature_cache_fetch(ctx, fc, skip_all, 1, gam_buf, 5, 0, fetch_out, fetch_pos)
-                pending = pending + sel_tok[0, :gamma].tolist()
+                pending = pending + [ms.vocab_offset + t for t in sel_tok[0, :gamma].tolist()]
+                log.append(("skip", gamma, float(sim.item())))
                 generated += gamma
                 v_last = False
                 skips += 1
             it += 1
         torch.cuda.synchronize()
-        return generated, forwards, skips, it
+        return generated, forwards, skips, it, fill, log
 
     results = {}
-    for name, thr in (("never skip (plain speculative decoding)", 2.0), ("dynamic skip, threshold 0.65", 0.65)):
-        one_image(thr)                                   # warm-up: captures the graphs of every block shape
+    for name, thr in runs:
+        if warm:
+            one_image(thr)                               # captures the graphs of every block shape
         t0 = time.perf_counter()
-        gen_tok, fw, sk, its = one_image(thr)
+        gen_tok, fw, sk, its, fill, log = one_image(thr)
         dt = time.perf_counter() - t0
         results[name] = {"tokens": gen_tok, "target_forwards": fw, "skipped_steps": sk, "iterations": its,
-                         "tokens_per_forward": gen_tok / max(fw, 1), "tokens_per_s": gen_tok / dt, "seconds": dt}
+                         "tokens_per_forward": gen_tok / max(fw, 1), "tokens_per_s": gen_tok / dt, "seconds": dt,
+                         "final_fill": fill, "log": log}
     status = vb.vvs_device_status(ctx)
+    vb.vvs_destroy(ctx)
+    return status, results
+
+
+def run_generation_loop(args) -> None:
+    import torch
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    wl = CONFIGS[1]
+    status, results = decoding_loops(wl.shape, wl.seed, (("never skip (plain speculative decoding)", 2.0),
+                                                         ("dynamic skip, threshold 0.65", 0.65)),
+                                     k=wl.n_draft_max, cfg_scale=wl.cfg_scale, latent_dim=wl.latent_dim)
+    for r in results.values():
+        r.pop("log")
     print(json.dumps({"metric": "VVS decoding loop (Alg. 2), one 576-token image, LlamaGen-XL shape, synthetic drafter",
                       "unit": "generated tokens/s (host loop included)", "dtype": "bf16", "data": "synthetic",
                       "device_status": status, "runs": results}))
