@@ -450,3 +450,90 @@ def select_unverified(paths: np.ndarray, path_len: np.ndarray, u: float):
     idx = min(n - 1, int(np.floor(float(u) * n)))
     gamma = min(int(path_len[idx]), int(np.floor(np.sum(path_len, dtype=np.int64) / n)))
     return idx, gamma, np.asarray(paths[idx][:gamma])
+
+
+# ---------------------------------------------------------------------------------------
+# Tree verification (Sec. 2 / Sec. 5: the drafter proposes a candidate TREE, EAGLE-2 style; the
+# paper verifies it with the target in one pass and walks it with the sequential rule of Sec. 2)
+#
+# The paper does not print the tree rule.  Reading (**parity unpinned** by the paper; pinned here
+# by the lossless identity and by "a tree that is a chain is the chain rule"): multi-round
+# speculative sampling over the children of the current node, in index order, the children being
+# independent draws from the drafter's distribution q at that node: child x is accepted iff
+# u < min(1, p_res(x) / q(x)); after a rejection p_res <- norm(max(0, p_res - q)) and the next
+# sibling is tried; when no child is left the next token is drawn from p_res (from the node's own
+# target row if it has no children).  Block row t attends the cache and its ancestors only, and
+# sits at position fill + depth(t).
+
+
+def tree_ancestors(parent, t: int) -> list:
+    """Block rows on the path root .. t (row 0 is the root; parent[0] = -1)."""
+    path = []
+    while t >= 0:
+        path.append(t)
+        t = int(parent[t])
+    return path[::-1]
+
+
+def tree_forward(ms, weights: dict, tokens: np.ndarray, parent: np.ndarray, kc: np.ndarray,
+                 vc: np.ndarray, fill: int):
+    """Features and keys/values of every node of the candidate tree: node t is the LAST row of
+    the plain chain forward over its root path (cache untouched).  Returns h [T, d],
+    k_node, v_node [n_layers, H, T, hd]."""
+    t_len = len(tokens)
+    h = np.zeros((t_len, ms.d_model))
+    k_node = np.zeros((ms.n_layers, ms.n_heads, t_len, ms.head_dim))
+    v_node = np.zeros_like(k_node)
+    for t in range(t_len):
+        path = tree_ancestors(parent, t)
+        kc_t, vc_t = kc.copy(), vc.copy()
+        ht = target_forward(ms, weights, np.asarray(tokens)[path], kc_t, vc_t, fill)
+        h[t] = ht[-1]
+        slot = fill + len(path) - 1
+        k_node[:, :, t] = kc_t[:, :, slot]
+        v_node[:, :, t] = vc_t[:, :, slot]
+    return h, k_node, v_node
+
+
+def tree_decide(p32: np.ndarray, draft_tokens: np.ndarray, parent: np.ndarray, n_forced: int,
+                q32: np.ndarray, u32: np.ndarray) -> dict:
+    """Walk of one image's candidate tree.  p32 [T, V] float32 target rows (row t = distribution
+    of the token after node t); draft node i = block row n_forced + i carries codebook token
+    draft_tokens[i], was drawn from q32[i] (the drafter's distribution at its parent) and is judged
+    with u32[i]; u32[K] drives the final sample.  The first residual is the float32 difference (as
+    in the chain rule); later rounds work in float64."""
+    p32 = np.asarray(p32, dtype=np.float32)
+    q32 = np.asarray(q32, dtype=np.float32)
+    t_len, k_max = p32.shape[0], len(u32) - 1
+    margins = np.full(k_max + 1, np.inf)
+    cur, path = n_forced - 1, []
+    while True:
+        children = [c for c in range(n_forced, t_len) if int(parent[c]) == cur]
+        if not children:
+            r = p32[cur].astype(np.float64)                      # leaf: the bonus token
+            break
+        p_res, first_round, accepted = p32[cur].astype(np.float64), True, None
+        sample_from = p_res                                      # un-normalised residual of the last rejection
+        for c in children:
+            i = c - n_forced
+            x = int(draft_tokens[i])
+            ratio = acceptance_ratio(float(p_res[x]), float(q32[i, x]))
+            margins[i] = abs(float(u32[i]) - ratio)
+            if float(u32[i]) < ratio:
+                accepted = c
+                break
+            if first_round:
+                r = np.maximum(np.float32(0.0), p32[cur] - q32[i]).astype(np.float64)   # IEEE float32
+            else:
+                r = np.maximum(0.0, p_res - q32[i].astype(np.float64))
+            z = float(np.sum(r))
+            if z > 0.0:                                          # p_res == q numerically: keep p_res
+                p_res, sample_from = r / z, r
+                first_round = False
+        if accepted is None:
+            r = sample_from
+            break
+        path.append(accepted)
+        cur = accepted
+    token, margins[k_max] = inverse_cdf(r, float(u32[k_max]))
+    return {"accept_len": len(path), "accept_path": path, "next_token": int(token), "margins": margins}
