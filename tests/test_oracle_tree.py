@@ -30,11 +30,12 @@ def test_chain_shaped_tree_is_the_chain_rule():
 def test_two_sibling_candidates_are_lossless_by_enumeration():
     """Root with two children drawn independently from q: the first emitted token (an accepted child
     or the residual sample) is distributed as p.  p, q chosen so that every ratio is a multiple of
-    1/4 and the last residual has masses 7/9, 2/9: the midpoint grids integrate exactly."""
-    p = np.array([[0.4, 0.3, 0.2, 0.1]] * 3, dtype=np.float32)
-    q = np.array([0.2, 0.2, 0.2, 0.4], dtype=np.float32)
+    1/4 and the last residual has masses 17/24, 7/24 (15/20, 5/20 if the first residual were not
+    normalised, which would break the identity): the midpoint grids integrate exactly."""
+    p = np.array([[0.5, 0.3, 0.1, 0.1]] * 3, dtype=np.float32)
+    q = np.array([0.1, 0.1, 0.4, 0.4], dtype=np.float32)
     parent = np.array([-1, 0, 0])
-    g, gs = 20, 90
+    g, gs = 20, 120
     out = np.zeros(4)
     for x1 in range(4):
         for x2 in range(4):
