@@ -166,6 +166,21 @@ typedef struct vvs_verify_args {
   int32_t nbr_k;            /* relaxed: use the first nbr_k entries of each CSR row */
   float delta;              /* relaxed: pooled neighbour mass (excluding p(x)) stays <= delta;
                                INFINITY = pool all nbr_k neighbours */
+  const int32_t* tree_parent; /* NULL: the K drafts are a chain.  Otherwise device [B, T]: parent block
+                               row of every block row of a candidate TREE (the drafter of the paper
+                               proposes a token tree, Sec. 5): -1 for row 0, t - 1 for the forced rows
+                               t < F, and for draft node t >= F any row in [F - 1, t).  Row t then
+                               attends the cache and its ancestors only and sits at position
+                               cache_len + depth(t); draft_probs[b, i] is the drafter's distribution
+                               at the PARENT of node F + i (siblings carry the same row) and the
+                               children of a node are taken to be independent draws from it.
+                               Verification walks the tree from row F - 1: the children of the current
+                               node are tried in index order, child x passes iff
+                               u < min(1, p_res(x) / q(x)), a rejection replaces p_res by
+                               norm(max(0, p_res - q)); when no child is left the next token is drawn
+                               from p_res (from the node's own target row if it is a leaf).  Tree
+                               calls need bf16, at most 32 block tokens, strict mode, n_draft == NULL
+                               and out->target_probs (the walk reads whole target rows). */
 } vvs_verify_args;
 
 /* Outputs, device memory allocated by the caller.  Optional ones may be NULL and are then
@@ -180,6 +195,10 @@ typedef struct vvs_verify_out {
   uint8_t* accept_mask; /* optional [B, K] */
   float* target_probs;  /* optional [B, T, V] float32 target distributions after guidance */
   void* hidden;         /* optional T [R, T, d_model] features (final-norm output) */
+  int32_t* accept_path; /* optional [B, K] (tree calls): block rows of the accepted nodes, root side
+                           first, then -1.  After a tree call the K/V of the accepted nodes have been
+                           moved to slots cache_len + F .. cache_len + F + accept_len - 1, so the
+                           cache is contiguous again; `hidden` stays in block-row order */
   float* margins;       /* optional [B, K+1]: |u_i - ratio_i| for judged drafts (INFINITY for
                            drafts not judged) and, in column K, the distance of the sample
                            point to the nearest CDF bin edge as a fraction of the total mass */

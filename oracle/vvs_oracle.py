@@ -537,3 +537,39 @@ def tree_decide(p32: np.ndarray, draft_tokens: np.ndarray, parent: np.ndarray, n
         cur = accepted
     token, margins[k_max] = inverse_cdf(r, float(u32[k_max]))
     return {"accept_len": len(path), "accept_path": path, "next_token": int(token), "margins": margins}
+
+
+def tree_verify(ms, weights: dict, block: np.ndarray, parent: np.ndarray, n_forced: int,
+                kv_k: np.ndarray, kv_v: np.ndarray, cache_len: np.ndarray, draft_probs: np.ndarray,
+                uniforms: np.ndarray, n_cfg: int, cfg_scale: float, temperature: float = 1.0) -> dict:
+    """One verification step over candidate trees: tree_forward per sequence, guidance and
+    softmax per image as in `epilogue`, then tree_decide.  block [B, T] embedding-table ids,
+    parent [B, T].  Returns accept_len, accept_path (list per image, block rows), next_token
+    (embedding-table id), new_len, target_probs [B, T, V], hidden [R, T, d] and the per-node
+    keys/values k_node, v_node [n_layers, R, H, T, hd] (node order, not cache order)."""
+    n_images, t_len = block.shape
+    n_rows = n_images * n_cfg
+    hidden = np.zeros((n_rows, t_len, ms.d_model))
+    k_node = np.zeros((ms.n_layers, n_rows, ms.n_heads, t_len, ms.head_dim))
+    v_node = np.zeros_like(k_node)
+    for r in range(n_rows):
+        b = r % n_images
+        hidden[r], k_node[:, r], v_node[:, r] = tree_forward(
+            ms, weights, block[b], parent[b], widen(kv_k[:, r]), widen(kv_v[:, r]), int(cache_len[r]))
+    out = {"accept_len": np.zeros(n_images, np.int32), "next_token": np.zeros(n_images, np.int32),
+           "accept_path": [], "margins": np.zeros((n_images, uniforms.shape[1])),
+           "target_probs": np.zeros((n_images, t_len, ms.vocab))}
+    for b in range(n_images):
+        l_c = lm_head_logits(ms, weights, widen(hidden[b]))
+        l_u = lm_head_logits(ms, weights, widen(hidden[n_images + b])) if n_cfg == 2 else None
+        out["target_probs"][b] = guided_probs(l_c, l_u, cfg_scale, temperature)
+        dec = tree_decide(out["target_probs"][b].astype(np.float32), block[b, n_forced:] - ms.vocab_offset,
+                          parent[b], n_forced, draft_probs[b], uniforms[b])
+        out["accept_len"][b] = dec["accept_len"]
+        out["accept_path"].append(dec["accept_path"])
+        out["next_token"][b] = dec["next_token"] + ms.vocab_offset
+        out["margins"][b] = dec["margins"]
+    out["hidden"], out["k_node"], out["v_node"] = hidden, k_node, v_node
+    out["new_len"] = np.array([int(cache_len[r]) + n_forced + int(out["accept_len"][r % n_images])
+                               for r in range(n_rows)], dtype=np.int32)
+    return out

@@ -49,12 +49,13 @@ class vvs_verify_args(C.Structure):
                 ("cache_len", C.c_void_p), ("cache_len_host", C.c_void_p),
                 ("draft_probs", C.c_void_p), ("uniforms", C.c_void_p), ("cfg_scale", C.c_float),
                 ("temperature", C.c_float), ("mode", C.c_int32), ("nbr_k", C.c_int32),
-                ("delta", C.c_float)]
+                ("delta", C.c_float), ("tree_parent", C.c_void_p)]
 
 
 class vvs_verify_out(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("accept_len", "next_token", "new_len", "n_commit", "accept_mask",
-                                          "target_probs", "hidden", "margins")]
+                                          "target_probs", "hidden", "accept_path",
+                                          "margins")]
 
 
 class vvs_fcache(C.Structure):
@@ -182,26 +183,28 @@ def vvs_bind_neighbors(ctx: int, row_ptr: torch.Tensor, col: torch.Tensor) -> No
 
 
 def _args(n_images, n_cfg, n_forced, n_draft_max, block, n_draft, kv_k, kv_v, kv_rows, cache_len,
-          cache_len_host, draft_probs, uniforms, cfg_scale, temperature, mode, nbr_k, delta):
+          cache_len_host, draft_probs, uniforms, cfg_scale, temperature, mode, nbr_k, delta,
+          tree_parent=None):
     return vvs_verify_args(int(n_images), int(n_cfg), int(n_forced), int(n_draft_max), _ptr(block),
                            _ptr(n_draft), _ptr(kv_k), _ptr(kv_v), int(kv_rows), _ptr(cache_len),
                            _ptr(cache_len_host), _ptr(draft_probs), _ptr(uniforms), float(cfg_scale),
-                           float(temperature), int(mode), int(nbr_k), float(delta))
+                           float(temperature), int(mode), int(nbr_k), float(delta), _ptr(tree_parent))
 
 
-def _out(accept_len, next_token, new_len, n_commit, accept_mask, target_probs, hidden, margins):
+def _out(accept_len, next_token, new_len, n_commit, accept_mask, target_probs, hidden, margins,
+         accept_path=None):
     return vvs_verify_out(_ptr(accept_len), _ptr(next_token), _ptr(new_len), _ptr(n_commit), _ptr(accept_mask),
-                          _ptr(target_probs), _ptr(hidden), _ptr(margins))
+                          _ptr(target_probs), _ptr(hidden), _ptr(accept_path), _ptr(margins))
 
 
 def vvs_verify(ctx: int, *, n_images, n_cfg, n_forced, n_draft_max, block, kv_k, kv_v, kv_rows,
                cache_len, draft_probs, uniforms, accept_len, next_token, new_len, n_draft=None,
                cache_len_host=None, cfg_scale=1.0, temperature=1.0, mode=VVS_MODE_STRICT, nbr_k=1,
                delta=float("inf"), n_commit=None, accept_mask=None, target_probs=None, hidden=None,
-               margins=None, stream=None) -> None:
+               margins=None, tree_parent=None, accept_path=None, stream=None) -> None:
     a = _args(n_images, n_cfg, n_forced, n_draft_max, block, n_draft, kv_k, kv_v, kv_rows, cache_len,
-              cache_len_host, draft_probs, uniforms, cfg_scale, temperature, mode, nbr_k, delta)
-    o = _out(accept_len, next_token, new_len, n_commit, accept_mask, target_probs, hidden, margins)
+              cache_len_host, draft_probs, uniforms, cfg_scale, temperature, mode, nbr_k, delta, tree_parent)
+    o = _out(accept_len, next_token, new_len, n_commit, accept_mask, target_probs, hidden, margins, accept_path)
     _check(lib.vvs_verify(ctx, C.byref(a), C.byref(o), _stream(stream)), "vvs_verify")
 
 

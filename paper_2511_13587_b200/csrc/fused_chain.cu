@@ -74,6 +74,7 @@ struct ChainParams {
   float* gu_acc;                       // [2][m, 2ff]
   float* ss;                           // [2 * n_layers][32] sums of squares of x rows
   const int32_t* cache_len;
+  const uint32_t* anc_mask;            // [m] block rows visible to each block row (chain or tree)
   __nv_bfloat16* kv_k;
   __nv_bfloat16* kv_v;
   const float* rope_cos;
@@ -294,6 +295,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_abort;
   __shared__ int s_fill[kMaxSeq], s_nch[kMaxSeq], s_prefix[kMaxSeq + 1];
+  __shared__ uint32_t s_anc[32];
   __shared__ float row_max[32], row_sum[32];
   VVS_TRACE_DECL
 
@@ -336,6 +338,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
     }
     s_prefix[p.n_rows] = acc;
   }
+  if (tid >= 32 && tid < 64) s_anc[tid - 32] = (int)(tid - 32) < p.m ? p.anc_mask[tid - 32] : 0u;
   // token operands: rows of tokens that do not exist stay zero for the whole kernel
   for (uint32_t i = tid; i < NS * (kTokSlabBytes / 16); i += kThreads)
     reinterpret_cast<uint4*>(ring + (size_t)(i / (kTokSlabBytes / 16)) * kStageBytes + kSlabBytes)[i % (kTokSlabBytes / 16)] =
@@ -661,9 +664,11 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
                 const float4 s4 = reinterpret_cast<const float4*>(sP + (t >> 4) * kSlabBytes + 4096)[(t & 15) * 32 + lane];
                 float sv[4] = {s4.x, s4.y, s4.z, s4.w};
                 float mx = -CUDART_INF_F;
+                const uint32_t anc = s_anc[r * T + t];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                  sv[j] = (key0 + 4 * lane + j <= fill + t) ? sv[j] * p.scale : -CUDART_INF_F;
+                  const int kj = key0 + 4 * lane + j - fill;   // < 0: cache; else block row kj
+                  sv[j] = (kj < 0 || (kj < 32 && ((anc >> kj) & 1u))) ? sv[j] * p.scale : -CUDART_INF_F;
                   mx = fmaxf(mx, sv[j]);
                 }
                 mx = warp_max_f(mx);
@@ -955,7 +960,7 @@ int launch_fused_chain(const FusedChainArgs& a, cudaStream_t s) {
   p.wmaps = a.wmaps; p.tok_emb = a.tok_emb; p.block = a.block;
   for (int i = 0; i < 2 * md.n_layers; ++i) p.norms[i] = a.norms_host[i];
   p.x = a.x; p.qkv_acc = a.qkv_acc; p.gu_acc = a.gu_acc; p.ss = a.ss;
-  p.cache_len = a.cache_len; p.kv_k = a.kv_k; p.kv_v = a.kv_v;
+  p.cache_len = a.cache_len; p.anc_mask = a.anc_mask; p.kv_k = a.kv_k; p.kv_v = a.kv_v;
   p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin;
   p.part_o = a.part_o; p.part_ml = a.part_ml; p.sync_words = a.sync_words; p.status = a.status;
   int stages = 0;

@@ -292,17 +292,52 @@ gemm_tc_kernel(const KernelParams p, const __grid_constant__ CUtensorMap tm_a,
 }
 
 // ---------------------------------------------------------------------------------------------
-// positions, validity and rotation tables of the block rows: the same for every layer of a call
+// positions, validity, visibility and rotation tables of the block rows: the same for every
+// layer of a call.  Chain: row t sits at position fill + t and sees block rows 0..t.  Tree
+// (tree_parent given): row t sits at fill + depth(t) and sees its ancestors and itself; its K/V
+// still go to cache slot fill + t.
 __global__ void rope_table_kernel(const int32_t* __restrict__ cache_len, const float* __restrict__ inv_freq,
-                                  int32_t* __restrict__ slot_pos, float* __restrict__ rope_cos,
-                                  float* __restrict__ rope_sin, int t_len, int hd, int s_max, int rope_mode,
-                                  int grid_w, int n_prefix, int32_t* status) {
+                                  const int32_t* __restrict__ tree_parent, int n_images, int n_forced,
+                                  int32_t* __restrict__ slot_pos, uint32_t* __restrict__ anc_mask,
+                                  float* __restrict__ rope_cos, float* __restrict__ rope_sin, int t_len, int hd,
+                                  int s_max, int rope_mode, int grid_w, int n_prefix, int32_t* status) {
+  __shared__ int s_depth;
   const int m = blockIdx.x, r = m / t_len, t = m % t_len;
   const int fill = cache_len[r];
   const bool ok = fill >= 0 && fill + t_len <= s_max;
   if (!ok && threadIdx.x == 0) atomicOr(status, VVS_DEV_CACHE_OVERFLOW);
-  const int pos = fill + t;
-  if (threadIdx.x == 0) slot_pos[m] = ok ? pos : -1;
+  if (threadIdx.x == 0) {
+    int depth = t;
+    uint32_t mask = t >= 31 ? 0xffffffffu : ((2u << t) - 1u);
+    if (tree_parent) {
+      const int32_t* par = tree_parent + (size_t)(r % n_images) * t_len;
+      bool bad = false;
+      depth = 0;
+      mask = 1u << t;
+      for (int c = t, steps = 0; c > 0 && steps < 32; ++steps) {
+        const int q = par[c];
+        // forced rows form a chain; a draft node hangs below the last forced row or a draft node
+        if (q < 0 || q >= c || (c < n_forced && q != c - 1) || (c >= n_forced && q < n_forced - 1)) {
+          bad = true;
+          break;
+        }
+        mask |= 1u << q;
+        ++depth;
+        c = q;
+      }
+      if (par[0] != -1) bad = true;
+      if (bad) {
+        atomicOr(status, VVS_DEV_BAD_ARG);
+        depth = t;
+        mask = t >= 31 ? 0xffffffffu : ((2u << t) - 1u);
+      }
+    }
+    s_depth = depth;
+    slot_pos[m] = ok ? fill + t : -1;
+    anc_mask[m] = mask;
+  }
+  __syncthreads();
+  const int pos = fill + s_depth;
   float c_lo = 0.f, c_hi = 0.f;
   if (rope_mode == VVS_ROPE_1D) {
     c_lo = c_hi = (float)pos;
@@ -440,11 +475,12 @@ int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStr
   return e == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
 }
 
-void launch_rope_table(const int32_t* cache_len, const Workspace& ws, const vvs_model_desc& md, int n_rows,
-                       int t_len, cudaStream_t s) {
-  rope_table_kernel<<<n_rows * t_len, 64, 0, s>>>(cache_len, ws.rope_inv_freq, ws.slot_pos, ws.rope_cos,
-                                                  ws.rope_sin, t_len, md.head_dim, md.s_max, md.rope_mode,
-                                                  md.rope_grid_w, md.n_prefix, ws.status);
+void launch_rope_table(const int32_t* cache_len, const int32_t* tree_parent, int n_images, int n_forced,
+                       const Workspace& ws, const vvs_model_desc& md, int n_rows, int t_len, cudaStream_t s) {
+  rope_table_kernel<<<n_rows * t_len, 64, 0, s>>>(cache_len, ws.rope_inv_freq, tree_parent, n_images, n_forced,
+                                                  ws.slot_pos, ws.anc_mask, ws.rope_cos, ws.rope_sin, t_len,
+                                                  md.head_dim, md.s_max, md.rope_mode, md.rope_grid_w, md.n_prefix,
+                                                  ws.status);
 }
 
 }  // namespace vvs

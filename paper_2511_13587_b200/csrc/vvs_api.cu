@@ -47,6 +47,9 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
       const size_t wide = 3 * dm > 2 * ff ? 3 * dm : 2 * ff;
       const size_t tiles = (wide + 127) / 128, passes = (M + 255) / 256;
       c.take(ws.slot_pos, M * 4);
+      c.take(ws.anc_mask, M * 4);
+      c.take(ws.tree_res, (size_t)2 * (d.max_rows < 32 ? d.max_rows : 32) * V * 8);
+      c.take(ws.tree_path, (size_t)32 * 32 * 4);
       c.take(ws.rope_cos, M * (size_t)(d.head_dim / 2) * 4);
       c.take(ws.rope_sin, M * (size_t)(d.head_dim / 2) * 4);
       c.take(ws.sk_scratch, M * wide * 4);
@@ -244,6 +247,45 @@ int run_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, 
   return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
 }
 
+// Tree calls: LM head with guidance over all block rows, probabilities written out, walk of the
+// tree on them, then the K/V of the accepted nodes move up behind the forced rows.
+int run_tree_decisions(vvs_ctx* ctx, const __nv_bfloat16* hid, const vvs_verify_args* a, const vvs_verify_out* o,
+                       cudaStream_t s) {
+  const vvs_model_desc& md = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const int B = a->n_images, C = a->n_cfg, R = B * C, Tn = a->n_forced + a->n_draft_max;
+  const int M = R * Tn, V = md.vocab, BT = B * Tn;
+  CUtensorMap tm_hid;
+  if (make_tmap_bf16_2d(&tm_hid, hid, (uint64_t)M, (uint64_t)md.d_model, (uint32_t)lmhead_box_rows(BT)) != VVS_OK)
+    return VVS_ERR_CUDA;
+  LmHeadArgs la{};
+  la.v = V; la.k = md.d_model; la.bt = BT; la.n_cfg = C; la.tm_a = &ctx->lm_map; la.tm_b = &tm_hid;
+  la.pdl = ctx->use_pdl; la.cfg_scale = a->cfg_scale; la.inv_temp = 1.f / a->temperature;
+  la.part_m = ws.part_m; la.part_s = ws.part_s; la.logits_out = o->target_probs; la.status = ws.status;
+  la.rows_per_seq = Tn; la.first_row = a->n_forced - 1; la.n_draft_max = 0;
+  la.vocab_offset = md.vocab_offset; la.relaxed = 0; la.nbr_k = 1; la.kmax = md.max_nbr_k; la.drafts_ld = Tn;
+  la.drafts = a->block + a->n_forced; la.row_ptr = ctx->nbr_row_ptr; la.col = ctx->nbr_col;
+  la.l_tok = ws.l_tok; la.l_nbr = ws.l_nbr;
+  int rc = VVS_OK;
+  VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_lmhead_tc(la, s));
+  if (rc != VVS_OK) return rc;
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_finalize_stats(ws, (V + 127) / 128, BT, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_probs_from_logits(o->target_probs, ws, o->target_probs, BT, V, s));
+  TreeParams tp{};
+  tp.n_images = B; tp.n_cfg = C; tp.n_forced = a->n_forced; tp.n_draft_max = a->n_draft_max; tp.t_len = Tn;
+  tp.vocab = V; tp.vocab_offset = md.vocab_offset; tp.parent = a->tree_parent; tp.drafts = a->block + a->n_forced;
+  tp.probs = o->target_probs; tp.draft_probs = a->draft_probs; tp.uniforms = a->uniforms; tp.cache_len = a->cache_len;
+  tp.res = ws.tree_res; tp.accept_len = o->accept_len;
+  tp.accept_path = o->accept_path ? o->accept_path : ws.tree_path;
+  tp.next_token = o->next_token; tp.new_len = o->new_len; tp.n_commit = o->n_commit;
+  tp.accept_mask = o->accept_mask; tp.margins = o->margins; tp.status = ws.status;
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_tree_walk(tp, s));
+  if (a->n_draft_max > 0)
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_tree_commit(a->kv_k, a->kv_v, a->cache_len, o->accept_len, tp.accept_path, md,
+                                                  a->kv_rows, B, C, a->n_forced, a->n_draft_max, s));
+  return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+}
+
 // bf16 contexts: projections on the tensor cores (gemm_tc.cu), everything else as above.
 int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, cudaStream_t s) {
   using T = __nv_bfloat16;
@@ -298,19 +340,21 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     fc.tok_emb = static_cast<const T*>(ctx->tok_emb); fc.block = a->block;
     fc.x = ws.x; fc.qkv_acc = ws.chain_qkv; fc.gu_acc = ws.chain_gu; fc.ss = ws.chain_ss;
     fc.cache_len = a->cache_len; fc.kv_k = kv_k; fc.kv_v = kv_v; fc.tm_k = &tm_k; fc.tm_v = &tm_v;
-    fc.slot_pos = ws.slot_pos; fc.rope_cos = ws.rope_cos; fc.rope_sin = ws.rope_sin;
+    fc.slot_pos = ws.slot_pos; fc.anc_mask = ws.anc_mask; fc.rope_cos = ws.rope_cos; fc.rope_sin = ws.rope_sin;
     fc.part_o = ws.attn_part_o; fc.part_ml = ws.attn_part_ml; fc.sync_words = ws.chain_sync;
     fc.status = ws.status;
-    VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, ws, md, R, Tn, s));
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, a->tree_parent, B, a->n_forced, ws, md, R, Tn, s));
     VVS_LAUNCH(VVS_PROF_CHAIN, rc = launch_fused_chain(fc, s));
     if (rc != VVS_OK) return rc;
     VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
     if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
+    if (a->tree_parent) return run_tree_decisions(ctx, hid, a, o, s);
     return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
   }
   VVS_LAUNCH(VVS_PROF_OTHER, launch_embed<T>(static_cast<const T*>(ctx->tok_emb), a->block, ws.x, B, C, Tn,
                                              d, md.tok_rows, ws.status, s));
-  VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, ws, md, R, Tn, s));
+  if (a->tree_parent) return VVS_ERR_SHAPE;   // trees run on the whole-chain kernel only
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, nullptr, B, a->n_forced, ws, md, R, Tn, s));
   for (int l = 0; l < md.n_layers && rc == VVS_OK; ++l) {
     const Layer& L = ctx->layers[l];
     const LayerMaps& W = ctx->layer_maps[l];
@@ -617,6 +661,12 @@ int vvs_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, 
   const int R = a->n_images * a->n_cfg;
   if (!a->block || !a->kv_k || !a->kv_v || !a->cache_len || !o->new_len) return VVS_ERR_INVALID_ARG;
   if (a->kv_rows < R) return VVS_ERR_SHAPE;
+  if (a->tree_parent) {
+    if (a->mode != VVS_MODE_STRICT || a->n_draft || !o->target_probs) return VVS_ERR_INVALID_ARG;
+    if (!ctx->tensor_core_path || !ctx->use_chain || !fused_chain_applicable(md, R, Tn)) return VVS_ERR_SHAPE;
+  } else if (o->accept_path) {
+    return VVS_ERR_INVALID_ARG;
+  }
   if (!aligned16(a->kv_k) || !aligned16(a->kv_v) || !aligned16(o->hidden)) return VVS_ERR_ALIGN;
   if (a->cache_len_host) {
     for (int r = 0; r < R; ++r)
@@ -639,7 +689,7 @@ int vvs_epilogue(vvs_ctx* ctx, const void* hidden, int32_t n_rows_per_seq, int32
   if (rc != VVS_OK) return rc;
   if (first_row < 0 || first_row + a->n_draft_max > n_rows_per_seq) return VVS_ERR_SHAPE;
   if (a->n_draft_max > 0 && !drafts) return VVS_ERR_INVALID_ARG;
-  if (o->new_len || o->hidden) return VVS_ERR_INVALID_ARG;
+  if (o->new_len || o->hidden || a->tree_parent || o->accept_path) return VVS_ERR_INVALID_ARG;
   if (!aligned16(hidden)) return VVS_ERR_ALIGN;
   ctx->launches = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -662,6 +712,7 @@ int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, 
   if (first_row < 0 || first_row + a->n_draft_max > n_rows_per_seq) return VVS_ERR_SHAPE;
   if (a->n_draft_max > 0 && !drafts) return VVS_ERR_INVALID_ARG;
   if (o->new_len || o->hidden || o->n_commit || o->target_probs) return VVS_ERR_INVALID_ARG;
+  if (a->tree_parent || o->accept_path) return VVS_ERR_INVALID_ARG;
   if (!aligned16(target_probs)) return VVS_ERR_ALIGN;
   ctx->launches = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

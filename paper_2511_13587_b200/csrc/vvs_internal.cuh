@@ -46,6 +46,9 @@ struct Workspace {
   float* rope_inv_freq = nullptr;  // [head_dim/2] angle per unit coordinate of each pair
   // tensor-core path
   int32_t* slot_pos = nullptr;   // [M] cache slot of each block row, -1 if its sequence overflows
+  uint32_t* anc_mask = nullptr;  // [M] bit j set: block row j of the same sequence is visible (ancestor or self)
+  double* tree_res = nullptr;    // [2][min(max_rows, 32), V] residuals of the tree walk (ping-pong)
+  int32_t* tree_path = nullptr;  // [32, 32] accepted nodes when the caller does not ask for them
   float* rope_cos = nullptr;     // [M, head_dim/2]
   float* rope_sin = nullptr;     // [M, head_dim/2]
   float* sk_scratch = nullptr;   // [M, max(3d, 2ff)] fp32 split-K sums; all zero between kernels
@@ -174,7 +177,8 @@ int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_
 int make_weight_tmap(CUtensorMap* out, const void* w, int rows, int cols);
 GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_sms);
 int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStream_t s);
-void launch_rope_table(const int32_t* cache_len, const Workspace& ws, const vvs_model_desc& md, int n_rows,
+void launch_rope_table(const int32_t* cache_len, const int32_t* tree_parent, int n_images, int n_forced,
+                       const Workspace& ws, const vvs_model_desc& md, int n_rows,
                        int t_len, cudaStream_t s);
 
 // ---- tensor-core attention, attention_tc.cu ----------------------------------------------------------
@@ -224,11 +228,29 @@ struct FusedChainArgs {
   __nv_bfloat16* kv_k; __nv_bfloat16* kv_v;
   const CUtensorMap* tm_k;              // host copies of the cache descriptors (box {64, 128})
   const CUtensorMap* tm_v;
-  const int32_t* slot_pos; const float* rope_cos; const float* rope_sin;
+  const int32_t* slot_pos; const uint32_t* anc_mask; const float* rope_cos; const float* rope_sin;
   float* part_o; float* part_ml;
   unsigned* sync_words;
   int32_t* status;
 };
+// Walk of the candidate trees (tree calls of vvs_verify) and the cache compaction after it.
+struct TreeParams {
+  int n_images, n_cfg, n_forced, n_draft_max, t_len, vocab, vocab_offset;
+  const int32_t* parent;      // [B, T]
+  const int32_t* drafts;      // block + n_forced, row stride t_len
+  const float* probs;         // [B, T, V] target rows of all block rows
+  const float* draft_probs;   // [B, K, V]
+  const float* uniforms;      // [B, K+1]
+  const int32_t* cache_len;
+  double* res;                // [2][B, V]
+  int32_t* accept_len; int32_t* accept_path; int32_t* next_token; int32_t* new_len; int32_t* n_commit;
+  uint8_t* accept_mask; float* margins;
+  int32_t* status;
+};
+void launch_tree_walk(const TreeParams& p, cudaStream_t s);
+void launch_tree_commit(void* kv_k, void* kv_v, const int32_t* cache_len, const int32_t* accept_len,
+                        const int32_t* accept_path, const vvs_model_desc& md, int kv_rows, int n_images, int n_cfg,
+                        int n_forced, int n_draft_max, cudaStream_t s);
 bool fused_chain_applicable(const vvs_model_desc& md, int n_rows, int t_len);
 size_t fused_chain_smem_bytes(const vvs_model_desc& md, int t_len, int* w_stages);
 int launch_fused_chain(const FusedChainArgs& a, cudaStream_t s);

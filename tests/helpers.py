@@ -203,3 +203,86 @@ def check_new_cache_rows(case, gpu: dict, ora: dict, rtol: float):
             np.testing.assert_array_equal(got[:, r, :, fill + t_len:], orig[:, r, :, fill + t_len:])
     for r in range(c["n_images"] * c["n_cfg"], c["kv_rows"]):
         np.testing.assert_array_equal(gpu["kv_k"][:, r], k0[:, r])
+
+
+# ---------------------------------------------------------------------------------------
+# candidate trees
+
+
+def build_tree_case(ms: ModelShape, seed: int, n_images: int, n_cfg: int, n_forced: int, parent,
+                    fills, cfg_scale: float = 2.0, temperature: float = 1.0, q_noise: float = 1.0,
+                    kv_rows=None, call_id: int = 0):
+    """Seeded inputs of one tree verify call.  parent int [T] (shared) or [B, T].  The children of
+    a node are independent draws from one drafter row, the oracle's guided target logits at that
+    node plus N(0, q_noise^2)."""
+    parent = np.asarray(parent, dtype=np.int32)
+    if parent.ndim == 1:
+        parent = np.tile(parent, (n_images, 1))
+    t_len = parent.shape[1]
+    k = t_len - n_forced
+    n_rows = n_images * n_cfg
+    kv_rows = kv_rows or n_rows
+    w = gen.make_weights(ms, seed)
+    kv_k, kv_v = gen.make_kv_cache(ms, seed, kv_rows)
+    fills = np.asarray(fills, dtype=np.int32)
+    cache_len = np.array([fills[r % n_images] for r in range(n_rows)], dtype=np.int32)
+    lo, hi = ms.vocab_offset, ms.vocab_offset + ms.vocab
+    block = np.zeros((n_images, t_len), dtype=np.int32)
+    block[:, :n_forced] = gen.random_tokens(seed, "forced", (n_images, n_forced), lo, hi)
+    q = np.zeros((n_images, k, ms.vocab), dtype=np.float32)
+    for b in range(n_images):
+        for pn in range(n_forced - 1, t_len):
+            kids = [c for c in range(n_forced, t_len) if parent[b, c] == pn]
+            if not kids:
+                continue
+            path = O.tree_ancestors(parent[b], pn)
+            ls = []
+            for c in range(n_cfg):
+                r = c * n_images + b
+                h = O.target_forward(ms, w, block[b][path], O.widen(kv_k[:, r]), O.widen(kv_v[:, r]),
+                                     int(cache_len[r]))
+                ls.append(O.lm_head_logits(ms, w, h[-1:])[0])
+            l = O.guided_logits(ls[0], ls[1] if n_cfg == 2 else None, cfg_scale) / temperature
+            q_row, _ = gen.perturbed_draft_row(seed, f"tdraft.{b}.{pn}", l, q_noise)
+            for c in kids:
+                q[b, c - n_forced] = q_row
+                tok = gen.sample_rows(q_row[None, :], gen.rng_for(seed, f"tchild.{b}.{c}").random(1))[0]
+                block[b, c] = lo + int(tok)
+    u = philox.verify_uniforms(seed, call_id, n_images, k)
+    return dict(ms=ms, w=w, kv_k=kv_k, kv_v=kv_v, kv_rows=kv_rows, cache_len=cache_len, block=block,
+                parent=parent, draft_probs=q, uniforms=u, n_images=n_images, n_cfg=n_cfg,
+                n_forced=n_forced, n_draft_max=k, cfg_scale=cfg_scale, temperature=temperature)
+
+
+def run_tree_oracle(case) -> dict:
+    c = case
+    n_rows = c["n_images"] * c["n_cfg"]
+    return O.tree_verify(c["ms"], c["w"], c["block"], c["parent"], c["n_forced"], c["kv_k"][:, :n_rows],
+                         c["kv_v"][:, :n_rows], c["cache_len"], c["draft_probs"], c["uniforms"],
+                         c["n_cfg"], c["cfg_scale"], c["temperature"])
+
+
+def run_tree_gpu(runner: "GpuRunner", case) -> dict:
+    import torch
+    vb, c, ms = runner.vb, case, runner.ms
+    b, cfg, k, f = c["n_images"], c["n_cfg"], c["n_draft_max"], c["n_forced"]
+    r, t_len = b * cfg, f + k
+    kv_k, kv_v = to_dev(c["kv_k"]), to_dev(c["kv_v"])
+    o = dict(accept_len=torch.full((b,), -7, dtype=torch.int32, device="cuda"),
+             next_token=torch.full((b,), -7, dtype=torch.int32, device="cuda"),
+             new_len=torch.full((r,), -7, dtype=torch.int32, device="cuda"),
+             n_commit=torch.full((r,), -7, dtype=torch.int32, device="cuda"),
+             accept_mask=torch.full((b, max(k, 1)), 9, dtype=torch.uint8, device="cuda"),
+             accept_path=torch.full((b, max(k, 1)), -7, dtype=torch.int32, device="cuda"),
+             margins=torch.zeros((b, k + 1), dtype=torch.float32, device="cuda"),
+             target_probs=torch.zeros((b, t_len, ms.vocab), dtype=torch.float32, device="cuda"),
+             hidden=torch.zeros((r, t_len, ms.d_model), dtype=torch.bfloat16, device="cuda"))
+    vb.vvs_verify(runner.ctx, n_images=b, n_cfg=cfg, n_forced=f, n_draft_max=k, block=to_dev(c["block"]),
+                  kv_k=kv_k, kv_v=kv_v, kv_rows=c["kv_rows"], cache_len=to_dev(c["cache_len"]),
+                  draft_probs=to_dev(c["draft_probs"]), uniforms=to_dev(c["uniforms"]),
+                  cfg_scale=c["cfg_scale"], temperature=c["temperature"], tree_parent=to_dev(c["parent"]), **o)
+    res = {k_: to_host(v) for k_, v in o.items()}
+    res["status"] = vb.vvs_device_status(runner.ctx)
+    res["launches"] = vb.vvs_last_launch_count(runner.ctx)
+    res["kv_k"], res["kv_v"] = to_host(kv_k), to_host(kv_v)
+    return res
