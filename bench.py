@@ -640,13 +640,96 @@ def run_generation_loop(args) -> None:
                       "device_status": status, "runs": results}))
 
 
+def run_tree_step(args) -> None:
+    """Workload 6: tree calls of the verify step on the configs[1] network (one image with
+    guidance, K = 8 nodes: a binary split at the root and below its first child, chains below),
+    beside the chain call of the same size.  Drafter rows are target-independent (the cost does
+    not depend on them); siblings are independent draws from one row."""
+    import torch
+    from paper_2511_13587_b200 import binding as vb
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    wl = CONFIGS[1]
+    ms = wl.shape
+    b, cfg, k, f = 1, 2, 8, 1
+    r, t_len = b * cfg, f + k
+    parent = np.array([[-1, 0, 0, 1, 1, 2, 3, 4, 6]], dtype=np.int32)
+
+    def dev(a):
+        a = np.ascontiguousarray(a)
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        return torch.from_numpy(a).cuda()
+
+    hw = gen.make_weights(ms, wl.seed)
+    wd = {n: dev(v) for n, v in hw.items() if n != "layers"}
+    wd["layers"] = [{n: dev(v) for n, v in hw["layers"][l].items()} for l in range(ms.n_layers)]
+    del hw
+    g = torch.Generator(device="cuda").manual_seed(wl.seed)
+    kv_k = torch.randn((ms.n_layers, r, ms.n_heads, ms.s_max, ms.head_dim), generator=g,
+                       device="cuda").to(torch.bfloat16)
+    kv_v = torch.randn_like(kv_k)
+    ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, 1))
+    vb.vvs_bind_weights(ctx, wd)
+    trials = []
+    for t in range(N_TRIALS):
+        h = host_trial(wl, t)
+        q = h["draft_probs"]
+        for c in range(f, t_len):                     # siblings share the drafter row of their parent
+            first = min(x for x in range(f, t_len) if parent[0, x] == parent[0, c])
+            q[:, c - f] = q[:, first - f]
+            u = gen.rng_for(wl.seed, f"tree.{t}.{c}").random(1)
+            h["block"][:, c] = ms.vocab_offset + gen.sample_rows(q[:, c - f], u)
+        trials.append({n: dev(h[n]) for n in ("cache_len", "block", "draft_probs", "uniforms")})
+    out = dict(accept_len=torch.zeros(b, dtype=torch.int32, device="cuda"),
+               next_token=torch.zeros(b, dtype=torch.int32, device="cuda"),
+               new_len=torch.zeros(r, dtype=torch.int32, device="cuda"),
+               n_commit=torch.zeros(r, dtype=torch.int32, device="cuda"),
+               target_probs=torch.zeros((b, t_len, ms.vocab), dtype=torch.float32, device="cuda"))
+    path = torch.zeros((b, k), dtype=torch.int32, device="cuda")
+    parent_d = dev(parent)
+
+    def step(inp, tree):
+        extra = dict(tree_parent=parent_d, accept_path=path) if tree else {}
+        vb.vvs_verify(ctx, n_images=b, n_cfg=cfg, n_forced=f, n_draft_max=k, block=inp["block"], kv_k=kv_k,
+                      kv_v=kv_v, kv_rows=r, cache_len=inp["cache_len"], draft_probs=inp["draft_probs"],
+                      uniforms=inp["uniforms"], cfg_scale=wl.cfg_scale, temperature=wl.temperature, **out, **extra)
+
+    res = {}
+    for name, tree in (("chain", False), ("tree", True)):
+        for i in range(max(args.warmup, 3)):
+            step(trials[i % N_TRIALS], tree)
+        torch.cuda.synchronize()
+        acc = 0
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            step(trials[i % N_TRIALS], tree)
+        e1.record()
+        torch.cuda.synchronize()
+        for i in range(min(args.steps, N_TRIALS)):     # acceptance statistics, untimed
+            step(trials[i], tree)
+            acc += int(out["accept_len"].sum().item())
+        msps = e0.elapsed_time(e1) / args.steps
+        res[name] = {"ms_per_step": round(msps, 4), "drafts_per_s": round(b * k / msps * 1e3, 1),
+                     "mean_accept_len": round(acc / min(args.steps, N_TRIALS), 3),
+                     "launches_per_step": vb.vvs_last_launch_count(ctx)}
+    status = vb.vvs_device_status(ctx)
+    print(json.dumps({"metric": "verify step on a candidate tree vs a chain, LlamaGen-XL shape, batch 1 with guidance, 8 drafted nodes",
+                      "unit": "drafted tokens verified per second", "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "configs[1] network, tree parents " + str(parent[0].tolist()),
+                                 "l2": "weights (1.48 GB) exceed L2", "probabilities_written": True},
+                      "device_status": status, "runs": res}))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3, 4, 5, 6])
     ap.add_argument("--cpu-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -654,6 +737,8 @@ def main() -> None:
         run_epilogue_sweep(args)
     elif args.workload == 5:
         run_generation_loop(args)
+    elif args.workload == 6:
+        run_tree_step(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

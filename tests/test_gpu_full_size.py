@@ -63,3 +63,18 @@ def test_config2_batch16_relaxed_two_layers():
     ora = H.run_oracle(case)
     _check_end_to_end(case, gpu, ora)
     run.close()
+
+
+def test_config1_full_shape_candidate_tree():
+    """The configs[1] network at full depth on a candidate tree (two siblings below the root, a
+    three-way split, chains): features, probabilities, walk and compacted cache rows."""
+    from test_gpu_tree import TREE_A, _check_tree
+    wl, fill = CONFIGS[1], 477
+    case = H.build_tree_case(wl.shape, wl.seed + 1, 1, 2, 1, TREE_A, [fill], cfg_scale=wl.cfg_scale, q_noise=0.3)
+    run = H.GpuRunner(wl.shape, case["w"], 2, 9)
+    gpu = H.run_tree_gpu(run, case)
+    assert gpu["launches"] < 40
+    ora = H.run_tree_oracle(case)
+    _check_tree(case, gpu, ora)
+    print("configs[1] tree: accept path", gpu["accept_path"][0][:gpu["accept_len"][0]], "oracle", ora["accept_path"])
+    run.close()
