@@ -223,7 +223,7 @@ def run_ours(args) -> None:
     fetch_pos = torch.zeros((r, 5), dtype=torch.int32, device="cuda")
     launches = [0]
 
-    def step(inp):
+    def step(inp, out=out):
         vb.vvs_verify(ctx, n_images=b, n_cfg=cfg, n_forced=f, n_draft_max=k, block=inp["block"],
                       n_draft=inp["n_draft"], kv_k=kv_k, kv_v=kv_v, kv_rows=r, cache_len=inp["cache_len"],
                       draft_probs=inp["draft_probs"], uniforms=inp["uniforms"], cfg_scale=wl.cfg_scale,
@@ -258,19 +258,36 @@ def run_ours(args) -> None:
     drafts_per_step = float(np.mean([trials[i % N_TRIALS]["n_draft"].sum() for i in range(args.steps)]))
 
     # ---- end to end: host buffers in, host results out, every step ------------------------------
-    pin = [{n: torch.from_numpy(np.ascontiguousarray(t[n])).pin_memory() for n in keys} for t in trials[:8]]
-    stage = {n: torch.empty_like(dtr[0][n]) for n in keys}
-    res_host = {n: torch.empty(out[n].shape, dtype=out[n].dtype).pin_memory()
-                for n in ("accept_len", "next_token", "new_len")}
-    h2d = sum(v.numel() * v.element_size() for v in pin[0].values())
-    d2h = sum(v.numel() * v.element_size() for v in res_host.values())
+    # The step's inputs sit in ONE pinned host buffer and its results come back in one: a call
+    # costs one host->device and one device->host copy whatever the number of arguments.
+    def packed(shapes, pinned):
+        off, views = 0, {}
+        for n, (shape, dtype) in shapes.items():
+            views[n] = (off, int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size(), shape, dtype)
+            off = (off + views[n][1] + 15) & ~15
+        buf = torch.empty(off, dtype=torch.uint8).pin_memory() if pinned else torch.empty(off, dtype=torch.uint8, device="cuda")
+        return buf, {n: buf[o:o + nb].view(dt).view(shape) for n, (o, nb, shape, dt) in views.items()}
+
+    in_shapes = {n: (tuple(dtr[0][n].shape), dtr[0][n].dtype) for n in keys}
+    res_names = ("accept_len", "next_token", "new_len")
+    out_shapes = {n: (tuple(out[n].shape), out[n].dtype) for n in res_names}
+    pin = []
+    for t in trials[:8]:
+        buf, views = packed(in_shapes, True)
+        for n in keys:
+            views[n].copy_(torch.from_numpy(np.ascontiguousarray(t[n])))
+        pin.append(buf)
+    stage_buf, stage = packed(in_shapes, False)
+    res_dev_buf, res_dev = packed(out_shapes, False)
+    res_host_buf, res_host = packed(out_shapes, True)
+    out_e2e = dict(out, **res_dev)
+    h2d = stage_buf.numel()
+    d2h = res_host_buf.numel()
 
     def step_e2e(i):
-        for n in keys:
-            stage[n].copy_(pin[i % len(pin)][n], non_blocking=True)
-        step(stage)
-        for n, h in res_host.items():
-            h.copy_(out[n], non_blocking=True)
+        stage_buf.copy_(pin[i % len(pin)], non_blocking=True)
+        step(stage, out_e2e)
+        res_host_buf.copy_(res_dev_buf, non_blocking=True)
         torch.cuda.current_stream().synchronize()
 
     for i in range(3):

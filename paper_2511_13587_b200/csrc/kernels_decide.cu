@@ -188,7 +188,7 @@ void launch_probs_from_logits(const float* logits, const Workspace& ws, float* p
   probs_kernel<<<grid, 256, 0, s>>>(logits, ws.stat_m, ws.stat_inv, probs, v);
 }
 
-// generic path: target probabilities of the row each image samples from
+// target probabilities of the row each image samples from, out of stored guided logits
 __global__ void select_p_row_kernel(const float* __restrict__ logits, Workspace ws, int v) {
   int b = blockIdx.y;
   int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -199,9 +199,9 @@ __global__ void select_p_row_kernel(const float* __restrict__ logits, Workspace 
   ws.p_row[(size_t)b * v + j] = pr;
 }
 
-void launch_select_p_row(const Workspace& ws, int n_images, int v, cudaStream_t s) {
+void launch_select_p_row(const float* logits, const Workspace& ws, int n_images, int v, cudaStream_t s) {
   dim3 grid((v + 255) / 256, n_images);
-  select_p_row_kernel<<<grid, 256, 0, s>>>(ws.logits, ws, v);
+  select_p_row_kernel<<<grid, 256, 0, s>>>(logits, ws, v);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -47,9 +47,6 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
       const size_t wide = 3 * dm > 2 * ff ? 3 * dm : 2 * ff;
       const size_t tiles = (wide + 127) / 128, passes = (M + 255) / 256;
       c.take(ws.slot_pos, M * 4);
-      c.take(ws.anc_mask, M * 4);
-      c.take(ws.tree_res, (size_t)2 * (d.max_rows < 32 ? d.max_rows : 32) * V * 8);
-      c.take(ws.tree_path, (size_t)32 * 32 * 4);
       c.take(ws.rope_cos, M * (size_t)(d.head_dim / 2) * 4);
       c.take(ws.rope_sin, M * (size_t)(d.head_dim / 2) * 4);
       c.take(ws.sk_scratch, M * wide * 4);
@@ -71,6 +68,7 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
     c.take(ws.logits, M * V * 4);
   } else {
     c.take(ws.sel_hid, (size_t)d.max_rows * dm * es);
+
   }
   c.take(ws.part_m, n_tiles * M * 4);
   c.take(ws.part_s, n_tiles * M * 4);
@@ -83,6 +81,12 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
   c.take(ws.p_row, (size_t)d.max_rows * V * 4);
   c.take(ws.r_part, (size_t)d.max_rows * n_chunks * 8);
   c.take(ws.p_part, (size_t)d.max_rows * n_chunks * 8);
+  if (d.dtype == VVS_DTYPE_BF16 && d.n_layers > 0) {
+    c.take(ws.anc_mask, M * 4);
+    c.take(ws.tree_res, (size_t)2 * (d.max_rows < 32 ? d.max_rows : 32) * V * 8);
+    c.take(ws.tree_path, (size_t)32 * 32 * 4);
+  }
+  if (d.dtype == VVS_DTYPE_BF16 && !std::getenv("VVS_DEBUG_GENERIC")) c.take(ws.logits_small, (M < 64 ? M : 64) * V * 4);
   return (c.off + 255) & ~size_t(255);
 }
 
@@ -170,7 +174,10 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
     LmHeadArgs la{};
     la.v = V; la.k = md.d_model; la.bt = BT; la.n_cfg = C; la.tm_a = &ctx->lm_map; la.tm_b = &tm_hid;
     la.pdl = ctx->use_pdl; la.cfg_scale = a->cfg_scale; la.inv_temp = 1.f / a->temperature;
-    la.part_m = ws.part_m; la.part_s = ws.part_s; la.logits_out = o->target_probs; la.status = ws.status;
+    // few decision rows: the guided logits are written out (under a megabyte at 9 rows) and the
+    // sampled row is read back from them; otherwise a second pass over the head recomputes it
+    float* lbuf = o->target_probs ? o->target_probs : (BT <= 64 ? ws.logits_small : nullptr);
+    la.part_m = ws.part_m; la.part_s = ws.part_s; la.logits_out = lbuf; la.status = ws.status;
     la.rows_per_seq = rows_per_seq; la.first_row = first_row; la.n_draft_max = p.n_draft_max;
     la.vocab_offset = md.vocab_offset; la.relaxed = (p.mode == VVS_MODE_RELAXED && p.nbr_k > 1) ? 1 : 0;
     la.nbr_k = p.nbr_k; la.kmax = p.kmax; la.drafts_ld = drafts_ld; la.drafts = drafts;
@@ -180,8 +187,14 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
     if (rc != VVS_OK) return rc;
     VVS_LAUNCH(VVS_PROF_OTHER, launch_finalize_stats(ws, (V + 127) / 128, BT, s));
     VVS_LAUNCH(VVS_PROF_OTHER, launch_accept(ws, p, s));
-    if (o->target_probs)
-      VVS_LAUNCH(VVS_PROF_OTHER, launch_probs_from_logits(o->target_probs, ws, o->target_probs, BT, V, s));
+    if (lbuf) {
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_select_p_row(lbuf, ws, B, V, s));
+      if (o->target_probs)
+        VVS_LAUNCH(VVS_PROF_OTHER, launch_probs_from_logits(o->target_probs, ws, o->target_probs, BT, V, s));
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_residual_mass(ws, p, s));
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_sample(ws, p, s));
+      return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+    }
     VVS_LAUNCH(VVS_PROF_OTHER, launch_gather_sel_rows(hid, ws.sel_row, ws.sel_hid, B, C, BT, md.d_model, s));
     LmHeadArgs lr{};
     lr.v = V; lr.k = md.d_model; lr.bt = B; lr.n_cfg = C; lr.tm_a = &ctx->lm_map; lr.tm_b = &tm_sel;
@@ -202,7 +215,7 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
   VVS_LAUNCH(VVS_PROF_OTHER, launch_accept(ws, p, s));
   if (o->target_probs)
     VVS_LAUNCH(VVS_PROF_OTHER, launch_probs_from_logits(ws.logits, ws, o->target_probs, BT, V, s));
-  VVS_LAUNCH(VVS_PROF_OTHER, launch_select_p_row(ws, B, V, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_select_p_row(ws.logits, ws, B, V, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_residual_mass(ws, p, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_sample(ws, p, s));
   return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;

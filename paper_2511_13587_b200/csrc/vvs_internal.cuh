@@ -40,6 +40,7 @@ struct Workspace {
   int32_t* sel_row = nullptr;   // [B] decision row (b*T + t) the next token is sampled from, -1 none
   int32_t* sel_kind = nullptr;  // [B] 0 = residual of draft n, 1 = bonus
   float* p_row = nullptr;    // [B, V] target probabilities of the selected row
+  float* logits_small = nullptr; // [min(M, 64), V] guided logits of calls with few decision rows (tensor-core path)
   void* sel_hid = nullptr;   // [n_cfg * B, d] features of the selected rows (tensor-core LM head, row mode)
   double* r_part = nullptr;  // [B, n_chunks] per-chunk residual mass
   double* p_part = nullptr;  // [B, n_chunks] per-chunk target mass (fallback when residual is 0)
@@ -283,7 +284,7 @@ void launch_gather_logits(const float* logits, const Workspace& ws, const Decide
 void launch_accept(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_probs_from_logits(const float* logits, const Workspace& ws, float* probs, int n_rows,
                               int v, cudaStream_t s);
-void launch_select_p_row(const Workspace& ws, int n_images, int v, cudaStream_t s);
+void launch_select_p_row(const float* logits, const Workspace& ws, int n_images, int v, cudaStream_t s);
 void launch_residual_mass(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_sample(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 
