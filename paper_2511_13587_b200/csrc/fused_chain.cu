@@ -537,6 +537,23 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
       for (int j = 0; j < NC; ++j) tma_load_2d(sK + j * kSlabBytes, &tm_k, &att_kv_full, j * 64, row);
       for (int j = 0; j < NC; ++j) tma_load_2d(sV + j * kSlabBytes, &tm_v, &att_kv_full, j * 64, row);
     };
+    // A CTA's second item of a layer: its K tile is requested as soon as the first item's score MMA
+    // has read the staging buffer, its V tile once the output MMA has; the K request only raises
+    // the byte count of the barrier's next phase, the V request also arrives on it.
+    auto issue_next_k = [&](int layer, int item) {   // one thread
+      int r, h, c;
+      decode_item(item, r, h, c);
+      const int row = kv_row_base(layer, r, h, c);
+      mbar_expect_tx_only(&att_kv_full, (uint32_t)(NC * kSlabBytes));
+      for (int j = 0; j < NC; ++j) tma_load_2d(sK + j * kSlabBytes, &tm_k, &att_kv_full, j * 64, row);
+    };
+    auto issue_next_v = [&](int layer, int item) {   // one thread
+      int r, h, c;
+      decode_item(item, r, h, c);
+      const int row = kv_row_base(layer, r, h, c);
+      mbar_expect_tx(&att_kv_full, (uint32_t)(NC * kSlabBytes));
+      for (int j = 0; j < NC; ++j) tma_load_2d(sV + j * kSlabBytes, &tm_v, &att_kv_full, j * 64, row);
+    };
 
     // ---- phase 0: clear the accumulators, gather the embeddings ----
     {
@@ -590,7 +607,6 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             const int row_base = kv_row_base(l, r, h, c);
             const int per_head = p.hd >> 3;
             if (!grp_e) {
-              if (tid_g == 0 && n_mine > 0) issue_kv(l, i);   // the first item was requested a layer ahead
               // Q operand: q * (1/rms) rotated, bf16, K-major with the 128-byte swizzle
 #pragma unroll 1
               for (int idx = tid_g; idx < T * per_head; idx += kGroup) {
@@ -644,6 +660,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               // scores: this thread owns key (quarter * 32 + lane) of the chunk
               wait_bar(&att_s_full, par, &s_abort, p.status);
               tc_fence_after();
+              if (tid_g == 0 && i + G < n_items && !s_abort) issue_next_k(l, i + G);
               if (tid_g == 0) VVS_TRACE(0x4F2);
               const int kl = quarter * 32 + lane;
               const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + kColS;
@@ -727,6 +744,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             }
             wait_bar(&att_o_full, par, &s_abort, p.status);
             tc_fence_after();
+            if (tid_w == 0 && i + G < n_items && !s_abort) issue_next_v(l, i + G);
             if (tid_w == 0) VVS_TRACE(0x4F4);
             if (grp_e && quarter == 0) {                  // TMEM lanes 0..31 = query rows
               const size_t rh = (size_t)r * H + h;
