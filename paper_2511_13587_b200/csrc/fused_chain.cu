@@ -507,14 +507,26 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
     unsigned target = epoch;
     uint32_t it_slab = 0, ita = 0, iatt = 0;         // ring position at the start of the phase, items, att items
 
-    auto grid_sync = [&]() {
+    // Plan of the projection that follows the next grid barrier (its share of units): worked out
+    // between the arrival at the barrier and the first poll, where its integer divisions cost
+    // nothing, instead of after the release, where they sat on every phase's critical path.
+    Phase f = phase_of(p, PH_QKV);
+    int lo = 0, hi = 0;
+    auto grid_sync = [&](int next_l, int next_ph) {
       if (tid_w == 0) VVS_TRACE(0x900);
       named_bar_sync(BAR_W, kWorkers);
       target += (unsigned)G;
       if (tid_w == 0) VVS_TRACE(0x901);
-      if (tid_w == 0 && !s_abort) {
+      const bool poll = tid_w == 0 && !s_abort;
+      if (poll) {
         __threadfence();
         atomicAdd(p.sync_words, 1u);
+      }
+      if (next_ph >= 0) {
+        f = phase_of(p, next_ph);
+        unit_range(f, next_l, next_ph, lo, hi);
+      }
+      if (poll) {
         bool ok = false;
         for (uint32_t i = 0; i < kGridSpinLimit; ++i) {
           if ((int)(ld_acquire_gpu(p.sync_words) - target) >= 0) { ok = true; break; }
@@ -581,7 +593,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
         dst[1] = make_float4(v[4], v[5], v[6], v[7]);
       }
       if (!grp_e && tid_g == 0 && (int)blockIdx.x < n_items) issue_kv(0, blockIdx.x);
-      grid_sync();
+      grid_sync(0, PH_QKV);
     }
 
     // per-thread constants of the merge builders (128 threads per unit: token, 16 columns)
@@ -593,6 +605,13 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
       const int par_l = l & 1;
       float* qkv = p.qkv_acc + (size_t)par_l * p.m * 3 * p.d;
       float* gu = p.gu_acc + (size_t)par_l * p.m * 2 * p.ff;
+      // The norm scales of a layer are first touched by its builders, right after a grid barrier:
+      // a miss to HBM there sits on the critical path, so the next layer's are pulled into L2 now.
+      if (l + 1 < L && tid_w < 2 * ((p.d + 63) >> 6)) {
+        const int which = tid_w & 1, line = tid_w >> 1;
+        const __nv_bfloat16* nx = p.norms[(l + 1) * 2 + which] + line * 64;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(nx));
+      }
 #pragma unroll 1
       for (int ph = 0; ph < 4; ++ph) {
         if (ph == PH_O) {
@@ -769,13 +788,11 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             named_bar_sync(BAR_W, kWorkers);
           }
           if (!grp_e && tid_g == 0 && l + 1 < L && (int)blockIdx.x < n_items) issue_kv(l + 1, blockIdx.x);
-          grid_sync();
+          grid_sync(l, PH_O);
         }
 
         // ================================ projection phase ==========================================
-        const Phase f = phase_of(p, ph);
-        int lo, hi;
-        unit_range(f, l, ph, lo, hi);
+        // (f, lo, hi were set inside the grid barrier that precedes this phase)
         const int n_units = hi - lo;
         const uint32_t per_unit = 1u + (uint32_t)f.dual;
 
@@ -953,7 +970,12 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             ++ita;
           }
         }
-        if (!(l == L - 1 && ph == PH_DOWN)) grid_sync();
+        // what follows: the attention items (no projection plan), or the next projection
+        if (!(l == L - 1 && ph == PH_DOWN)) {
+          if (ph == PH_QKV) grid_sync(l, -1);
+          else if (ph == PH_DOWN) grid_sync(l + 1, PH_QKV);
+          else grid_sync(l, ph + 1);
+        }
       }
     }
     if (blockIdx.x == 0 && tid_w == 0 && !s_abort)
