@@ -49,7 +49,6 @@ __global__ void __launch_bounds__(kTreeThreads) tree_walk_kernel(TreeParams p) {
   __shared__ double s_warp[kTreeThreads / 32];
   __shared__ int s_child[32];
   __shared__ int s_n, s_pass, s_first, s_last;
-  __shared__ double s_t;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int F = p.n_forced, K = p.n_draft_max, T = p.t_len, V = p.vocab;
   const int32_t* par = p.parent + (size_t)b * T;

@@ -165,8 +165,7 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
 
 
   if (ctx->tensor_core_path) {
-    // LM head with guidance, softmax partials and gathers fused into its epilogue; the one row
-    // per image that sampling needs comes from a second pass over the selected rows
+    // LM head with guidance, softmax partials and gathers fused into its epilogue
     CUtensorMap tm_hid, tm_sel;
     if (make_tmap_bf16_2d(&tm_hid, hid, (uint64_t)M, (uint64_t)md.d_model, (uint32_t)lmhead_box_rows(BT)) != VVS_OK ||
         make_tmap_bf16_2d(&tm_sel, ws.sel_hid, (uint64_t)R, (uint64_t)md.d_model, (uint32_t)lmhead_box_rows(B)) != VVS_OK)
