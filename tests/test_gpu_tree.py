@@ -165,3 +165,25 @@ def test_tree_argument_errors():
     with pytest.raises(vb.VvsError):
         vb.vvs_verify(run.ctx, mode=MODE_RELAXED, nbr_k=1, target_probs=probs, **common)
     run.close()
+
+
+@pytest.mark.parametrize("name,seed,parent,n_forced,n_cfg,q_noise",
+                         [("seven siblings, all rejected", 407, [-1, 0, 0, 0, 0, 0, 0, 0], 1, 2, 3.0),
+                          ("seven siblings, the last accepted", 400, [-1, 0, 0, 0, 0, 0, 0, 0], 1, 2, 3.0),
+                          ("chain ending in three leaves", 308, [-1, 0, 1, 2, 3, 4, 4, 4], 1, 2, 0.3),
+                          ("17 block rows, no guidance", 317, [-1, 0, 1, 2, 2, 3, 3, 4, 4, 5, 6, 7, 8, 9, 10, 11, 12], 3, 1, 1.0),
+                          ("forced rows only", 303, [-1, 0, 1], 3, 2, 1.0)])
+def test_tree_shapes(name, seed, parent, n_forced, n_cfg, q_noise):
+    """Wide, deep, long and degenerate trees.  A drafter far from the target (noise 3.0) makes
+    siblings fail one after the other, so the walk goes through one residual update per rejected
+    sibling (the float64 rounds) before it accepts or samples; a tree without draft nodes samples
+    from the last forced row."""
+    ms = XL_SMALL
+    case = H.build_tree_case(ms, seed, 1, n_cfg, n_forced, parent, [77], q_noise=q_noise)
+    run = H.GpuRunner(ms, case["w"], n_cfg, len(parent))
+    gpu = H.run_tree_gpu(run, case)
+    ora = H.run_tree_oracle(case)
+    assert _check_tree(case, gpu, ora) == 0
+    np.testing.assert_array_equal(gpu["accept_len"], ora["accept_len"])
+    print(name, "accepted", gpu["accept_path"][0][:gpu["accept_len"][0]], "oracle", ora["accept_path"][0])
+    run.close()
