@@ -202,9 +202,10 @@ __device__ __forceinline__ bool wait_fast(uint64_t* bar, uint32_t parity, volati
 }
 
 // One round of token-operand building by the 256 worker threads: nb <= (1 << lg) units,
-// 256 >> lg threads per unit.  A unit's slab is m rows x 16 positions of 4 columns; thread j of
-// the unit takes positions j, j + tpu, ... so that consecutive lanes read consecutive 16 bytes
-// and every load of the round is in flight before the first use (MAXI = positions per thread).
+// 256 >> lg threads per unit.  A unit's slab is m rows x 8 groups of 8 columns (one 16-byte
+// swizzle chunk each); thread j of the unit takes group j & 7 of rows (j >> 3) + k * (tpu >> 3),
+// so eight consecutive lanes read one row's 256 contiguous bytes and every load of the round is
+// in flight before the first use (MAXI = rows per thread; 32 rows need MAXI = 1 << lg).
 //   DOWN == false: slab = bf16(x * norm scale); the CTAs that own tile 0 also add the row sums
 //                  of squares into ss_out
 //   DOWN == true : slab = bf16(silu(gate / rms) * (up / rms)), rms from ss_in
@@ -220,68 +221,66 @@ __device__ __noinline__ void build_round(const ChainParams& p, uint8_t* ring, ui
   if (use > 0) wait_fast(&empty[st], (use - 1) & 1, s_abort, p.status);
   const int s = s0 + u, tile = s / kbs, kb = s - tile * kbs;
   const int m = p.m, ff = p.ff;
-  const int q = j & 15, row0 = j >> 4, rstep = tpu >> 4;  // this thread: column group q, rows row0 + k * rstep
-  const int col = kb * 64 + q * 4;
+  const int q = j & 7, row0 = j >> 3, rstep = tpu >> 3;
+  const int col = kb * 64 + q * 8;
   const int ld = DOWN ? 2 * ff : p.d;
   const float* sp = src + (size_t)row0 * ld + col;
   const size_t sstep = (size_t)rstep * ld;
   const bool col_ok = !DOWN || col < ff;
-  float4 a[MAXI];
-  float4 b[DOWN ? MAXI : 1];
+  const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 a0[MAXI], a1[MAXI];
+  float4 b0[DOWN ? MAXI : 1], b1[DOWN ? MAXI : 1];
   float sv[DOWN ? MAXI : 1];
-  uint2 g = make_uint2(0u, 0u);
-  if (!DOWN) g = __ldg(reinterpret_cast<const uint2*>(gsc + col));
+  uint4 g = make_uint4(0u, 0u, 0u, 0u);
+  if (!DOWN) g = __ldg(reinterpret_cast<const uint4*>(gsc + col));
 #pragma unroll
   for (int k = 0; k < MAXI; ++k) {
-    a[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (DOWN) { b[k] = a[k]; sv[k] = 1.f; }
+    a0[k] = z4;
+    a1[k] = z4;
+    if (DOWN) { b0[k] = z4; b1[k] = z4; sv[k] = 1.f; }
     if (row0 + k * rstep < m) {
       if (col_ok) {
-        a[k] = __ldcg(reinterpret_cast<const float4*>(sp));
-        if (DOWN) b[k] = __ldcg(reinterpret_cast<const float4*>(sp + ff));
+        a0[k] = __ldcg(reinterpret_cast<const float4*>(sp));
+        a1[k] = __ldcg(reinterpret_cast<const float4*>(sp) + 1);
+        if (DOWN) {
+          b0[k] = __ldcg(reinterpret_cast<const float4*>(sp + ff));
+          b1[k] = __ldcg(reinterpret_cast<const float4*>(sp + ff) + 1);
+        }
       }
       if (DOWN) sv[k] = __ldcg(ss_in + row0 + k * rstep);
     }
     sp += sstep;
   }
-  float gv[4] = {1.f, 1.f, 1.f, 1.f};
-  if (!DOWN) {
-    const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g.x));
-    const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g.y));
-    gv[0] = g01.x; gv[1] = g01.y; gv[2] = g23.x; gv[3] = g23.y;
-  }
+  float gv[8];
+  unpack8(g, gv);
   const float inv_d = 1.f / (float)p.d, eps = p.eps;
-  uint8_t* out = ring + (size_t)st * kStageBytes + kSlabBytes + row0 * 128 + ((q & 1) << 3);
-  int row = row0;
+  uint8_t* out = ring + (size_t)st * kStageBytes + kSlabBytes;
 #pragma unroll
   for (int k = 0; k < MAXI; ++k) {
-    float v[4] = {a[k].x, a[k].y, a[k].z, a[k].w};
+    const int row = row0 + k * rstep;
+    float v[8] = {a0[k].x, a0[k].y, a0[k].z, a0[k].w, a1[k].x, a1[k].y, a1[k].z, a1[k].w};
     if (DOWN) {
       const float rinv = rsqrtf(fmaf(sv[k], inv_d, eps));
-      const float w[4] = {b[k].x, b[k].y, b[k].z, b[k].w};
+      const float w[8] = {b0[k].x, b0[k].y, b0[k].z, b0[k].w, b1[k].x, b1[k].y, b1[k].z, b1[k].w};
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
+      for (int e = 0; e < 8; ++e) {
         const float t = v[e] * rinv;
         v[e] = __fdividef(t, 1.f + __expf(-t)) * (w[e] * rinv);
       }
     } else {
       if (tile == 0) {                                   // uniform per warp
-        float ssq = v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
+        float ssq = 0.f;
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, o);   // 16 lanes = one row
+        for (int e = 0; e < 8; ++e) ssq = fmaf(v[e], v[e], ssq);
+        ssq += __shfl_xor_sync(0xffffffffu, ssq, 4);     // 8 lanes = one row
+        ssq += __shfl_xor_sync(0xffffffffu, ssq, 2);
+        ssq += __shfl_xor_sync(0xffffffffu, ssq, 1);
         if (q == 0 && row < m) atomicAdd(ss_out + row, ssq);
       }
 #pragma unroll
-      for (int e = 0; e < 4; ++e) v[e] *= gv[e];
+      for (int e = 0; e < 8; ++e) v[e] *= gv[e];
     }
-    if (row < m) {
-      uint2 o;
-      *reinterpret_cast<__nv_bfloat162*>(&o.x) = __floats2bfloat162_rn(v[0], v[1]);
-      *reinterpret_cast<__nv_bfloat162*>(&o.y) = __floats2bfloat162_rn(v[2], v[3]);
-      *reinterpret_cast<uint2*>(out + ((((q >> 1) ^ row) & 7) << 4)) = o;
-    }
-    row += rstep;
-    out += rstep * 128;
+    if (row < m) *reinterpret_cast<uint4*>(out + row * 128 + ((q ^ (row & 7)) << 4)) = pack8(v);
   }
 }
 
@@ -883,13 +882,13 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             const int lg = nb <= 1 ? 0 : nb <= 2 ? 1 : nb <= 4 ? 2 : 3;
             const uint32_t it0 = it_slab + (uint32_t)b0 * per_unit;
             if (ph == PH_DOWN)
-              build_round<8, true>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, gu, nullptr,
+              build_round<4, true>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, gu, nullptr,
                                    p.ss + (2 * l + 1) * 32, nullptr);
             else if (lg == 3)
-              build_round<16, false>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, p.x, gsc,
+              build_round<8, false>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, p.x, gsc,
                                      nullptr, p.ss + (2 * l + which) * 32);
             else
-              build_round<8, false>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, p.x, gsc,
+              build_round<4, false>(p, ring, empty, &s_abort, tid_w, nb, lg, it0, per_unit, lo + b0, f.kbs, p.x, gsc,
                                     nullptr, p.ss + (2 * l + which) * 32);
             fence_proxy_async();
             if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | (b0 & 15));
