@@ -175,23 +175,24 @@ __device__ __forceinline__ void rope8(const ChainParams& p, int tok, int e, floa
 }
 
 // The MMA warp runs its loop with all 32 lanes (so that descriptors and addresses stay warp-uniform
-// values) and one elected lane issues; the election is inside the asm block, the same lane every time.
-__device__ __forceinline__ void mma_elect(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
+// values); the lane elected once at the start of the role issues, as a predicated instruction
+// (an election per instruction cost ~0.2 us per layer, a lone lane running the loop far more).
+__device__ __forceinline__ void mma_pred(uint32_t leader, uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                         uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred pe, pa;\n\t"
-      "elect.sync _|pe, 0xffffffff;\n\t"
+      "setp.ne.b32 pe, %5, 0;\n\t"
       "setp.ne.b32 pa, %4, 0;\n\t"
       "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pa;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
       : "memory");
 }
-__device__ __forceinline__ void commit_elect(uint64_t* bar) {
+__device__ __forceinline__ void commit_pred(uint32_t leader, uint64_t* bar) {
   asm volatile(
       "{\n\t.reg .pred pe;\n\t"
-      "elect.sync _|pe, 0xffffffff;\n\t"
+      "setp.ne.b32 pe, %1, 0;\n\t"
       "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-      ::"r"(smem_u32(bar))
+      ::"r"(smem_u32(bar)), "r"(leader)
       : "memory");
 }
 
@@ -401,6 +402,10 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
     // =================================== MMA issuer ==================================================
     {
       uint32_t st = 0, par = 0, ita = 0, iatt = 0;
+      // one lane is elected once; every MMA and commit below is predicated on it, so the whole
+      // warp runs the loop and its waits without diverging
+      uint32_t leader;
+      asm volatile("{\n\t.reg .pred pe;\n\telect.sync _|pe, 0xffffffff;\n\tselp.u32 %0, 1, 0, pe;\n\t}" : "=r"(leader));
       bool alive = true;
       const uint32_t idesc_gemm = idesc_bf16_f32(128, 32);
       const uint64_t desc0 = smem_desc_sw128(smem_u32(ring));   // + (byte offset >> 4) selects a slab
@@ -422,9 +427,9 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               for (int k16 = 0; k16 < p.hd / 16; ++k16) {
                 const uint32_t a = smem_u32(sK + (k16 >> 2) * kSlabBytes) + (k16 & 3) * 32;
                 const uint32_t b = smem_u32(sQ + (k16 >> 2) * q_chunk_bytes) + (k16 & 3) * 32;
-                mma_elect(tmem_base + kColS, smem_desc_sw128(a), smem_desc_sw128(b), idesc_s, k16 > 0 ? 1u : 0u);
+                mma_pred(leader, tmem_base + kColS, smem_desc_sw128(a), smem_desc_sw128(b), idesc_s, k16 > 0 ? 1u : 0u);
               }
-              commit_elect(&att_s_full);
+              commit_pred(leader, &att_s_full);
               VVS_TRACE_MMA(0x2F2);
               if (!wait_bar(&att_p_ready, apar, &s_abort, p.status)) { alive = false; break; }
               __syncwarp();
@@ -434,10 +439,10 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
               for (int k16 = 0; k16 < 8; ++k16) {
                 const uint32_t a = smem_u32(sP + (k16 >> 2) * kSlabBytes) + (k16 & 3) * 32;
                 const uint32_t b = smem_u32(sV) + k16 * 2048;
-                mma_elect(tmem_base + kColO, smem_desc_sw128(a), smem_desc_mn_sw128(b, kSlabBytes), idesc_o,
+                mma_pred(leader, tmem_base + kColO, smem_desc_sw128(a), smem_desc_mn_sw128(b, kSlabBytes), idesc_o,
                          k16 > 0 ? 1u : 0u);
               }
-              commit_elect(&att_o_full);
+              commit_pred(leader, &att_o_full);
               VVS_TRACE_MMA(0x2F4);
             }
             if (!alive) break;
@@ -451,7 +456,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
           for (int s = lo; s < hi; ++s) {
             const bool first = (s == lo) || (kb == 0);
             if (first) {
-              if (s != lo) commit_elect(&acc_full[slot]);
+              if (s != lo) commit_pred(leader, &acc_full[slot]);
               slot = ita % kAccSlots;
               const uint32_t use = ita / kAccSlots;
               if (use > 0 && !wait_bar(&acc_empty[slot], (use - 1) & 1, &s_abort, p.status)) { alive = false; break; }
@@ -474,26 +479,26 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             tc_fence_after();
             VVS_TRACE_MMA(0x200 | (ph << 4) | ((s - lo) & 15));
             const uint32_t acc = tmem_base + slot * 64;
-            mma_elect(acc, a_desc, b_desc, idesc_gemm, first ? 0u : 1u);
-            mma_elect(acc, a_desc + 2, b_desc + 2, idesc_gemm, 1u);
-            mma_elect(acc, a_desc + 4, b_desc + 4, idesc_gemm, 1u);
-            mma_elect(acc, a_desc + 6, b_desc + 6, idesc_gemm, 1u);
+            mma_pred(leader, acc, a_desc, b_desc, idesc_gemm, first ? 0u : 1u);
+            mma_pred(leader, acc, a_desc + 2, b_desc + 2, idesc_gemm, 1u);
+            mma_pred(leader, acc, a_desc + 4, b_desc + 4, idesc_gemm, 1u);
+            mma_pred(leader, acc, a_desc + 6, b_desc + 6, idesc_gemm, 1u);
             if (f.dual) {
               // the second weight slab multiplies the token slab of the FIRST stage: that stage is
               // released only after these have been issued as well
-              mma_elect(acc + 32, a2_desc, b_desc, idesc_gemm, first ? 0u : 1u);
-              mma_elect(acc + 32, a2_desc + 2, b_desc + 2, idesc_gemm, 1u);
-              mma_elect(acc + 32, a2_desc + 4, b_desc + 4, idesc_gemm, 1u);
-              mma_elect(acc + 32, a2_desc + 6, b_desc + 6, idesc_gemm, 1u);
-              commit_elect(&empty[st_a]);
-              commit_elect(&empty[st_b]);
+              mma_pred(leader, acc + 32, a2_desc, b_desc, idesc_gemm, first ? 0u : 1u);
+              mma_pred(leader, acc + 32, a2_desc + 2, b_desc + 2, idesc_gemm, 1u);
+              mma_pred(leader, acc + 32, a2_desc + 4, b_desc + 4, idesc_gemm, 1u);
+              mma_pred(leader, acc + 32, a2_desc + 6, b_desc + 6, idesc_gemm, 1u);
+              commit_pred(leader, &empty[st_a]);
+              commit_pred(leader, &empty[st_b]);
             } else {
-              commit_elect(&empty[st_a]);
+              commit_pred(leader, &empty[st_a]);
             }
             VVS_TRACE_MMA(0x280 | (ph << 4) | ((s - lo) & 15));
             if (++kb == f.kbs) kb = 0;
           }
-          if (alive && hi > lo) commit_elect(&acc_full[slot]);
+          if (alive && hi > lo) commit_pred(leader, &acc_full[slot]);
         }
       }
     }
