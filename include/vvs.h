@@ -179,8 +179,8 @@ typedef struct vvs_verify_args {
                                u < min(1, p_res(x) / q(x)), a rejection replaces p_res by
                                norm(max(0, p_res - q)); when no child is left the next token is drawn
                                from p_res (from the node's own target row if it is a leaf).  Tree
-                               calls need bf16, at most 32 block tokens, strict mode, n_draft == NULL
-                               and out->target_probs (the walk reads whole target rows). */
+                               calls need a bf16 context, strict mode, n_draft == NULL and
+                               out->target_probs (the walk reads whole target rows). */
 } vvs_verify_args;
 
 /* Outputs, device memory allocated by the caller.  Optional ones may be NULL and are then

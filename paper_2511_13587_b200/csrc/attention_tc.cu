@@ -29,6 +29,7 @@ constexpr int kChunkKeys = 128;
 
 struct AttnParams {
   const int32_t* cache_len;
+  const uint32_t* anc_mask;  // [M] block rows visible to each block row (chain or tree)
   __nv_bfloat16* out;     // [M, d]
   float* part_o;          // [R*H, n_chunks_max, T, hd]
   float* part_ml;         // [R*H, n_chunks_max, T, 2]
@@ -172,16 +173,22 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
       for (int t = 0; t < 32; ++t)
         if (t < p.tq) reinterpret_cast<float*>(sP + (t >> 4) * kKVBytes + 4096)[(t & 15) * 128 + tid] = sc[t];
     }
+    // visibility masks of this sequence's block rows, one per lane (written by the table kernel
+    // at the start of the step, several launches ago)
+    const uint32_t anc_l = lane < T ? p.anc_mask[r * T + lane] : 0u;
     __syncthreads();
     // one warp per query row: mask, max, exp, sum; lane owns keys 4*lane .. 4*lane+3
 #pragma unroll 1
     for (int t = warp; t < T; t += 4) {
+      const uint32_t anc = __shfl_sync(0xffffffffu, anc_l, t);
       const float4 s4 = reinterpret_cast<const float4*>(sP + (t >> 4) * kKVBytes + 4096)[(t & 15) * 32 + lane];
       float sv[4] = {s4.x, s4.y, s4.z, s4.w};
       float mx = -CUDART_INF_F;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        sv[j] = (key0 + 4 * lane + j <= fill + t) ? sv[j] * p.scale : -CUDART_INF_F;
+        const int kj = key0 + 4 * lane + j - fill;   // < 0: cache slot; else block row kj
+        const uint32_t vis = (kj < 0 ? 1u : 0u) | (((uint32_t)kj < 32u ? 1u : 0u) & (anc >> (kj & 31)));
+        sv[j] = (vis & 1u) ? sv[j] * p.scale : -CUDART_INF_F;
         mx = fmaxf(mx, sv[j]);
       }
       mx = warp_max_f(mx);
@@ -305,7 +312,7 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
 
 int launch_attention_tc(const AttentionTcArgs& a, cudaStream_t s) {
   AttnParams p{};
-  p.cache_len = a.cache_len; p.out = a.out; p.part_o = a.part_o; p.part_ml = a.part_ml;
+  p.cache_len = a.cache_len; p.anc_mask = a.anc_mask; p.out = a.out; p.part_o = a.part_o; p.part_ml = a.part_ml;
   p.counters = a.counters; p.status = a.status;
   p.d = a.d; p.n_heads = a.n_heads; p.hd = a.hd; p.s_max = a.s_max; p.layer = a.layer;
   p.kv_rows = a.kv_rows; p.t_len = a.t_len; p.tq = a.t_len <= 16 ? 16 : 32;

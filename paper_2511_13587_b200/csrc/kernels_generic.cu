@@ -163,7 +163,8 @@ __global__ void rope_append_kernel(const float* __restrict__ qkv, const float* _
                                    T* __restrict__ q, T* __restrict__ kv_k, T* __restrict__ kv_v,
                                    const int32_t* __restrict__ cache_len, int d, int n_heads, int hd,
                                    int s_max, int rope_mode, int grid_w, int n_prefix, int layer,
-                                   int kv_rows, int t_len, int32_t* status) {
+                                   int kv_rows, int t_len, int32_t* status,
+                                   const float* __restrict__ tab_cos, const float* __restrict__ tab_sin) {
   int m = blockIdx.x;
   int r = m / t_len, t = m % t_len;
   int fill = cache_len[r];
@@ -182,9 +183,13 @@ __global__ void rope_append_kernel(const float* __restrict__ qkv, const float* _
   int half = hd / 2;
   for (int p = threadIdx.x; p < d / 2; p += blockDim.x) {
     int h = p / half, i = p % half;
-    float ang = ((i < half / 2) ? c_lo : c_hi) * inv_freq[i];
     float sn, cs;
-    sincosf(ang, &sn, &cs);
+    if (tab_cos) {                        // rotation tables of the step (tree calls: position = fill + depth)
+      cs = tab_cos[(size_t)m * half + i];
+      sn = tab_sin[(size_t)m * half + i];
+    } else {
+      sincosf(((i < half / 2) ? c_lo : c_hi) * inv_freq[i], &sn, &cs);
+    }
     int e = h * hd + 2 * i;
     float q0 = src[e], q1 = src[e + 1];
     q[(size_t)m * d + e] = from_f<T>(q0 * cs - q1 * sn);
@@ -203,10 +208,11 @@ __global__ void rope_append_kernel(const float* __restrict__ qkv, const float* _
 template <typename T>
 void launch_rope_append(const float* qkv, const float* inv_freq, T* q, T* kv_k, T* kv_v,
                         const int32_t* cache_len, const vvs_model_desc& md, int layer, int kv_rows,
-                        int n_rows, int t_len, int32_t* status, cudaStream_t s) {
+                        int n_rows, int t_len, int32_t* status, cudaStream_t s, const float* tab_cos,
+                        const float* tab_sin) {
   rope_append_kernel<T><<<n_rows * t_len, 256, 0, s>>>(
       qkv, inv_freq, q, kv_k, kv_v, cache_len, md.d_model, md.n_heads, md.head_dim, md.s_max,
-      md.rope_mode, md.rope_grid_w, md.n_prefix, layer, kv_rows, t_len, status);
+      md.rope_mode, md.rope_grid_w, md.n_prefix, layer, kv_rows, t_len, status, tab_cos, tab_sin);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -363,7 +369,7 @@ void launch_row_stats(const float* logits, float* part_m, float* part_s, int n_r
   template void launch_gemm_nt<T>(const T*, const T*, float*, int, int, int, int, bool, cudaStream_t); \
   template void launch_rope_append<T>(const float*, const float*, T*, T*, T*, const int32_t*,        \
                                       const vvs_model_desc&, int, int, int, int, int32_t*,           \
-                                      cudaStream_t);                                                 \
+                                      cudaStream_t, const float*, const float*);                     \
   template void launch_attention<T>(const T*, const T*, const T*, const int32_t*, T*,                \
                                     const vvs_model_desc&, int, int, int, int, cudaStream_t);        \
   template void launch_silu_mul<T>(const float*, T*, int, int, cudaStream_t);

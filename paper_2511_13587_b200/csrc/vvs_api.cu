@@ -83,8 +83,8 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
   c.take(ws.p_part, (size_t)d.max_rows * n_chunks * 8);
   if (d.dtype == VVS_DTYPE_BF16 && d.n_layers > 0) {
     c.take(ws.anc_mask, M * 4);
-    c.take(ws.tree_res, (size_t)2 * (d.max_rows < 32 ? d.max_rows : 32) * V * 8);
-    c.take(ws.tree_path, (size_t)32 * 32 * 4);
+    c.take(ws.tree_res, (size_t)2 * d.max_rows * V * 8);
+    c.take(ws.tree_path, (size_t)d.max_rows * 32 * 4);
   }
   if (d.dtype == VVS_DTYPE_BF16 && !std::getenv("VVS_DEBUG_GENERIC")) c.take(ws.logits_small, (M < 64 ? M : 64) * V * 4);
   return (c.off + 255) & ~size_t(255);
@@ -326,7 +326,8 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
       make_tmap_bf16_2d(&tm_v, kv_v, kv_total_rows, (uint64_t)md.head_dim, 128u) != VVS_OK)
     return VVS_ERR_CUDA;
   AttentionTcArgs at{};
-  at.tm_q = &tm_q; at.tm_k = &tm_k; at.tm_v = &tm_v; at.cache_len = a->cache_len; at.out = attn;
+  at.tm_q = &tm_q; at.tm_k = &tm_k; at.tm_v = &tm_v; at.cache_len = a->cache_len; at.anc_mask = ws.anc_mask;
+  at.out = attn;
   at.part_o = ws.attn_part_o; at.part_ml = ws.attn_part_ml; at.counters = ws.attn_counters;
   at.status = ws.status; at.d = d; at.n_heads = md.n_heads; at.hd = md.head_dim; at.s_max = md.s_max;
   at.kv_rows = a->kv_rows; at.t_len = Tn; at.n_rows = R; at.pdl = ctx->use_pdl;
@@ -365,8 +366,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   }
   VVS_LAUNCH(VVS_PROF_OTHER, launch_embed<T>(static_cast<const T*>(ctx->tok_emb), a->block, ws.x, B, C, Tn,
                                              d, md.tok_rows, ws.status, s));
-  if (a->tree_parent) return VVS_ERR_SHAPE;   // trees run on the whole-chain kernel only
-  VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, nullptr, B, a->n_forced, ws, md, R, Tn, s));
+  VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, a->tree_parent, B, a->n_forced, ws, md, R, Tn, s));
   for (int l = 0; l < md.n_layers && rc == VVS_OK; ++l) {
     const Layer& L = ctx->layers[l];
     const LayerMaps& W = ctx->layer_maps[l];
@@ -379,7 +379,9 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
       g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.out = ws.qkv; g.ldo = 3 * d;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_qkv, g, s));
       VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_append<T>(ws.qkv, ws.rope_inv_freq, q, kv_k, kv_v, a->cache_len, md,
-                                                       l, a->kv_rows, R, Tn, ws.status, s));
+                                                       l, a->kv_rows, R, Tn, ws.status, s,
+                                                       a->tree_parent ? ws.rope_cos : nullptr,
+                                                       a->tree_parent ? ws.rope_sin : nullptr));
     } else {
       GemmTcArgs g = base;
       g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.ld_scratch = 3 * d; g.layer = l;
@@ -417,6 +419,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   if (rc != VVS_OK) return rc;
   VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
   if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
+  if (a->tree_parent) return run_tree_decisions(ctx, hid, a, o, s);
   return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
 }
 
@@ -675,7 +678,7 @@ int vvs_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, 
   if (a->kv_rows < R) return VVS_ERR_SHAPE;
   if (a->tree_parent) {
     if (a->mode != VVS_MODE_STRICT || a->n_draft || !o->target_probs) return VVS_ERR_INVALID_ARG;
-    if (!ctx->tensor_core_path || !ctx->use_chain || !fused_chain_applicable(md, R, Tn)) return VVS_ERR_SHAPE;
+    if (!ctx->tensor_core_path) return VVS_ERR_SHAPE;     // Tn <= 32 = max_block holds for every call
   } else if (o->accept_path) {
     return VVS_ERR_INVALID_ARG;
   }

@@ -48,8 +48,8 @@ struct Workspace {
   // tensor-core path
   int32_t* slot_pos = nullptr;   // [M] cache slot of each block row, -1 if its sequence overflows
   uint32_t* anc_mask = nullptr;  // [M] bit j set: block row j of the same sequence is visible (ancestor or self)
-  double* tree_res = nullptr;    // [2][min(max_rows, 32), V] residuals of the tree walk (ping-pong)
-  int32_t* tree_path = nullptr;  // [32, 32] accepted nodes when the caller does not ask for them
+  double* tree_res = nullptr;    // [2][max_rows, V] residuals of the tree walk (ping-pong)
+  int32_t* tree_path = nullptr;  // [max_rows, 32] accepted nodes when the caller does not ask for them
   float* rope_cos = nullptr;     // [M, head_dim/2]
   float* rope_sin = nullptr;     // [M, head_dim/2]
   float* sk_scratch = nullptr;   // [M, max(3d, 2ff)] fp32 split-K sums; all zero between kernels
@@ -144,7 +144,8 @@ void launch_gemm_nt(const T* a, const T* w, float* c, int m, int n, int k, int l
 template <typename T>
 void launch_rope_append(const float* qkv, const float* inv_freq, T* q, T* kv_k, T* kv_v,
                         const int32_t* cache_len, const vvs_model_desc& md, int layer, int kv_rows,
-                        int n_rows, int t_len, int32_t* status, cudaStream_t s);
+                        int n_rows, int t_len, int32_t* status, cudaStream_t s, const float* tab_cos = nullptr,
+                        const float* tab_sin = nullptr);
 template <typename T>
 void launch_attention(const T* q, const T* kv_k, const T* kv_v, const int32_t* cache_len, T* out,
                       const vvs_model_desc& md, int layer, int kv_rows, int n_rows, int t_len,
@@ -188,6 +189,7 @@ struct AttentionTcArgs {
   const CUtensorMap* tm_k;   // cache viewed as [layers*kv_rows*heads*s_max, hd], box {64, 128}
   const CUtensorMap* tm_v;
   const int32_t* cache_len;
+  const uint32_t* anc_mask;  // [M] visible block rows per block row
   __nv_bfloat16* out;
   float* part_o; float* part_ml; int* counters; int32_t* status;
   int d, n_heads, hd, s_max, layer, kv_rows, t_len, n_rows;

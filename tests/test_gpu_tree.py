@@ -187,3 +187,21 @@ def test_tree_shapes(name, seed, parent, n_forced, n_cfg, q_noise):
     np.testing.assert_array_equal(gpu["accept_len"], ora["accept_len"])
     print(name, "accepted", gpu["accept_path"][0][:gpu["accept_len"][0]], "oracle", ora["accept_path"][0])
     run.close()
+
+
+@pytest.mark.parametrize("n_images,parent,n_forced,fills",
+                         [(2, TREE_A, 1, [130, 17]),                     # 36 tokens: QKV epilogue with rotation tables
+                          (4, TREE_B, 2, [124, 300, 5, 511]),            # 72 tokens: split-K sums + rotate/append kernel
+                          (3, [-1, 0, 1, 2, 2, 3, 3, 4, 4, 5, 6, 7, 8, 9, 10, 11, 12, 12, 12, 13, 14], 3, [60, 400, 222])])
+def test_tree_parity_per_projection_kernels(n_images, parent, n_forced, fills):
+    """More than 32 block tokens: the per-projection tensor-core kernels (attention with the same
+    visibility masks, rotation by depth from the step's tables)."""
+    ms = XL_SMALL
+    case = H.build_tree_case(ms, 900 + n_images, n_images, 2, n_forced, parent, fills, q_noise=0.7)
+    run = H.GpuRunner(ms, case["w"], 2 * n_images, len(parent))
+    gpu = H.run_tree_gpu(run, case)
+    assert gpu["launches"] > 20            # not the whole-chain kernel
+    ora = H.run_tree_oracle(case)
+    _check_tree(case, gpu, ora)
+    print("accept paths", [list(g[:n]) for g, n in zip(gpu["accept_path"], gpu["accept_len"])], "oracle", ora["accept_path"])
+    run.close()
