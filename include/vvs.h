@@ -225,7 +225,11 @@ int vvs_epilogue(vvs_ctx* ctx, const void* hidden, int32_t n_rows_per_seq, int32
  * residual / bonus sample on target probabilities the caller already holds (guidance and
  * softmax already applied).  target_probs is device float32 [B, n_rows_per_seq, V]; rows,
  * first_row and drafts as in vvs_epilogue.  args->n_cfg must be 1; cfg_scale and temperature are
- * ignored; out->new_len, n_commit, hidden and target_probs must be NULL.  Needs no weights. */
+ * ignored; out->new_len, n_commit, hidden and target_probs must be NULL.  Needs no weights.
+ * With args->tree_parent (device [B, n_rows_per_seq], as in vvs_verify with n_forced =
+ * first_row + 1 and first_row + 1 + K == n_rows_per_seq) the K drafts are the nodes of a
+ * candidate tree and the walk of vvs_verify's tree calls runs on the given rows;
+ * out->accept_path may then be given.  No cache is touched. */
 int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, int32_t first_row,
                const int32_t* drafts, const vvs_verify_args* args, const vvs_verify_out* out,
                void* stream);

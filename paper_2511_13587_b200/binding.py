@@ -221,10 +221,11 @@ def vvs_epilogue(ctx: int, *, hidden_in, n_rows_per_seq, first_row, drafts, n_im
 
 def vvs_decide(ctx: int, *, target_probs, n_rows_per_seq, first_row, drafts, n_images, n_draft_max,
                draft_probs, uniforms, accept_len, next_token, n_draft=None, mode=VVS_MODE_STRICT,
-               nbr_k=1, delta=float("inf"), accept_mask=None, margins=None, stream=None) -> None:
+               nbr_k=1, delta=float("inf"), accept_mask=None, margins=None, tree_parent=None,
+               accept_path=None, stream=None) -> None:
     a = _args(n_images, 1, 1, n_draft_max, None, n_draft, None, None, 0, None, None, draft_probs,
-              uniforms, 1.0, 1.0, mode, nbr_k, delta)
-    o = _out(accept_len, next_token, None, None, accept_mask, None, None, margins)
+              uniforms, 1.0, 1.0, mode, nbr_k, delta, tree_parent)
+    o = _out(accept_len, next_token, None, None, accept_mask, None, None, margins, accept_path)
     _check(lib.vvs_decide(ctx, _ptr(target_probs), int(n_rows_per_seq), int(first_row), _ptr(drafts),
                           C.byref(a), C.byref(o), _stream(stream)), "vvs_decide")
 

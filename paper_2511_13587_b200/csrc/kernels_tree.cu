@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(kTreeThreads) tree_walk_kernel(TreeParams p) {
     for (int ci = 0; ci < n_child; ++ci) {
       const int c = s_child[ci], i = c - F;
       const float* qrow = p.draft_probs + ((size_t)b * K + i) * V;
-      const int x = p.drafts[(size_t)b * T + i] - p.vocab_offset;
+      const int x = p.drafts[(size_t)b * p.drafts_ld + i] - p.vocab_offset;
       const bool x_ok = x >= 0 && x < V;
       if (tid == 0) {
         int pass = 0;
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(kTreeThreads) tree_walk_kernel(TreeParams p) {
     p.accept_len[b] = n_acc;
     for (int c = 0; c < p.n_cfg; ++c) {
       const int r = c * p.n_images + b;
-      if (p.new_len) p.new_len[r] = p.cache_len[r] + F + n_acc;
+      if (p.new_len && p.cache_len) p.new_len[r] = p.cache_len[r] + F + n_acc;
       if (p.n_commit) p.n_commit[r] = F + n_acc;
     }
   }

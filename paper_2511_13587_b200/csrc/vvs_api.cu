@@ -81,11 +81,9 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
   c.take(ws.p_row, (size_t)d.max_rows * V * 4);
   c.take(ws.r_part, (size_t)d.max_rows * n_chunks * 8);
   c.take(ws.p_part, (size_t)d.max_rows * n_chunks * 8);
-  if (d.dtype == VVS_DTYPE_BF16 && d.n_layers > 0) {
-    c.take(ws.anc_mask, M * 4);
-    c.take(ws.tree_res, (size_t)2 * d.max_rows * V * 8);
-    c.take(ws.tree_path, (size_t)d.max_rows * 32 * 4);
-  }
+  if (d.dtype == VVS_DTYPE_BF16 && d.n_layers > 0) c.take(ws.anc_mask, M * 4);
+  c.take(ws.tree_res, (size_t)2 * d.max_rows * V * 8);
+  c.take(ws.tree_path, (size_t)d.max_rows * 32 * 4);
   if (d.dtype == VVS_DTYPE_BF16 && !std::getenv("VVS_DEBUG_GENERIC")) c.take(ws.logits_small, (M < 64 ? M : 64) * V * 4);
   return (c.off + 255) & ~size_t(255);
 }
@@ -286,6 +284,7 @@ int run_tree_decisions(vvs_ctx* ctx, const __nv_bfloat16* hid, const vvs_verify_
   TreeParams tp{};
   tp.n_images = B; tp.n_cfg = C; tp.n_forced = a->n_forced; tp.n_draft_max = a->n_draft_max; tp.t_len = Tn;
   tp.vocab = V; tp.vocab_offset = md.vocab_offset; tp.parent = a->tree_parent; tp.drafts = a->block + a->n_forced;
+  tp.drafts_ld = Tn;
   tp.probs = o->target_probs; tp.draft_probs = a->draft_probs; tp.uniforms = a->uniforms; tp.cache_len = a->cache_len;
   tp.res = ws.tree_res; tp.accept_len = o->accept_len;
   tp.accept_path = o->accept_path ? o->accept_path : ws.tree_path;
@@ -727,11 +726,25 @@ int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, 
   if (first_row < 0 || first_row + a->n_draft_max > n_rows_per_seq) return VVS_ERR_SHAPE;
   if (a->n_draft_max > 0 && !drafts) return VVS_ERR_INVALID_ARG;
   if (o->new_len || o->hidden || o->n_commit || o->target_probs) return VVS_ERR_INVALID_ARG;
-  if (a->tree_parent || o->accept_path) return VVS_ERR_INVALID_ARG;
+  if (!a->tree_parent && o->accept_path) return VVS_ERR_INVALID_ARG;
   if (!aligned16(target_probs)) return VVS_ERR_ALIGN;
   ctx->launches = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   Workspace& ws = ctx->ws;
+  if (a->tree_parent) {
+    // the tree walk on the caller's rows: block rows 0 .. first_row are the forced chain
+    if (a->mode != VVS_MODE_STRICT || a->n_draft || !ws.tree_res) return VVS_ERR_INVALID_ARG;
+    if (first_row + 1 + a->n_draft_max != n_rows_per_seq) return VVS_ERR_SHAPE;
+    TreeParams tp{};
+    tp.n_images = a->n_images; tp.n_cfg = 1; tp.n_forced = first_row + 1; tp.n_draft_max = a->n_draft_max;
+    tp.t_len = n_rows_per_seq; tp.vocab = ctx->desc.vocab; tp.vocab_offset = ctx->desc.vocab_offset;
+    tp.parent = a->tree_parent; tp.drafts = drafts; tp.drafts_ld = a->n_draft_max; tp.probs = target_probs;
+    tp.draft_probs = a->draft_probs; tp.uniforms = a->uniforms; tp.res = ws.tree_res;
+    tp.accept_len = o->accept_len; tp.accept_path = o->accept_path ? o->accept_path : ws.tree_path;
+    tp.next_token = o->next_token; tp.accept_mask = o->accept_mask; tp.margins = o->margins; tp.status = ws.status;
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_tree_walk(tp, s));
+    return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+  }
   DecideParams p = decide_params(ctx, n_rows_per_seq, first_row, drafts, a->n_draft_max, a, o, false);
   p.direct_probs = target_probs;
   if (p.n_draft_max > 0) VVS_LAUNCH(VVS_PROF_OTHER, launch_gather_logits(target_probs, ws, p, s));

@@ -240,7 +240,8 @@ struct FusedChainArgs {
 struct TreeParams {
   int n_images, n_cfg, n_forced, n_draft_max, t_len, vocab, vocab_offset;
   const int32_t* parent;      // [B, T]
-  const int32_t* drafts;      // block + n_forced, row stride t_len
+  const int32_t* drafts;      // embedding-table ids of the draft nodes, row stride drafts_ld
+  int drafts_ld;
   const float* probs;         // [B, T, V] target rows of all block rows
   const float* draft_probs;   // [B, K, V]
   const float* uniforms;      // [B, K+1]

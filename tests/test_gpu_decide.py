@@ -108,3 +108,82 @@ def test_decide_is_bit_exact_with_oracle(v, n_images, k, rows, first_row, mode, 
     rate = want["accept_len"].sum() / max(1, c["n_draft"].sum())
     assert 0.0 <= rate <= 1.0
     vb.vvs_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------------------
+# candidate trees: the walk of vvs_verify's tree calls on given probabilities
+
+
+def tree_decide_case(seed, v, n_images, k, n_forced, tau, gumbel, off=0):
+    """Random trees (every draft node hangs below a uniformly drawn earlier node or the last
+    forced row), target rows softmax(2 N(0,1)), one drafter row per parent node (its target
+    logits cooled / perturbed), siblings drawn independently from it."""
+    rng = gen.rng_for(seed, "tree_decide")
+    rows = n_forced + k
+    t_logits = rng.standard_normal((n_images, rows, v)) * 2.0
+    p = gen.softmax_rows_f32(t_logits)
+    parent = np.zeros((n_images, rows), np.int32)
+    parent[:, :n_forced] = np.arange(-1, n_forced - 1)
+    q = np.zeros((n_images, k, v), np.float32)
+    drafts = np.zeros((n_images, k), np.int32)
+    for b in range(n_images):
+        for c in range(n_forced, rows):
+            parent[b, c] = rng.integers(n_forced - 1, c)
+        for pn in range(n_forced - 1, rows):
+            kids = [c for c in range(n_forced, rows) if parent[b, c] == pn]
+            if not kids:
+                continue
+            q_row, _ = gen.perturbed_draft_row(seed, f"tq.{b}.{pn}", t_logits[b, pn], 0.0, tau, gumbel)
+            for c in kids:
+                q[b, c - n_forced] = q_row
+                drafts[b, c - n_forced] = gen.sample_rows(q_row[None, :], gen.rng_for(seed, f"tc.{b}.{c}").random(1))[0]
+    return dict(ms=ModelShape("tdec", 0, 64, 0, 0, 0, v, vocab_offset=off, dtype=DTYPE_BF16), probs=p,
+                draft_probs=q, drafts=drafts + off, parent=parent,
+                uniforms=philox.verify_uniforms(seed, 5, n_images, k), n_images=n_images, n_draft_max=k,
+                rows=rows, n_forced=n_forced)
+
+
+@pytest.mark.parametrize("v,n_images,k,n_forced,tau,gumbel,off",
+                         [(1000, 64, 12, 1, 1.0, 0.5, 0), (16384, 32, 15, 3, 0.5, 1.5, 100),
+                          (4096 + 40, 16, 31, 1, 1.0, 2.5, 0), (512, 64, 6, 2, 2.0, 3.0, 7)])
+def test_tree_walk_is_exact_on_random_trees(v, n_images, k, n_forced, tau, gumbel, off):
+    """Same float32 inputs on both sides: accepted paths and sampled tokens must be equal; only
+    decisions within 1e-12 of their threshold (float64 summation order of a later-round
+    normaliser, or of the sampling CDF) are left out."""
+    import torch
+    from paper_2511_13587_b200 import binding as vb
+    c = tree_decide_case(v + k, v, n_images, k, n_forced, tau, gumbel, off)
+    rows = c["rows"]
+    ctx = vb.vvs_create(vb.make_desc(c["ms"], n_images, rows, 1))
+    o = dict(accept_len=torch.full((n_images,), -7, dtype=torch.int32, device="cuda"),
+             next_token=torch.full((n_images,), -7, dtype=torch.int32, device="cuda"),
+             accept_mask=torch.full((n_images, k), 9, dtype=torch.uint8, device="cuda"),
+             accept_path=torch.full((n_images, k), -7, dtype=torch.int32, device="cuda"),
+             margins=torch.zeros((n_images, k + 1), dtype=torch.float32, device="cuda"))
+    vb.vvs_decide(ctx, target_probs=H.to_dev(c["probs"]), n_rows_per_seq=rows, first_row=n_forced - 1,
+                  drafts=H.to_dev(c["drafts"]), n_images=n_images, n_draft_max=k,
+                  draft_probs=H.to_dev(c["draft_probs"]), uniforms=H.to_dev(c["uniforms"]),
+                  tree_parent=H.to_dev(c["parent"]), **o)
+    torch.cuda.synchronize()
+    assert vb.vvs_device_status(ctx) == 0
+    got = {k_: H.to_host(t) for k_, t in o.items()}
+    judged = rejected_rounds = 0
+    for b in range(n_images):
+        d = O.tree_decide(c["probs"][b], c["drafts"][b] - off, c["parent"][b], n_forced, c["draft_probs"][b],
+                          c["uniforms"][b])
+        if np.any(d["margins"][:k] < 1e-12):
+            continue
+        n = int(got["accept_len"][b])
+        assert n == d["accept_len"], b
+        assert [int(x) for x in got["accept_path"][b][:n]] == d["accept_path"], b
+        assert (got["accept_path"][b][n:] == -1).all()
+        mask = np.zeros(k, np.uint8)
+        mask[[x - n_forced for x in d["accept_path"]]] = 1
+        np.testing.assert_array_equal(got["accept_mask"][b], mask)
+        np.testing.assert_allclose(np.minimum(got["margins"][b][:k], 1e30), np.minimum(d["margins"][:k], 1e30), atol=1e-6)
+        if d["margins"][k] >= 1e-12:
+            assert got["next_token"][b] == d["next_token"] + off, b
+        judged += int(np.isfinite(d["margins"][:k]).sum())
+        rejected_rounds += int(np.isfinite(d["margins"][:k]).sum()) - d["accept_len"]
+    assert judged > n_images and rejected_rounds > 0      # the cases exercise both outcomes
+    vb.vvs_destroy(ctx)
