@@ -155,12 +155,15 @@ gemm_tc_kernel(const KernelParams p, const __grid_constant__ CUtensorMap tm_a,
   uint32_t it_p = 0, it_c = 0;
   bool alive = true;
 
-  for (int pass = 0; pass < p.passes && alive; ++pass) {
+  // One token pass per CTA (blockIdx.z): with more than 256 tokens the passes of a tile run as
+  // separate CTAs, two to an SM, so that one's epilogue overlaps the other's loads and MMAs.
+  const int pass0 = blockIdx.z;
+  for (int pass = pass0; pass < pass0 + 1 && alive; ++pass) {
     const int tok0 = pass * p.nt;
     if (warp == 0 && lane == 0) {
       // ---- TMA producer ------------------------------------------------------------------
       int kb = kb0;
-      if (pass == 0) {
+      {
         const int n_pre = nkb < p.stages ? nkb : p.stages;  // all stages are free: weights first
         for (int i = 0; i < n_pre; ++i) {
           uint8_t* st = smem + (size_t)i * stage_bytes;
@@ -215,7 +218,7 @@ gemm_tc_kernel(const KernelParams p, const __grid_constant__ CUtensorMap tm_a,
     __syncwarp();
     pdl_wait();
     // ---- epilogue: all four warps ----------------------------------------------------------
-    bool got = wait_or_abort(&acc_bar, pass & 1, &s_abort);
+    bool got = wait_or_abort(&acc_bar, 0, &s_abort);
     if (!got) s_abort = 1;
     if (__syncthreads_or(got ? 0 : 1)) {
       if (threadIdx.x == 0) atomicOr(p.status, VVS_DEV_TIMEOUT);
@@ -382,7 +385,7 @@ cudaError_t launch_one(const GemmTcPlan& plan, const KernelParams& kp, const CUt
     configured = 200 * 1024 + 1024;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(tiles, plan.splits, 1);
+  cfg.gridDim = dim3(tiles, plan.splits, plan.passes);
   cfg.blockDim = dim3(128, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = s;
@@ -427,9 +430,10 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
   int best = 1;
   long long best_cost = -1;
   const int max_splits = allow_split ? (pl.kb_total < 32 ? pl.kb_total : 32) : 1;
+  const long long slots = (long long)n_sms * (pl.passes > 1 ? 2 : 1);   // several passes: two CTAs per SM
   for (int s = 1; s <= max_splits; ++s) {
     const long long per_cta = (pl.kb_total + s - 1) / s;
-    const long long waves = ((long long)pl.tiles * s + n_sms - 1) / n_sms;
+    const long long waves = ((long long)pl.tiles * s * pl.passes + slots - 1) / slots;
     const long long cost = per_cta * waves * 64 + s;  // mild preference for fewer splits
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
@@ -439,7 +443,7 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
   pl.splits = best;
   const uint32_t stage_bytes = kATileBytes * (dual ? 2u : 1u) + (uint32_t)pl.nt * kBlockK * 2u;
   const int per_cta = (pl.kb_total + pl.splits - 1) / pl.splits;
-  int stages = (200 * 1024) / (int)stage_bytes;
+  int stages = ((pl.passes > 1 ? 110 : 200) * 1024) / (int)stage_bytes;   // two CTAs per SM when passes are CTAs
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages > per_cta) stages = per_cta;
   if (stages < 1) stages = 1;
