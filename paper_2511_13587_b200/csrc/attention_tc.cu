@@ -177,39 +177,58 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
     // at the start of the step, several launches ago)
     const uint32_t anc_l = lane < T ? p.anc_mask[r * T + lane] : 0u;
     __syncthreads();
-    // one warp per query row: mask, max, exp, sum; lane owns keys 4*lane .. 4*lane+3
+    // eight lanes per query row (16 keys each), sixteen rows per pass: mask, max, exp, sum.
+    // Visible: a cache key (kj < 0) or block row kj with its bit set in the row's mask.
 #pragma unroll 1
-    for (int t = warp; t < T; t += 4) {
-      const uint32_t anc = __shfl_sync(0xffffffffu, anc_l, t);
-      const float4 s4 = reinterpret_cast<const float4*>(sP + (t >> 4) * kKVBytes + 4096)[(t & 15) * 32 + lane];
-      float sv[4] = {s4.x, s4.y, s4.z, s4.w};
+    for (int t0 = 0; t0 < T; t0 += 16) {
+      const int t = t0 + warp * 4 + (lane >> 3), sub = lane & 7;
+      const bool live = t < T;
+      const uint32_t anc = __shfl_sync(0xffffffffu, anc_l, t & 31);
+      float sv[16];
       float mx = -CUDART_INF_F;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int kj = key0 + 4 * lane + j - fill;   // < 0: cache slot; else block row kj
-        const uint32_t vis = (kj < 0 ? 1u : 0u) | (((uint32_t)kj < 32u ? 1u : 0u) & (anc >> (kj & 31)));
-        sv[j] = (vis & 1u) ? sv[j] * p.scale : -CUDART_INF_F;
-        mx = fmaxf(mx, sv[j]);
+      for (int c = 0; c < 4; ++c) {
+        const int cc = (c + (sub >> 1)) & 3;          // rotation: conflict-free 128-bit loads
+        float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (live) s4 = reinterpret_cast<const float4*>(sP + (t >> 4) * kKVBytes + 4096)[(t & 15) * 32 + sub * 4 + cc];
+        const float in[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int kj = key0 + sub * 16 + cc * 4 + j - fill;
+          const uint32_t vis = (kj < 0 ? 1u : 0u) | (((uint32_t)kj < 32u ? 1u : 0u) & (anc >> (kj & 31)));
+          sv[c * 4 + j] = (live && (vis & 1u)) ? in[j] * p.scale : -CUDART_INF_F;
+          mx = fmaxf(mx, sv[c * 4 + j]);
+        }
       }
-      mx = warp_max_f(mx);
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
       float sum = 0.f;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        sv[j] = (sv[j] == -CUDART_INF_F) ? 0.f : __expf(sv[j] - mx);
-        sum += sv[j];
+      for (int i = 0; i < 16; ++i) {
+        sv[i] = (sv[i] == -CUDART_INF_F) ? 0.f : __expf(sv[i] - mx);
+        sum += sv[i];
       }
-      sum = warp_sum_f(sum);
-      if (lane == 0) {
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+      if (live && sub == 0) {
         red_max[0][t] = mx;
         red_sum[0][t] = sum;
       }
-      // P[t, key] as bf16, K-major rows of 64 keys with the 128-byte swizzle
-      const int k4 = 4 * lane;
-      uint2 pk;
-      *reinterpret_cast<__nv_bfloat162*>(&pk.x) = __floats2bfloat162_rn(sv[0], sv[1]);
-      *reinterpret_cast<__nv_bfloat162*>(&pk.y) = __floats2bfloat162_rn(sv[2], sv[3]);
-      uint8_t* dst = sP + (k4 >> 6) * kKVBytes + t * 128 + (((((k4 & 63) >> 3) ^ (t & 7)) << 4) | ((k4 & 7) << 1));
-      *reinterpret_cast<uint2*>(dst) = pk;
+      if (live) {
+        // P[t, key] as bf16, K-major rows of 64 keys with the 128-byte swizzle
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int cc = (c + (sub >> 1)) & 3;
+          const int k4 = sub * 16 + cc * 4;
+          uint2 pk;
+          *reinterpret_cast<__nv_bfloat162*>(&pk.x) = __floats2bfloat162_rn(sv[c * 4], sv[c * 4 + 1]);
+          *reinterpret_cast<__nv_bfloat162*>(&pk.y) = __floats2bfloat162_rn(sv[c * 4 + 2], sv[c * 4 + 3]);
+          uint8_t* dst = sP + (k4 >> 6) * kKVBytes + t * 128 + (((((k4 & 63) >> 3) ^ (t & 7)) << 4) | ((k4 & 7) << 1));
+          *reinterpret_cast<uint2*>(dst) = pk;
+        }
+      }
     }
     // V rows of keys that no query may see: cleared, so unwritten cache slots cannot inject NaN
     if (!wait_bounded(&bar_v, 0)) atomicOr(p.status, VVS_DEV_TIMEOUT);
