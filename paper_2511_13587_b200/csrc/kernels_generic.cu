@@ -159,12 +159,13 @@ void launch_gemm_nt(const T* a, const T* w, float* c, int m, int n, int k, int l
 // ---------------------------------------------------------------------------------------------
 // RoPE on q and k of the block rows, k/v appended to the cache at slots L_r + t.
 template <typename T>
-__global__ void rope_append_kernel(const float* __restrict__ qkv, const float* __restrict__ inv_freq,
+__global__ void rope_append_kernel(float* __restrict__ qkv, const float* __restrict__ inv_freq,
                                    T* __restrict__ q, T* __restrict__ kv_k, T* __restrict__ kv_v,
                                    const int32_t* __restrict__ cache_len, int d, int n_heads, int hd,
                                    int s_max, int rope_mode, int grid_w, int n_prefix, int layer,
                                    int kv_rows, int t_len, int32_t* status,
-                                   const float* __restrict__ tab_cos, const float* __restrict__ tab_sin) {
+                                   const float* __restrict__ tab_cos, const float* __restrict__ tab_sin,
+                                   int clear_src) {
   int m = blockIdx.x;
   int r = m / t_len, t = m % t_len;
   int fill = cache_len[r];
@@ -179,7 +180,7 @@ __global__ void rope_append_kernel(const float* __restrict__ qkv, const float* _
     c_lo = (float)(n / grid_w);
     c_hi = (float)(n % grid_w);
   }
-  const float* src = qkv + (size_t)m * 3 * d;
+  float* src = qkv + (size_t)m * 3 * d;
   int half = hd / 2;
   for (int p = threadIdx.x; p < d / 2; p += blockDim.x) {
     int h = p / half, i = p % half;
@@ -202,17 +203,23 @@ __global__ void rope_append_kernel(const float* __restrict__ qkv, const float* _
       kv_v[slot] = from_f<T>(src[2 * d + e]);
       kv_v[slot + 1] = from_f<T>(src[2 * d + e + 1]);
     }
+    if (clear_src) {                           // split-K sums are added into this buffer: leave it zero
+      const float2 z = make_float2(0.f, 0.f);
+      *reinterpret_cast<float2*>(src + e) = z;
+      *reinterpret_cast<float2*>(src + d + e) = z;
+      *reinterpret_cast<float2*>(src + 2 * d + e) = z;
+    }
   }
 }
 
 template <typename T>
-void launch_rope_append(const float* qkv, const float* inv_freq, T* q, T* kv_k, T* kv_v,
+void launch_rope_append(float* qkv, const float* inv_freq, T* q, T* kv_k, T* kv_v,
                         const int32_t* cache_len, const vvs_model_desc& md, int layer, int kv_rows,
                         int n_rows, int t_len, int32_t* status, cudaStream_t s, const float* tab_cos,
-                        const float* tab_sin) {
+                        const float* tab_sin, bool clear_src) {
   rope_append_kernel<T><<<n_rows * t_len, 256, 0, s>>>(
       qkv, inv_freq, q, kv_k, kv_v, cache_len, md.d_model, md.n_heads, md.head_dim, md.s_max,
-      md.rope_mode, md.rope_grid_w, md.n_prefix, layer, kv_rows, t_len, status, tab_cos, tab_sin);
+      md.rope_mode, md.rope_grid_w, md.n_prefix, layer, kv_rows, t_len, status, tab_cos, tab_sin, clear_src ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -297,8 +304,8 @@ void launch_attention(const T* q, const T* kv_k, const T* kv_v, const int32_t* c
 // ---------------------------------------------------------------------------------------------
 // act[m, j] = silu(gate[m, j]) * up[m, j]; grid (column chunks of 1024, rows), 4 columns per thread
 template <typename T>
-__global__ void silu_mul_kernel(const float* __restrict__ gu, T* __restrict__ act, int ff) {
-  const float* row = gu + (size_t)blockIdx.y * 2 * ff;
+__global__ void silu_mul_kernel(float* __restrict__ gu, T* __restrict__ act, int ff, int clear_src) {
+  float* row = gu + (size_t)blockIdx.y * 2 * ff;
   T* o = act + (size_t)blockIdx.y * ff;
   const int j = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (j >= ff) return;                       // ff is a multiple of 8
@@ -308,11 +315,16 @@ __global__ void silu_mul_kernel(const float* __restrict__ gu, T* __restrict__ ac
   o[j + 1] = from_f<T>(g.y / (1.f + expf(-g.y)) * u.y);
   o[j + 2] = from_f<T>(g.z / (1.f + expf(-g.z)) * u.z);
   o[j + 3] = from_f<T>(g.w / (1.f + expf(-g.w)) * u.w);
+  if (clear_src) {                             // split-K sums are added into this buffer: leave it zero
+    const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+    *reinterpret_cast<float4*>(row + j) = z;
+    *reinterpret_cast<float4*>(row + ff + j) = z;
+  }
 }
 
 template <typename T>
-void launch_silu_mul(const float* gu, T* act, int m, int ff, cudaStream_t s) {
-  silu_mul_kernel<T><<<dim3((ff + 1023) / 1024, m), 256, 0, s>>>(gu, act, ff);
+void launch_silu_mul(float* gu, T* act, int m, int ff, cudaStream_t s, bool clear_src) {
+  silu_mul_kernel<T><<<dim3((ff + 1023) / 1024, m), 256, 0, s>>>(gu, act, ff, clear_src ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -367,12 +379,12 @@ void launch_row_stats(const float* logits, float* part_m, float* part_s, int n_r
                                 cudaStream_t);                                                       \
   template void launch_rmsnorm<T>(const float*, const T*, T*, int, int, float, cudaStream_t);        \
   template void launch_gemm_nt<T>(const T*, const T*, float*, int, int, int, int, bool, cudaStream_t); \
-  template void launch_rope_append<T>(const float*, const float*, T*, T*, T*, const int32_t*,        \
+  template void launch_rope_append<T>(float*, const float*, T*, T*, T*, const int32_t*,              \
                                       const vvs_model_desc&, int, int, int, int, int32_t*,           \
-                                      cudaStream_t, const float*, const float*);                     \
+                                      cudaStream_t, const float*, const float*, bool);               \
   template void launch_attention<T>(const T*, const T*, const T*, const int32_t*, T*,                \
                                     const vvs_model_desc&, int, int, int, int, cudaStream_t);        \
-  template void launch_silu_mul<T>(const float*, T*, int, int, cudaStream_t);
+  template void launch_silu_mul<T>(float*, T*, int, int, cudaStream_t, bool);
 VVS_INSTANTIATE(float)
 VVS_INSTANTIATE(__nv_bfloat16)
 

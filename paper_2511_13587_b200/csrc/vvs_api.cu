@@ -366,6 +366,14 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   VVS_LAUNCH(VVS_PROF_OTHER, launch_embed<T>(static_cast<const T*>(ctx->tok_emb), a->block, ws.x, B, C, Tn,
                                              d, md.tok_rows, ws.status, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, a->tree_parent, B, a->n_forced, ws, md, R, Tn, s));
+  if (wide) {
+    // the split-K sums of the QKV and gate / up projections are added into these buffers; the
+    // kernels that consume them clear what they read, so one clearing per call is enough (it also
+    // covers a previous call that ended early)
+    if (cudaMemsetAsync(ws.qkv, 0, (size_t)M * 3 * d * sizeof(float), s) != cudaSuccess ||
+        cudaMemsetAsync(ws.gu, 0, (size_t)M * 2 * ff * sizeof(float), s) != cudaSuccess)
+      return VVS_ERR_CUDA;
+  }
   for (int l = 0; l < md.n_layers && rc == VVS_OK; ++l) {
     const Layer& L = ctx->layers[l];
     const LayerMaps& W = ctx->layer_maps[l];
@@ -373,14 +381,13 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     if (wide) {
       // many tokens: a per-thread epilogue over hundreds of tokens is slower than a plain split-K
       // sum into fp32 followed by one thread per element for rotation, rounding and cache append
-      if (cudaMemsetAsync(ws.qkv, 0, (size_t)M * 3 * d * sizeof(float), s) != cudaSuccess) return VVS_ERR_CUDA;
       GemmTcArgs g = base;
       g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.out = ws.qkv; g.ldo = 3 * d;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_qkv, g, s));
       VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_append<T>(ws.qkv, ws.rope_inv_freq, q, kv_k, kv_v, a->cache_len, md,
                                                        l, a->kv_rows, R, Tn, ws.status, s,
                                                        a->tree_parent ? ws.rope_cos : nullptr,
-                                                       a->tree_parent ? ws.rope_sin : nullptr));
+                                                       a->tree_parent ? ws.rope_sin : nullptr, true));
     } else {
       GemmTcArgs g = base;
       g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.ld_scratch = 3 * d; g.layer = l;
@@ -397,13 +404,12 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     }
     VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm2), xn, M, d, md.rms_eps, s));
     if (rc == VVS_OK && wide) {
-      if (cudaMemsetAsync(ws.gu, 0, (size_t)M * 2 * ff * sizeof(float), s) != cudaSuccess) return VVS_ERR_CUDA;
       GemmTcArgs g = base;
       g.n = ff; g.k = d; g.tm_a = &W.w_gate; g.tm_b = &tm_xn; g.out = ws.gu; g.ldo = 2 * ff;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_g1, g, s));
       g.tm_a = &W.w_up; g.out = ws.gu + ff;
       if (rc == VVS_OK) VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_g1, g, s));
-      VVS_LAUNCH(VVS_PROF_OTHER, launch_silu_mul<T>(ws.gu, act, M, ff, s));
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_silu_mul<T>(ws.gu, act, M, ff, s, true));
     } else if (rc == VVS_OK) {
       GemmTcArgs g = base;
       g.n = ff; g.k = d; g.tm_a = &W.w_gate; g.tm_a2 = &W.w_up; g.tm_b = &tm_xn; g.ld_scratch = 2 * ff;

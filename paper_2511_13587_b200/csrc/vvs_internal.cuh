@@ -142,16 +142,16 @@ template <typename T>
 void launch_gemm_nt(const T* a, const T* w, float* c, int m, int n, int k, int ldc, bool accumulate,
                     cudaStream_t s);
 template <typename T>
-void launch_rope_append(const float* qkv, const float* inv_freq, T* q, T* kv_k, T* kv_v,
+void launch_rope_append(float* qkv, const float* inv_freq, T* q, T* kv_k, T* kv_v,
                         const int32_t* cache_len, const vvs_model_desc& md, int layer, int kv_rows,
                         int n_rows, int t_len, int32_t* status, cudaStream_t s, const float* tab_cos = nullptr,
-                        const float* tab_sin = nullptr);
+                        const float* tab_sin = nullptr, bool clear_src = false);
 template <typename T>
 void launch_attention(const T* q, const T* kv_k, const T* kv_v, const int32_t* cache_len, T* out,
                       const vvs_model_desc& md, int layer, int kv_rows, int n_rows, int t_len,
                       cudaStream_t s);
 template <typename T>
-void launch_silu_mul(const float* gu, T* act, int m, int ff, cudaStream_t s);
+void launch_silu_mul(float* gu, T* act, int m, int ff, cudaStream_t s, bool clear_src = false);
 void launch_guide(const float* raw, float* logits, int n_images, int n_cfg, int rows_per_seq, int v,
                   float cfg_scale, float inv_temp, cudaStream_t s);
 void launch_row_stats(const float* logits, float* part_m, float* part_s, int n_rows, int v,
