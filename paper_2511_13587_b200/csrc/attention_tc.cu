@@ -10,7 +10,10 @@
 //   3. Each thread owns one key: scale, causal mask, per-query max / sum over the 128 keys by
 //      warp shuffles + shared memory, P = exp(S - max) written as bf16 into swizzled shared
 //      memory.  V rows of masked-out keys are zeroed so stale cache contents cannot leak.
-//   4. O = P V  (tcgen05.mma, M = 128 (rows >= T are don't-care), N = hd, V as MN-major operand).
+//   4. O^T = V^T P^T  (tcgen05.mma, M = 128 head-dimension rows (rows >= hd are don't-care), N = 16/32
+//      queries, V as MN-major A operand, P as K-major B operand of only 16/32 rows: the P tile is
+//      4-8 KB instead of the 32 KB a 128-row A operand would take, which is what lets four CTAs
+//      share an SM).
 //   5. Query rows write (max, sum, O) partials; the CTA that arrives last for (r, h) merges the
 //      chunks (exact softmax re-normalisation) and writes the bf16 attention output.  No CTA
 //      waits for another.
@@ -69,9 +72,10 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sK = smem;
   uint8_t* sV = sK + NC * kKVBytes;
-  uint8_t* sP = sV + NC * kKVBytes;                 // 2 chunks of 64 keys: [128 rows x 128 B] each
-  uint8_t* sQ = sP + 2 * kKVBytes;                  // NC chunks: [tq rows x 128 B]
   const uint32_t q_chunk_bytes = (uint32_t)p.tq * 128u;
+  uint8_t* sP = sV + NC * kKVBytes;                 // 2 chunks of 64 keys: [tq rows x 128 B] each
+  uint8_t* sQ = sP + 2 * q_chunk_bytes;             // NC chunks: [tq rows x 128 B]
+  float* sS = reinterpret_cast<float*>(sQ + NC * q_chunk_bytes);   // scores, [tq queries][128 keys] fp32
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
   const int c = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
@@ -164,14 +168,13 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
     const int key = key0 + tid;
     const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
     {
-      // scores of this key for all queries -> shared memory, transposed ([query][key], fp32; kept in
-      // rows of the P tiles that belong to no query)
+      // scores of this key for all queries -> shared memory, transposed ([query][key], fp32)
       float sc[32];
       tmem_ld16(t_row, sc);
       if (p.tq > 16) tmem_ld16(t_row + 16, sc + 16);
 #pragma unroll
       for (int t = 0; t < 32; ++t)
-        if (t < p.tq) reinterpret_cast<float*>(sP + (t >> 4) * kKVBytes + 4096)[(t & 15) * 128 + tid] = sc[t];
+        if (t < p.tq) sS[t * 128 + tid] = sc[t];
     }
     // visibility masks of this sequence's block rows, one per lane (written by the table kernel
     // at the start of the step, several launches ago)
@@ -190,7 +193,7 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
       for (int c = 0; c < 4; ++c) {
         const int cc = (c + (sub >> 1)) & 3;          // rotation: conflict-free 128-bit loads
         float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (live) s4 = reinterpret_cast<const float4*>(sP + (t >> 4) * kKVBytes + 4096)[(t & 15) * 32 + sub * 4 + cc];
+        if (live) s4 = reinterpret_cast<const float4*>(sS)[t * 32 + sub * 4 + cc];
         const float in[4] = {s4.x, s4.y, s4.z, s4.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -225,7 +228,7 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
           uint2 pk;
           *reinterpret_cast<__nv_bfloat162*>(&pk.x) = __floats2bfloat162_rn(sv[c * 4], sv[c * 4 + 1]);
           *reinterpret_cast<__nv_bfloat162*>(&pk.y) = __floats2bfloat162_rn(sv[c * 4 + 2], sv[c * 4 + 3]);
-          uint8_t* dst = sP + (k4 >> 6) * kKVBytes + t * 128 + (((((k4 & 63) >> 3) ^ (t & 7)) << 4) | ((k4 & 7) << 1));
+          uint8_t* dst = sP + (k4 >> 6) * q_chunk_bytes + t * 128 + (((((k4 & 63) >> 3) ^ (t & 7)) << 4) | ((k4 & 7) << 1));
           *reinterpret_cast<uint2*>(dst) = pk;
         }
       }
@@ -245,13 +248,14 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
     __syncthreads();
     tc_fence_after();
     if (warp == 1 && lane == 0) {
-      // O[query, e] = sum_key P[query, key] V[key, e]
-      const uint32_t idesc = idesc_bf16_f32(128, (uint32_t)HD) | (1u << 16);  // B is MN-major
+      // O^T[e, query] = sum_key V[key, e] P[query, key]; with hd = 64 the rows 64..127 of the A operand
+      // come from whatever follows the V tile in shared memory and land in TMEM lanes nobody reads
+      const uint32_t idesc = idesc_bf16_f32(128, (uint32_t)p.tq) | (1u << 15);  // A is MN-major
 #pragma unroll
       for (int k16 = 0; k16 < kChunkKeys / 16; ++k16) {
-        const uint32_t a = smem_u32(sP + (k16 / 4) * kKVBytes) + (k16 % 4) * 32;
-        const uint32_t b = smem_u32(sV) + k16 * 2048;
-        mma_bf16(tmem_base + 32, smem_desc_sw128(a), smem_desc_mn_sw128(b, kKVBytes), idesc, k16 > 0 ? 1u : 0u);
+        const uint32_t a = smem_u32(sV) + k16 * 2048;
+        const uint32_t b = smem_u32(sP + (k16 / 4) * q_chunk_bytes) + (k16 % 4) * 32;
+        mma_bf16(tmem_base + 32, smem_desc_mn_sw128(a, kKVBytes), smem_desc_sw128(b), idesc, k16 > 0 ? 1u : 0u);
       }
       mma_commit(&bar_o);
     }
@@ -265,32 +269,26 @@ attention_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_q
   if (alive) {
     tc_fence_after();
     const size_t rh = (size_t)r * p.n_heads + h;
-    if (warp == 0) {                                  // TMEM lanes 0..31 = query rows
-      const uint32_t t_row = tmem_base + 32;
-      float* po = p.part_o + ((rh * p.n_chunks_max + c) * T + lane) * HD;
-      // chunk-wide max and sum of query `lane` (the four warps' reductions are still in place)
-      const float mine_max = red_max[0][lane];
-      const float mine_sum = red_sum[0][lane];
-      for (int e0 = 0; e0 < HD; e0 += 16) {
-        float o[16];
-        tmem_ld16(t_row + e0, o);
-        if (lane < T) {
-          if (n_chunks == 1) {
-            const float inv = 1.f / mine_sum;
-            __nv_bfloat16* dst = p.out + ((size_t)r * T + lane) * p.d + (size_t)h * HD + e0;
+    if (warp * 32 < HD) {                             // TMEM lane = head-dimension index e
+      const int e = warp * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16) + 32;
+      float o[32];
+      tmem_ld16(t_row, o);
+      if (p.tq > 16) tmem_ld16(t_row + 16, o + 16);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) dst[i] = __float2bfloat16_rn(o[i] * inv);
-          } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) po[e0 + i] = o[i];
-          }
+      for (int t = 0; t < 32; ++t) {
+        if (t < T) {                                  // chunk-wide max / sum of query t are in red_max / red_sum
+          if (n_chunks == 1)
+            p.out[((size_t)r * T + t) * p.d + (size_t)h * HD + e] = __float2bfloat16_rn(o[t] / red_sum[0][t]);
+          else
+            p.part_o[((rh * p.n_chunks_max + c) * T + t) * HD + e] = o[t];
         }
       }
-      if (lane < T && n_chunks > 1) {
-        float* ml = p.part_ml + ((rh * p.n_chunks_max + c) * T + lane) * 2;
-        ml[0] = mine_max;
-        ml[1] = mine_sum;
-      }
+    }
+    if (tid < T && n_chunks > 1) {
+      float* ml = p.part_ml + ((rh * p.n_chunks_max + c) * T + tid) * 2;
+      ml[0] = red_max[0][tid];
+      ml[1] = red_sum[0][tid];
     }
     if (n_chunks > 1) {
       __threadfence();
@@ -336,10 +334,19 @@ int launch_attention_tc(const AttentionTcArgs& a, cudaStream_t s) {
   p.d = a.d; p.n_heads = a.n_heads; p.hd = a.hd; p.s_max = a.s_max; p.layer = a.layer;
   p.kv_rows = a.kv_rows; p.t_len = a.t_len; p.tq = a.t_len <= 16 ? 16 : 32;
   p.n_chunks_max = (a.s_max + kChunkKeys - 1) / kChunkKeys;
-  p.tmem_cols = a.hd == 64 ? 128u : 256u;
+  p.tmem_cols = 64u;                                  // scores at column 0, O^T at column 32 (16 or 32 wide each)
   p.scale = 1.0f / sqrtf((float)a.hd);
   const int nc = a.hd / 64;
-  const int smem = nc * 2 * kChunkKeys * 128 + 2 * kChunkKeys * 128 + nc * 32 * 128 + 1024;
+  // K and V chunk tiles, P (2 key chunks) and Q (nc chunks) of tq rows, transposed scores, alignment slack
+  // With hd = 64 the 128-row A operand of O^T = V^T P^T reaches one V tile (16 KB) past the V tile:
+  // what follows it must be at least that large, whatever it holds.
+  auto tail_bytes = [&](int tq) {
+    const int t = (2 + nc) * tq * 128 + tq * 512;
+    return (a.hd == 64 && t < kChunkKeys * 128) ? kChunkKeys * 128 : t;
+  };
+  const int smem = nc * 2 * kChunkKeys * 128 + tail_bytes(p.tq) + 1024;
+
+  const int smem_max = nc * 2 * kChunkKeys * 128 + tail_bytes(32) + 1024;
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p.n_chunks_max, a.n_heads, a.n_rows);
@@ -355,14 +362,14 @@ int launch_attention_tc(const AttentionTcArgs& a, cudaStream_t s) {
   static bool configured64 = false, configured128 = false;
   if (a.hd == 64) {
     if (!configured64) {
-      if (cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      if (cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess)
         return VVS_ERR_CUDA;
       configured64 = true;
     }
     e = cudaLaunchKernelEx(&cfg, attention_tc_kernel<64>, p, *a.tm_q, *a.tm_k, *a.tm_v);
   } else {
     if (!configured128) {
-      if (cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      if (cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess)
         return VVS_ERR_CUDA;
       configured128 = true;
     }

@@ -127,6 +127,22 @@ def test_7b_shape_small_bf16():
     run.close()
 
 
+@pytest.mark.parametrize("ms,n_images,n_forced,k,fills",
+                         [(B7_SMALL, 3, 1, 8, [300, 7, 120]),          # head_dim 128, 54 block tokens
+                          (XL_SMALL, 2, 3, 14, [100, 240]),            # 17 rows per sequence, 68 tokens
+                          (B7_SMALL, 2, 2, 17, [377, 128])])           # head_dim 128, 19 rows, 76 tokens
+def test_per_projection_kernels_head_dims_and_long_blocks(ms, n_images, n_forced, k, fills):
+    """More than 32 block tokens: the per-projection tensor-core kernels, with both head
+    dimensions and with more than 16 query rows per sequence."""
+    case = H.build_case(ms, 61 + k, n_images, 2, n_forced, k, fills, q_noise=0.8)
+    run = H.GpuRunner(ms, case["w"], 2 * n_images, n_forced + k)
+    gpu = run.verify(case)
+    assert gpu["launches"] > 20
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    run.close()
+
+
 def test_ragged_drafts_forced_prefix_and_cache_edges():
     """n_draft below K (including 0), two forced rows, an empty cache and a cache that the block
     fills to capacity."""
