@@ -202,6 +202,13 @@ __device__ __forceinline__ bool wait_fast(uint64_t* bar, uint32_t parity, volati
   return wait_bar(bar, parity, s_abort, status);
 }
 
+// x / d for 0 <= x < 2^21 and d >= 1 through the float unit (a handful of instructions; an integer
+// division is a dependent chain of ~30).  (x + 0.5) / d is at least 1 / (2d) away from every
+// integer; reciprocal and product are each rounded once, an error below (x / d) * 2^-23 < 1 / (4d).
+__device__ __forceinline__ int div_small(int x, int d) {
+  return (int)(((float)x + 0.5f) * __frcp_rn((float)d));
+}
+
 // One round of token-operand building by the 256 worker threads: nb <= (1 << lg) units,
 // 256 >> lg threads per unit.  A unit's slab is m rows x 8 groups of 8 columns (one 16-byte
 // swizzle chunk each); thread j of the unit takes group j & 7 of rows (j >> 3) + k * (tpu >> 3),
@@ -218,9 +225,10 @@ __device__ __noinline__ void build_round(const ChainParams& p, uint8_t* ring, ui
   const uint32_t NS = (uint32_t)p.n_stages;
   const int tpu = 256 >> lg, u = tid_w >> (8 - lg), j = tid_w & (tpu - 1);
   if (u >= nb) return;                                   // uniform per warp (tpu >= 32)
-  const uint32_t it = it0 + (uint32_t)u * per_unit, st = it % NS, use = it / NS;
+  const uint32_t it = it0 + (uint32_t)u * per_unit;
+  const uint32_t use = (uint32_t)div_small((int)it, (int)NS), st = it - use * NS;
   if (use > 0) wait_fast(&empty[st], (use - 1) & 1, s_abort, p.status);
-  const int s = s0 + u, tile = s / kbs, kb = s - tile * kbs;
+  const int s = s0 + u, tile = div_small(s, kbs), kb = s - tile * kbs;
   const int m = p.m, ff = p.ff;
   const int q = j & 7, row0 = j >> 3, rstep = tpu >> 3;
   const int col = kb * 64 + q * 8;
@@ -629,11 +637,12 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             const int fill = s_fill[r], n_keys = fill + T, key0 = c * 128;
             const int row_base = kv_row_base(l, r, h, c);
             const int per_head = p.hd >> 3;
+            const int ph_sh = p.hd == 64 ? 3 : 4;            // head_dim is 64 or 128: shifts, not divisions
             if (!grp_e) {
               // Q operand: q * (1/rms) rotated, bf16, K-major with the 128-byte swizzle
 #pragma unroll 1
               for (int idx = tid_g; idx < T * per_head; idx += kGroup) {
-                const int t = idx / per_head, ch = idx - t * per_head, e = ch << 3, tok = r * T + t;
+                const int t = idx >> ph_sh, ch = idx - (t << ph_sh), e = ch << 3, tok = r * T + t;
                 const float ssv = __ldcg(p.ss + (2 * l) * 32 + tok);
                 float v[8];
                 ldcg8(qkv + (size_t)tok * 3 * p.d + h * p.hd + e, v);
@@ -657,9 +666,9 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
                 const int n_new = new_hi - new_lo;
 #pragma unroll 1
                 for (int idx = tid_g; idx < n_new * per_head * 2; idx += kGroup) {
-                  const int which = idx / (n_new * per_head);       // 0 = K, 1 = V
+                  const int which = idx >= n_new * per_head ? 1 : 0;   // 0 = K, 1 = V
                   const int rem = idx - which * n_new * per_head;
-                  const int kk = rem / per_head, ch = rem - kk * per_head, e = ch << 3;
+                  const int kk = rem >> ph_sh, ch = rem - (kk << ph_sh), e = ch << 3;
                   const int key = new_lo + kk, t = key - fill, tok = r * T + t;
                   const float ssv = __ldcg(p.ss + (2 * l) * 32 + tok);
                   float v[8];
@@ -808,12 +817,14 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
           for (int b0 = 0; b0 < n_units; b0 += 2) {
             const int k = b0 + (grp_e ? 1 : 0);
             if (k < n_units) {
-              const uint32_t it = it_slab + (uint32_t)k, st = it % NS, use = it / NS;
+              const uint32_t it = it_slab + (uint32_t)k;
+              const uint32_t use = (uint32_t)div_small((int)it, (int)NS), st = it - use * NS;
               if (use > 0) wait_bar(&empty[st], (use - 1) & 1, &s_abort, p.status);
               if (b_tok < p.m) {
-                const int kb = (lo + k) % f.kbs;
+                const int kb = (lo + k) - div_small(lo + k, f.kbs) * f.kbs;
                 const int k0 = kb * 64 + b_qtr * 16;
-                const int h = k0 / p.hd, e = k0 - h * p.hd;
+                const int hd_sh = p.hd == 64 ? 6 : 7;
+                const int h = k0 >> hd_sh, e = k0 - (h << hd_sh);
                 const int nch = s_nch[b_r];
                 const size_t base = (((size_t)b_r * H + h) * p.n_chunks_max) * T + b_t;
                 float v[16];
