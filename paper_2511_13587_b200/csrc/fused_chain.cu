@@ -366,7 +366,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
   const int n_items = s_prefix[p.n_rows] * H;     // attention items of one layer, all CTAs
 
   auto decode_item = [&](int i, int& r, int& h, int& c) {
-    const int rc = i / H;
+    const int rc = div_small(i, H);
     h = i - rc * H;
     r = 0;
     while (r + 1 < p.n_rows && s_prefix[r + 1] <= rc) ++r;
@@ -638,6 +638,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             const int row_base = kv_row_base(l, r, h, c);
             const int per_head = p.hd >> 3;
             const int ph_sh = p.hd == 64 ? 3 : 4;            // head_dim is 64 or 128: shifts, not divisions
+            const float inv_d = 1.f / (float)p.d;
             if (!grp_e) {
               // Q operand: q * (1/rms) rotated, bf16, K-major with the 128-byte swizzle
 #pragma unroll 1
@@ -646,7 +647,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
                 const float ssv = __ldcg(p.ss + (2 * l) * 32 + tok);
                 float v[8];
                 ldcg8(qkv + (size_t)tok * 3 * p.d + h * p.hd + e, v);
-                const float rinv = rsqrtf(ssv / (float)p.d + p.eps);
+                const float rinv = rsqrtf(fmaf(ssv, inv_d, p.eps));
 #pragma unroll
                 for (int j = 0; j < 8; ++j) v[j] *= rinv;
                 rope8(p, tok, e, v);
@@ -673,7 +674,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
                   const float ssv = __ldcg(p.ss + (2 * l) * 32 + tok);
                   float v[8];
                   ldcg8(qkv + (size_t)tok * 3 * p.d + (which + 1) * p.d + h * p.hd + e, v);
-                  const float rinv = rsqrtf(ssv / (float)p.d + p.eps);
+                  const float rinv = rsqrtf(fmaf(ssv, inv_d, p.eps));
 #pragma unroll
                   for (int j = 0; j < 8; ++j) v[j] *= rinv;
                   if (which == 0) rope8(p, tok, e, v);
@@ -877,7 +878,10 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             if (tid_w == 0) VVS_TRACE(0x300 | (ph << 4) | (b0 & 15));
             named_bar_sync(BAR_W, kWorkers);
             if (tid_w == 0) VVS_TRACE(0x380 | (ph << 4) | (b0 & 15));
-            if (tid_w < 2 && b0 + tid_w < n_units && !s_abort) mbar_arrive(&full[(it_slab + (uint32_t)(b0 + tid_w)) % NS]);
+            if (tid_w < 2 && b0 + tid_w < n_units && !s_abort) {
+              const uint32_t it = it_slab + (uint32_t)(b0 + tid_w);
+              mbar_arrive(&full[it - (uint32_t)div_small((int)it, (int)NS) * NS]);
+            }
           }
         } else {
           // x * norm scale (QKV, gate/up) or silu(gate) * up (down): up to four units per round
@@ -891,7 +895,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             // A round may not reach around the ring: its threads wait for the slot of their own
             // unit to be free before any of them reports a unit of the round as built, so two
             // units of one round must never share a slot.
-            const int ring_cap = ((int)NS + (int)per_unit - 1) / (int)per_unit;
+            const int ring_cap = ((int)NS + f.dual) >> f.dual;            // ceil(NS / per_unit), per_unit = 1 or 2
             int cap = (ph != PH_DOWN && left > 4) ? 8 : 4;
             if (cap > ring_cap) cap = ring_cap;
             const int nb = left < cap ? left : cap;
@@ -912,13 +916,14 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
             if (tid_w == 0) VVS_TRACE(0x380 | (ph << 4) | (b0 & 15));
             if (tid_w < nb && !s_abort) {
               const uint32_t it = it0 + (uint32_t)tid_w * per_unit;
-              mbar_arrive(&full[it % NS]);
+              const uint32_t use1 = (uint32_t)div_small((int)it, (int)NS);
+              mbar_arrive(&full[it - use1 * NS]);
               if (f.dual) {
                 // the second stage of the unit holds no token slab, but its barrier must be in the
                 // phase of this use before it takes the arrival
-                const uint32_t it2 = it + 1, use2 = it2 / NS;
-                if (use2 > 0) wait_fast(&empty[it2 % NS], (use2 - 1) & 1, &s_abort, p.status);
-                if (!s_abort) mbar_arrive(&full[it2 % NS]);
+                const uint32_t it2 = it + 1, use2 = (uint32_t)div_small((int)it2, (int)NS), st2 = it2 - use2 * NS;
+                if (use2 > 0) wait_fast(&empty[st2], (use2 - 1) & 1, &s_abort, p.status);
+                if (!s_abort) mbar_arrive(&full[st2]);
               }
             }
             b0 += nb;
@@ -943,7 +948,7 @@ fused_chain_kernel(const __grid_constant__ ChainParams p, const __grid_constant_
           int s = lo;
 #pragma unroll 1
           while (s < hi) {
-            const int tile = s / f.kbs;
+            const int tile = div_small(s, f.kbs);
             int next = (tile + 1) * f.kbs;
             s = next < hi ? next : hi;
             const uint32_t slot = ita % kAccSlots;
