@@ -29,7 +29,7 @@ from vvs_synth.configs import CONFIGS, MODE_RELAXED  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu
 # capture summarised under profiles/ (None until one has been taken for the current kernel).
-NCU_TRAFFIC = {1: 1.4827e9, 2: None, 3: None}   # fused_chain_kernel, capture of the current kernel
+NCU_TRAFFIC = {1: 1.4825e9, 2: None, 3: None}   # fused_chain_kernel, capture of the current kernel
 N_TRIALS = 32           # distinct (fill, block, draft) inputs cycled through the steps
 DRAFT_LOGIT_STD = 1.0   # target-independent drafter: q = softmax(N(0, std^2))
 
