@@ -47,3 +47,31 @@ def test_random_chain_and_tree_calls(sweep_seed):
         paths["whole_chain_kernel" if gpu["launches"] < 20 else "per_projection"] += 1
     print("sweep", sweep_seed, paths)
     assert min(paths.values()) > 0          # the sweep reaches both kinds of call and both kernel paths
+
+
+def test_random_relaxed_and_ragged_calls():
+    """Relaxed acceptance with 1-64 neighbours and thresholds from 0 to infinity, ragged draft
+    counts (including images with no draft at all), up to five images."""
+    from vvs_synth.configs import MODE_RELAXED, MODE_STRICT
+    rng = np.random.default_rng(3)
+    n_relaxed = 0
+    for i in range(16):
+        ms = XL_SMALL if rng.random() < 0.7 else B7_SMALL
+        n_images, n_cfg = int(rng.integers(1, 6)), int(rng.integers(1, 3))
+        f, k = int(rng.integers(1, 4)), int(rng.integers(1, 13))
+        t_len = f + k
+        fills = [int(x) for x in rng.integers(0, ms.s_max - t_len + 1, size=n_images)]
+        relaxed = rng.random() < 0.6
+        nbr_k = int(rng.choice([1, 4, 16, 64])) if relaxed else 1
+        delta = float(rng.choice([0.0, 0.05, 0.3, np.inf])) if relaxed else float("inf")
+        n_draft = [int(x) for x in rng.integers(0, k + 1, size=n_images)]
+        case = H.build_case(ms, 9000 + i, n_images, n_cfg, f, k, fills, cfg_scale=2.0 if n_cfg == 2 else 1.0,
+                            mode=MODE_RELAXED if relaxed else MODE_STRICT, nbr_k=nbr_k, delta=delta,
+                            q_noise=float(rng.choice([0.3, 1.0, 2.5])), n_draft=n_draft)
+        run = H.GpuRunner(ms, case["w"], n_images * n_cfg, t_len, max_nbr_k=nbr_k)
+        gpu = run.verify(case)
+        _check_end_to_end(case, gpu, H.run_oracle(case))
+        assert (gpu["accept_len"] <= np.asarray(n_draft)).all()
+        run.close()
+        n_relaxed += int(relaxed)
+    assert 0 < n_relaxed < 16
