@@ -78,3 +78,17 @@ def test_config1_full_shape_candidate_tree():
     _check_tree(case, gpu, ora)
     print("configs[1] tree: accept path", gpu["accept_path"][0][:gpu["accept_len"][0]], "oracle", ora["accept_path"])
     run.close()
+
+
+@pytest.mark.parametrize("fill", [1, 583])
+def test_config1_full_shape_cache_edges(fill):
+    """Full depth with an almost empty cache (one 128-key chunk, 40 attention items) and with a
+    cache that the block fills exactly (five chunks, 200 items: two per CTA for a third of them)."""
+    wl = CONFIGS[1]
+    assert fill + 9 <= wl.shape.s_max
+    case = H.build_case(wl.shape, wl.seed + fill, 1, 2, 1, 8, [fill], cfg_scale=wl.cfg_scale, q_noise=0.3)
+    run = H.GpuRunner(wl.shape, case["w"], 2, 9)
+    gpu = run.verify(case)
+    assert gpu["launches"] < 40
+    _check_end_to_end(case, gpu, H.run_oracle(case))
+    run.close()
