@@ -199,7 +199,7 @@ def run_ours(args) -> None:
             hk, hv = gen.make_kv_row(ms, seed, row)
             kv_k[:, row].copy_(dev(hk))
             kv_v[:, row].copy_(dev(hv))
-    ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, wl.nbr_k))
+    ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, wl.nbr_k, deterministic=bool(args.deterministic)))
     vb.vvs_bind_weights(ctx, wd)
     if relaxed:
         rp, col = gen.neighbour_csr(gen.make_codebook(seed, ms.vocab, wl.latent_dim), wl.nbr_k)
@@ -750,6 +750,8 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3, 4, 5, 6])
+    ap.add_argument("--deterministic", type=int, default=0, choices=[0, 1],
+                    help="1: fixed-order sums (bitwise repeatable), 0: arrival-order split-K sums (faster)")
     ap.add_argument("--cpu-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -14,7 +14,8 @@
  *
  * General rules
  *   - Every function returns VVS_OK (0) or a negative vvs_status.  Host-side argument errors
- *     are returned before anything is launched.  No exceptions, no global state.
+ *     are returned before anything is launched.  No exceptions.  Process-wide state is limited
+ *     to per-device kernel attributes set once and the scratch array of vvs_decide_noalloc.
  *   - "device" pointers are CUDA device memory of the context's GPU, owned by the caller,
  *     16-byte aligned unless stated otherwise.  "host" pointers are ordinary host memory.
  *     The library never frees caller memory and keeps no reference to host arrays after a
@@ -97,6 +98,17 @@ typedef struct vvs_model_desc {
   int32_t max_nbr_k;     /* largest neighbour count k in relaxed mode (>= 1) */
   float rms_eps;
   float rope_base;
+  int32_t deterministic; /* bf16 contexts, calls of at most 32 block tokens (n_images * n_cfg * T):
+                            1 = every sum of the decoder is taken in a fixed order, so the same call
+                                gives the same bits every time (target_probs, hidden, the appended
+                                K / V rows and hence next_token); vvs_bind_weights then keeps a private
+                                re-packed copy of the layer weights (as many bytes again, device memory);
+                            0 = split-K partial sums are added in L2 in arrival order: faster (see
+                                the measured numbers in the repository's notes), the last bits of the
+                                logits differ from run to run, and a residual sample over many nearly
+                                equally likely codes need not repeat.
+                            Calls of more than 32 block tokens use arrival-order sums in either mode;
+                            float32 contexts are always repeatable. */
 } vvs_model_desc;
 
 /* Per-layer weights, device, type T.  Projection matrices are [out_features, in_features]
@@ -128,7 +140,10 @@ int vvs_destroy(vvs_ctx* ctx);
 /* Scratch bytes vvs_create will allocate for this description (host computation only). */
 int vvs_workspace_bytes(const vvs_model_desc* desc, size_t* out_bytes);
 
-/* Bind caller-owned weights.  Checks non-NULL and 16-byte alignment (VVS_ERR_ALIGN). */
+/* Bind caller-owned weights.  Checks non-NULL and 16-byte alignment (VVS_ERR_ALIGN).  Contexts
+ * created with deterministic = 1 also build their re-packed copy of the layer weights here (a
+ * device allocation of the layers' size and a one-time packing kernel; synchronises the device);
+ * the caller's layer weights are still read by calls of more than 32 block tokens. */
 int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w);
 
 /* Bind the latent-space neighbour table used by relaxed acceptance (Sec. 2, LANTERN rule):
@@ -204,7 +219,12 @@ typedef struct vvs_verify_out {
                            point to the nearest CDF bin edge as a fraction of the total mass */
 } vvs_verify_out;
 
-/* The verification step.  Steps: embedding gather; n_layers x { RMSNorm, QKV projection,
+/* The verification step.  The first call with a given set of argument and output pointers captures
+ * the step into a CUDA graph (a few milliseconds of host time, graph memory allocated by the
+ * runtime); later calls with the same pointers replay it, so a decode loop should reuse its
+ * buffers (up to 64 distinct argument sets are kept).  A call made while `stream` is itself being
+ * captured is enqueued directly.
+ * Steps: embedding gather; n_layers x { RMSNorm, QKV projection,
  * RoPE, KV append, block-vs-cache attention causal inside the block, output projection,
  * RMSNorm, SwiGLU MLP }; final RMSNorm (= features); LM head over the codebook rows; guidance;
  * softmax; strict min(1, p/q) or relaxed min(1, P_A/q) acceptance with the accepted-prefix

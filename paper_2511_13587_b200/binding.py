@@ -30,7 +30,8 @@ class vvs_model_desc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "d_model", "n_heads", "head_dim", "d_ff", "vocab", "vocab_offset", "lm_rows",
         "tok_rows", "s_max", "rope_mode", "rope_grid_w", "n_prefix", "dtype", "max_rows",
-        "max_block", "max_nbr_k")] + [("rms_eps", C.c_float), ("rope_base", C.c_float)]
+        "max_block", "max_nbr_k")] + [("rms_eps", C.c_float), ("rope_base", C.c_float),
+                                      ("deterministic", C.c_int32)]
 
 
 class vvs_layer_weights(C.Structure):
@@ -130,7 +131,8 @@ def _stream(stream):
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 
-def make_desc(shape, max_rows: int, max_block: int, max_nbr_k: int = 1) -> vvs_model_desc:
+def make_desc(shape, max_rows: int, max_block: int, max_nbr_k: int = 1,
+              deterministic: bool = True) -> vvs_model_desc:
     """Fill a vvs_model_desc from any object with the ModelShape attribute names."""
     d = vvs_model_desc()
     for name in ("n_layers", "d_model", "n_heads", "head_dim", "d_ff", "vocab", "vocab_offset",
@@ -139,6 +141,7 @@ def make_desc(shape, max_rows: int, max_block: int, max_nbr_k: int = 1) -> vvs_m
     d.rms_eps = float(shape.rms_eps)
     d.rope_base = float(shape.rope_base)
     d.max_rows, d.max_block, d.max_nbr_k = int(max_rows), int(max_block), int(max_nbr_k)
+    d.deterministic = 1 if deterministic else 0
     return d
 
 

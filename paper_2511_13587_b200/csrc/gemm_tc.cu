@@ -303,9 +303,13 @@ __global__ void rope_table_kernel(const int32_t* __restrict__ cache_len, const f
                                   const int32_t* __restrict__ tree_parent, int n_images, int n_forced,
                                   int32_t* __restrict__ slot_pos, uint32_t* __restrict__ anc_mask,
                                   float* __restrict__ rope_cos, float* __restrict__ rope_sin, int t_len, int hd,
-                                  int s_max, int rope_mode, int grid_w, int n_prefix, int32_t* status) {
+                                  int s_max, int rope_mode, int grid_w, int n_prefix, int32_t* status,
+                                  unsigned* clear_words, int n_clear) {
   __shared__ int s_depth;
   const int m = blockIdx.x, r = m / t_len, t = m % t_len;
+  // the stage counters of the chain kernel that follows in the stream start from zero
+  if (blockIdx.x == 0)
+    for (int i = threadIdx.x; i < n_clear; i += blockDim.x) clear_words[i] = 0u;
   const int fill = cache_len[r];
   const bool ok = fill >= 0 && fill + t_len <= s_max;
   if (!ok && threadIdx.x == 0) atomicOr(status, VVS_DEV_CACHE_OVERFLOW);
@@ -480,11 +484,12 @@ int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStr
 }
 
 void launch_rope_table(const int32_t* cache_len, const int32_t* tree_parent, int n_images, int n_forced,
-                       const Workspace& ws, const vvs_model_desc& md, int n_rows, int t_len, cudaStream_t s) {
+                       const Workspace& ws, const vvs_model_desc& md, int n_rows, int t_len, cudaStream_t s,
+                       unsigned* clear_words, int n_clear) {
   rope_table_kernel<<<n_rows * t_len, 64, 0, s>>>(cache_len, ws.rope_inv_freq, tree_parent, n_images, n_forced,
                                                   ws.slot_pos, ws.anc_mask, ws.rope_cos, ws.rope_sin, t_len,
                                                   md.head_dim, md.s_max, md.rope_mode, md.rope_grid_w, md.n_prefix,
-                                                  ws.status);
+                                                  ws.status, clear_words, n_clear);
 }
 
 }  // namespace vvs

@@ -60,6 +60,13 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
       c.take(ws.chain_gu, (size_t)2 * 32 * 2 * ff * 4);
       c.take(ws.chain_ss, (size_t)2 * d.n_layers * 32 * 4);
       c.take(ws.chain_sync, 256);
+      c.take(ws.cs_xn1, (size_t)32 * dm * 2);
+      c.take(ws.cs_xn2, (size_t)32 * dm * 2);
+      c.take(ws.cs_attn, (size_t)32 * dm * 2);
+      c.take(ws.cs_act, (size_t)32 * ff * 2);
+      c.take(ws.cs_ss1, (size_t)(dm / 16 + 1) * 32 * 4);
+      c.take(ws.cs_ss2, (size_t)(dm / 16 + 1) * 32 * 4);
+      c.take(ws.cs_flags, chain_stream_flag_words(d) * 4);
     }
   }
   // full logits exist only on the generic path (float32 contexts, or bf16 ones forced onto it)
@@ -91,6 +98,7 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
 int check_desc(const vvs_model_desc* d) {
   if (!d) return VVS_ERR_INVALID_ARG;
   if (d->dtype != VVS_DTYPE_FP32 && d->dtype != VVS_DTYPE_BF16) return VVS_ERR_INVALID_ARG;
+  if (d->deterministic != 0 && d->deterministic != 1) return VVS_ERR_INVALID_ARG;
   if (d->rope_mode < VVS_ROPE_NONE || d->rope_mode > VVS_ROPE_2D_GRID) return VVS_ERR_INVALID_ARG;
   if (d->n_layers < 0 || d->d_model <= 0 || d->vocab <= 0 || d->vocab_offset < 0) return VVS_ERR_SHAPE;
   if (d->lm_rows < d->vocab_offset + d->vocab) return VVS_ERR_SHAPE;
@@ -344,6 +352,33 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   base.kv_rows = a->kv_rows; base.t_len = Tn; base.act = act; base.ff = ff;
 
   int rc = VVS_OK;
+  if (ctx->use_chain && md.deterministic && ctx->cs_packed && chain_stream_applicable(md, R, Tn)) {
+    // at most 32 tokens: embedding and every decoder layer run as one persistent dataflow kernel
+    CUtensorMap ck, cv;
+    const uint32_t kb = (uint32_t)chain_stream_kb(md);
+    if (make_tmap_bf16_2d(&ck, kv_k, kv_total_rows, (uint64_t)md.head_dim, kb) != VVS_OK ||
+        make_tmap_bf16_2d(&cv, kv_v, kv_total_rows, (uint64_t)md.head_dim, kb) != VVS_OK)
+      return VVS_ERR_CUDA;
+    ChainStreamArgs cs{};
+    cs.md = &md; cs.n_rows = R; cs.n_images = B; cs.t_len = Tn; cs.kv_rows = a->kv_rows;
+    cs.plan = &ctx->cs_plan; cs.d_plan = ctx->cs_d_plan; cs.packed = ctx->cs_packed;
+    cs.norms_host = ctx->chain_norms.data();
+    cs.tok_emb = static_cast<const T*>(ctx->tok_emb); cs.block = a->block;
+    cs.x = ws.x; cs.xn1 = static_cast<T*>(ws.cs_xn1); cs.xn2 = static_cast<T*>(ws.cs_xn2); cs.qbuf = q;
+    cs.attn = static_cast<T*>(ws.cs_attn); cs.act = static_cast<T*>(ws.cs_act);
+    cs.ss1 = ws.cs_ss1; cs.ss2 = ws.cs_ss2;
+    cs.cache_len = a->cache_len; cs.kv_k = kv_k; cs.kv_v = kv_v; cs.tm_k = &ck; cs.tm_v = &cv;
+    cs.slot_pos = ws.slot_pos; cs.anc_mask = ws.anc_mask; cs.rope_cos = ws.rope_cos; cs.rope_sin = ws.rope_sin;
+    cs.flags = ws.cs_flags; cs.status = ws.status;
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_table(a->cache_len, a->tree_parent, B, a->n_forced, ws, md, R, Tn, s,
+                                                 ws.cs_flags, (int)chain_stream_flag_words(md)));
+    VVS_LAUNCH(VVS_PROF_CHAIN, rc = launch_chain_stream(cs, s));
+    if (rc != VVS_OK) return rc;
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
+    if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
+    if (a->tree_parent) return run_tree_decisions(ctx, hid, a, o, s);
+    return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
+  }
   if (ctx->use_chain && fused_chain_applicable(md, R, Tn)) {
     // at most 32 tokens: the whole decoder chain runs as one persistent kernel
     FusedChainArgs fc{};
@@ -577,6 +612,10 @@ int vvs_create(const vvs_model_desc* desc, vvs_ctx** out) {
   if (cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess ||
       ctx->n_sms < 1)
     ctx->n_sms = 148;
+  if (ctx->tensor_core_path && desc->n_layers > 0 && chain_stream_configure() != VVS_OK) {
+    cudaGetLastError();
+    ctx->use_chain = false;
+  }
   *out = ctx;
   return VVS_OK;
 }
@@ -593,6 +632,8 @@ int vvs_destroy(vvs_ctx* ctx) {
   drop_graphs(ctx);
   if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
   if (ctx->arena) cudaFree(ctx->arena);
+  if (ctx->cs_packed) cudaFree(ctx->cs_packed);
+  if (ctx->cs_d_plan) cudaFree(ctx->cs_d_plan);
   delete[] ctx->layers;
   delete[] ctx->layer_maps;
   delete ctx;
@@ -649,6 +690,24 @@ int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w) {
       if (cudaMemcpy(ctx->ws.chain_wmaps, ctx->layer_maps, (size_t)n * sizeof(LayerMaps),
                      cudaMemcpyHostToDevice) != cudaSuccess)
         return VVS_ERR_CUDA;
+      // private copy of the layer weights in the streaming order of the chain kernel
+      if (ctx->cs_packed) { cudaFree(ctx->cs_packed); ctx->cs_packed = nullptr; }
+      if (ctx->cs_d_plan) { cudaFree(ctx->cs_d_plan); ctx->cs_d_plan = nullptr; }
+      if (ctx->use_chain && md.deterministic && chain_stream_applicable(md, 1, 1) &&
+          chain_stream_plan(md, ctx->n_sms, ctx->cs_plan)) {
+        const size_t pbytes = chain_stream_packed_bytes(md, ctx->cs_plan);
+        const size_t plbytes = ctx->cs_plan.cta.size() * sizeof(ChainCtaPlan);
+        if (cudaMalloc(&ctx->cs_packed, pbytes) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&ctx->cs_d_plan), plbytes) != cudaSuccess) {
+          cudaGetLastError();
+          if (ctx->cs_packed) { cudaFree(ctx->cs_packed); ctx->cs_packed = nullptr; }
+          return VVS_ERR_NOMEM;
+        }
+        if (cudaMemcpy(ctx->cs_d_plan, ctx->cs_plan.cta.data(), plbytes, cudaMemcpyHostToDevice) != cudaSuccess)
+          return VVS_ERR_CUDA;
+        rc = chain_stream_pack(md, ctx->cs_plan, ctx->cs_d_plan, ctx->layers, ctx->cs_packed, nullptr);
+        if (rc != VVS_OK || cudaDeviceSynchronize() != cudaSuccess) return VVS_ERR_CUDA;
+      }
     }
   }
   drop_graphs(ctx);  // captured steps hold the old pointers

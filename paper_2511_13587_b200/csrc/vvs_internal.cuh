@@ -63,6 +63,15 @@ struct Workspace {
   float* chain_gu = nullptr;     // [2][32, 2ff] fp32 split-K sums of gate | up
   float* chain_ss = nullptr;     // [2 * n_layers][32] sums of squares of the residual rows
   unsigned* chain_sync = nullptr;  // [4] grid-barrier arrivals, epoch base, abort flag
+  // streaming chain kernel (at most 32 block tokens)
+  // stage inputs in B-fragment order (32 tokens x width bf16 each)
+  void* cs_xn1 = nullptr;        // residual * first norm scale
+  void* cs_xn2 = nullptr;        // residual * second norm scale
+  void* cs_attn = nullptr;       // attention output
+  void* cs_act = nullptr;        // silu(gate) * up
+  float* cs_ss1 = nullptr;       // [d / 16][32] sums of squares of the residual rows per 16-column tile
+  float* cs_ss2 = nullptr;
+  unsigned* cs_flags = nullptr;  // [n_layers * 5 + 2] stage arrival counters, embedding counter, abort word
   int32_t* status = nullptr; // device status word
 };
 
@@ -87,6 +96,26 @@ struct GraphEntry {
 };
 }  // namespace vvs
 
+namespace vvs {
+// Share of the decoder weights one CTA of the streaming chain kernel owns, the same in every layer:
+// contiguous ranges of 16-row tiles of the QKV, output, gate / up (pairs) and down projections,
+// its rank in the order attention items are dealt out, and the byte offset of its stream inside a
+// layer's packed block.
+struct ChainCtaPlan {
+  int t0[4];
+  int n[4];
+  int att_rank;
+  int pad;
+  unsigned long long off;
+};
+struct ChainStreamPlan {
+  int grid = 0;
+  std::vector<ChainCtaPlan> cta;
+  unsigned long long layer_bytes = 0;
+  int n_prod[5] = {0, 0, 0, 0, 0};   // CTAs with work in each stage (attention: set per call)
+};
+}  // namespace vvs
+
 struct vvs_ctx {
   vvs_model_desc desc;
   vvs::Workspace ws;
@@ -102,6 +131,9 @@ struct vvs_ctx {
   bool use_chain = true;             // whole-chain persistent kernel for calls of at most 32 tokens
   vvs::LayerMaps* layer_maps = nullptr;  // host array [n_layers]
   std::vector<const __nv_bfloat16*> chain_norms;  // host [n_layers][2] norm-scale pointers
+  vvs::ChainStreamPlan cs_plan;        // streaming chain kernel: split of the weights over the CTAs
+  void* cs_packed = nullptr;           // device: private re-packed copy of the layer weights
+  vvs::ChainCtaPlan* cs_d_plan = nullptr;  // device copy of cs_plan.cta
   CUtensorMap lm_map;
   int n_sms = 148;
   // CUDA-graph replay of vvs_verify (one graph per distinct argument set, small LRU cache)
@@ -181,7 +213,7 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
 int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStream_t s);
 void launch_rope_table(const int32_t* cache_len, const int32_t* tree_parent, int n_images, int n_forced,
                        const Workspace& ws, const vvs_model_desc& md, int n_rows,
-                       int t_len, cudaStream_t s);
+                       int t_len, cudaStream_t s, unsigned* clear_words = nullptr, int n_clear = 0);
 
 // ---- tensor-core attention, attention_tc.cu ----------------------------------------------------------
 struct AttentionTcArgs {
@@ -258,6 +290,37 @@ void launch_tree_commit(void* kv_k, void* kv_v, const int32_t* cache_len, const 
 bool fused_chain_applicable(const vvs_model_desc& md, int n_rows, int t_len);
 size_t fused_chain_smem_bytes(const vvs_model_desc& md, int t_len, int* w_stages);
 int launch_fused_chain(const FusedChainArgs& a, cudaStream_t s);
+
+// ---- streaming chain kernel, chain_stream.cu ------------------------------------------------------
+struct ChainStreamArgs {
+  const vvs_model_desc* md;
+  int n_rows, n_images, t_len, kv_rows;
+  const ChainStreamPlan* plan;
+  const ChainCtaPlan* d_plan;           // device
+  const void* packed;                   // device
+  const __nv_bfloat16* const* norms_host;  // HOST array [n_layers][2] of device pointers
+  const __nv_bfloat16* tok_emb;
+  const int32_t* block;
+  float* x;
+  __nv_bfloat16 *xn1, *xn2, *qbuf, *attn, *act;
+  float *ss1, *ss2;
+  const int32_t* cache_len;
+  __nv_bfloat16* kv_k; __nv_bfloat16* kv_v;
+  const CUtensorMap* tm_k;              // host: cache as [rows, head_dim], box {64, chain_stream_kb()}
+  const CUtensorMap* tm_v;
+  const int32_t* slot_pos; const uint32_t* anc_mask; const float* rope_cos; const float* rope_sin;
+  unsigned* flags;                      // zero at launch
+  int32_t* status;
+};
+bool chain_stream_applicable(const vvs_model_desc& md, int n_rows, int t_len);
+bool chain_stream_plan(const vvs_model_desc& md, int grid, ChainStreamPlan& out);
+size_t chain_stream_packed_bytes(const vvs_model_desc& md, const ChainStreamPlan& plan);
+int chain_stream_pack(const vvs_model_desc& md, const ChainStreamPlan& plan, const ChainCtaPlan* d_plan,
+                      const Layer* layers, void* packed, cudaStream_t s);
+int chain_stream_kb(const vvs_model_desc& md);
+size_t chain_stream_flag_words(const vvs_model_desc& md);
+int chain_stream_configure();
+int launch_chain_stream(const ChainStreamArgs& a, cudaStream_t s);
 
 // ---- decision stage, kernels_decide.cu -----------------------------------------------------
 struct DecideParams {

@@ -93,11 +93,12 @@ def weights_to_dev(w: dict) -> dict:
 class GpuRunner:
     """Owns a library context plus device copies of one case's weights."""
 
-    def __init__(self, ms: ModelShape, w: dict, max_rows: int, max_block: int, max_nbr_k: int = 1):
+    def __init__(self, ms: ModelShape, w: dict, max_rows: int, max_block: int, max_nbr_k: int = 1,
+                 deterministic: bool = True):
         from paper_2511_13587_b200 import binding as vb
         self.vb = vb
         self.ms = ms
-        self.ctx = vb.vvs_create(vb.make_desc(ms, max_rows, max_block, max_nbr_k))
+        self.ctx = vb.vvs_create(vb.make_desc(ms, max_rows, max_block, max_nbr_k, deterministic))
         self.wd = weights_to_dev(w)
         vb.vvs_bind_weights(self.ctx, self.wd)
 

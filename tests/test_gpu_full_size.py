@@ -16,26 +16,31 @@ from vvs_synth.configs import B7, CONFIGS, MODE_RELAXED, XL
 pytestmark = pytest.mark.gpu
 
 
-def test_config1_full_llamagen_xl_shape():
+@pytest.mark.parametrize("deterministic", [True, False])
+def test_config1_full_llamagen_xl_shape(deterministic):
     """Fill 477 needs four 128-key chunks per (sequence, head), i.e. more attention work items
     than SMs, and the block's own rows straddle no chunk boundary; the small-shape tests cover
-    the other fills."""
+    the other fills.  Both whole-chain kernels: fixed-order sums and arrival-order sums."""
     wl, fill = CONFIGS[1], 477
     case = H.build_case(wl.shape, wl.seed + fill, 1, 2, 1, 8, [fill], cfg_scale=wl.cfg_scale, q_noise=0.3)
-    run = H.GpuRunner(wl.shape, case["w"], 2, 9)
+    run = H.GpuRunner(wl.shape, case["w"], 2, 9, deterministic=deterministic)
     gpu = run.verify(case)
     assert gpu["launches"] < 40            # the whole-chain kernel ran, not one kernel per projection
     ora = H.run_oracle(case)
     _check_end_to_end(case, gpu, ora)
     print("configs[1] full size: accept_len", gpu["accept_len"], "oracle", ora["accept_len"])
-    # The configuration the benchmark times does not ask for probabilities.  Split-K sums are
-    # added in L2 in arrival order, so two runs differ in the last bits of the logits: the accepted
-    # prefix (margins far above that) must repeat, the residual sample over 16384 almost equally
-    # likely codes need not and is only checked for range.
+    # The configuration the benchmark times does not ask for probabilities.  With fixed-order sums
+    # the step repeats bit for bit, so the sampled token is the one of the checked call.  With
+    # arrival-order sums two runs differ in the last bits of the logits: the accepted prefix
+    # (margins far above that) must repeat, the residual sample over 16384 almost equally likely
+    # codes need not and is only checked for range.
     gpu2 = run.verify(case, want_probs=False)
     np.testing.assert_array_equal(gpu2["accept_len"], gpu["accept_len"])
     ms = wl.shape
     assert ((gpu2["next_token"] >= ms.vocab_offset) & (gpu2["next_token"] < ms.vocab_offset + ms.vocab)).all()
+    if deterministic:
+        np.testing.assert_array_equal(gpu2["next_token"], gpu["next_token"])
+        np.testing.assert_array_equal(gpu2["hidden"], gpu["hidden"])
     run.close()
 
 

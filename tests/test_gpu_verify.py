@@ -81,13 +81,14 @@ def test_config0_tiny_fp32_strict():
         run.close()
 
 
+@pytest.mark.parametrize("deterministic", [True, False])
 @pytest.mark.parametrize("n_images,fills", [(1, [288]), (3, [1, 575, 130])])
-def test_xl_shape_small_bf16_cfg(n_images, fills):
+def test_xl_shape_small_bf16_cfg(n_images, fills, deterministic):
     """LlamaGen-XL structure (2-D grid rope, 1 prefix token, guidance 2.0, K = 8) at reduced
     width/depth; an extra unused cache row must stay untouched."""
     ms = XL_SMALL
     case = H.build_case(ms, 11 + n_images, n_images, 2, 1, 8, fills, kv_rows=2 * n_images + 1)
-    run = H.GpuRunner(ms, case["w"], 2 * n_images, 9)
+    run = H.GpuRunner(ms, case["w"], 2 * n_images, 9, deterministic=deterministic)
     gpu = run.verify(case)
     ora = H.run_oracle(case)
     _check_end_to_end(case, gpu, ora)
@@ -115,11 +116,12 @@ def test_relaxed_acceptance_bf16(delta):
     run.close()
 
 
-def test_7b_shape_small_bf16():
+@pytest.mark.parametrize("deterministic", [True, False])
+def test_7b_shape_small_bf16(deterministic):
     """7B structure: head_dim 128, 1-D rope, codebook inside a larger vocabulary."""
     ms = B7_SMALL
     case = H.build_case(ms, 31, 1, 2, 1, 8, [300])
-    run = H.GpuRunner(ms, case["w"], 2, 9)
+    run = H.GpuRunner(ms, case["w"], 2, 9, deterministic=deterministic)
     gpu = run.verify(case)
     ora = H.run_oracle(case)
     _check_end_to_end(case, gpu, ora)
@@ -143,12 +145,13 @@ def test_per_projection_kernels_head_dims_and_long_blocks(ms, n_images, n_forced
     run.close()
 
 
-def test_ragged_drafts_forced_prefix_and_cache_edges():
+@pytest.mark.parametrize("deterministic", [True, False])
+def test_ragged_drafts_forced_prefix_and_cache_edges(deterministic):
     """n_draft below K (including 0), two forced rows, an empty cache and a cache that the block
     fills to capacity."""
     ms = replace(XL_SMALL, s_max=64)
     case = H.build_case(ms, 41, 4, 2, 2, 6, [0, 64 - 8, 5, 17], n_draft=[6, 3, 0, 1], q_noise=0.5)
-    run = H.GpuRunner(ms, case["w"], 8, 8)
+    run = H.GpuRunner(ms, case["w"], 8, 8, deterministic=deterministic)
     gpu = run.verify(case)
     ora = H.run_oracle(case)
     _check_end_to_end(case, gpu, ora)
@@ -210,13 +213,29 @@ def test_device_side_checks_report_instead_of_faulting():
 
 
 def test_repeatable_across_calls():
-    """Two calls on the same inputs: the float32 context is bitwise repeatable; the bf16 context
-    adds split-K partial sums with float atomics, so its low bits (and, through bf16 rounding of
+    """Two calls on the same inputs.  A bf16 context created with deterministic = 1 (the default of
+    the binding) takes every sum in a fixed order: all outputs and the appended K / V rows repeat bit
+    for bit, with and without the probabilities being written out.  With deterministic = 0 split-K
+    partial sums are added with float atomics, so the low bits (and, through bf16 rounding of
     activations, ~1e-2 of a probability) may move, but every decision must replay exactly on the
-    probabilities of its own call."""
+    probabilities of its own call.  The float32 context is bitwise repeatable."""
     ms = XL_SMALL
     case = H.build_case(ms, 71, 2, 2, 1, 8, [50, 400])
-    run = H.GpuRunner(ms, case["w"], 4, 9)
+    for n_images, fills in ((1, [288]), (1, [50])):
+        c1 = H.build_case(ms, 71 + fills[0], n_images, 2, 1, 8, fills)
+        run = H.GpuRunner(ms, c1["w"], 2 * n_images, 9, deterministic=True)
+        a = run.verify(c1)
+        b = run.verify(c1)
+        assert a["launches"] < 20            # the whole-chain kernel (at most 32 block tokens)
+        for key in ("accept_len", "next_token", "accept_mask", "new_len", "target_probs", "hidden", "kv_k", "kv_v"):
+            np.testing.assert_array_equal(a[key], b[key], err_msg=key)
+        c_ = run.verify(c1, want_probs=False)
+        d_ = run.verify(c1, want_probs=False)
+        for key in ("accept_len", "next_token", "new_len", "hidden"):
+            np.testing.assert_array_equal(c_[key], d_[key], err_msg=key)
+        np.testing.assert_array_equal(c_["accept_len"], a["accept_len"])
+        run.close()
+    run = H.GpuRunner(ms, case["w"], 4, 9, deterministic=False)
     a = run.verify(case)
     b = run.verify(case)
     np.testing.assert_allclose(a["target_probs"], b["target_probs"], rtol=5e-2, atol=1e-7)
