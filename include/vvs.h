@@ -266,6 +266,8 @@ int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, 
  * Capacity (larger sizes return VVS_ERR_SHAPE): n_images <= 64, n_draft_max <= 16,
  * nbr_k <= 64, vocab <= 65536.
  *
+ * Chains only: args->tree_parent and out->accept_path must be NULL (VVS_ERR_INVALID_ARG).
+ *
  * Arguments are those of vvs_decide, with what a context would carry passed explicitly: vocab,
  * vocab_offset, and the CSR neighbour table (device int32, may be NULL in strict mode).
  * status_bits: optional device int32 the VVS_DEV_* bits are OR-ed into (caller clears it);
@@ -355,6 +357,15 @@ int vvs_select_unverified(vvs_ctx* ctx, const int32_t* paths, const int32_t* pat
 /* Synchronise `stream`, copy the device status word to *out_bits (VVS_DEV_* bits) and clear
  * it.  Returns VVS_ERR_DEVICE_TIMEOUT / VVS_ERR_DEVICE_BOUNDS if such a bit was set. */
 int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits);
+
+/* Self-test of the failure path of the library's bounded device-side waits (no counterpart in the
+ * paper).  Launches one tiny kernel in which a thread waits, through the same helpers the tensor-core
+ * kernels and the streaming chain kernel use but with a limit of a few hundred polls, on barriers
+ * nobody ever arrives on.  Each wait must give up and return: gave_up[0] / gave_up[1] (host int32[2])
+ * are set to 1 for the two helpers, the VVS_DEV_TIMEOUT bit is left in the device status word (so
+ * the next vvs_device_status returns VVS_ERR_DEVICE_TIMEOUT and clears it), and the context stays
+ * usable.  Synchronises `stream`.  Nothing in it can hang: the waits are the bounded ones. */
+int vvs_selftest_bounded_wait(vvs_ctx* ctx, void* stream, int32_t* gave_up);
 
 /* Number of kernels the last vvs_verify / vvs_epilogue call on this context launched. */
 int vvs_last_launch_count(const vvs_ctx* ctx);

@@ -79,6 +79,7 @@ lib.vvs_decide.restype = C.c_int
 lib.vvs_decide_noalloc.argtypes = [_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P,
                                    C.POINTER(vvs_verify_args), C.POINTER(vvs_verify_out), _P, _P]
 lib.vvs_decide_noalloc.restype = C.c_int
+lib.vvs_selftest_bounded_wait.argtypes = [_P, _P, C.POINTER(C.c_int32)]
 lib.vvs_feature_cache_reset.argtypes = [_P, C.POINTER(vvs_fcache), _P]
 lib.vvs_feature_cache_store.argtypes = [_P, C.POINTER(vvs_fcache), _P, C.c_int32, _P, _P, _P]
 lib.vvs_feature_cache_fetch.argtypes = [_P, C.POINTER(vvs_fcache), _P, C.c_int32, _P, C.c_int32,
@@ -237,17 +238,25 @@ def vvs_decide_noalloc(*, target_probs, vocab, vocab_offset, n_rows_per_seq, fir
                        n_images, n_draft_max, draft_probs, uniforms, accept_len, next_token,
                        nbr_row_ptr=None, nbr_col=None, n_draft=None, mode=VVS_MODE_STRICT, nbr_k=1,
                        delta=float("inf"), accept_mask=None, margins=None, status_bits=None,
-                       stream=None) -> None:
+                       tree_parent=None, accept_path=None, stream=None) -> None:
     """vvs_decide for callers that must not allocate device memory: no context, scratch in a fixed
-    device array inside the library (limits: 64 images, 16 drafts, 64 neighbours, vocab 65536).
-    Calls on one device share that array and must not overlap on the GPU."""
+    device array inside the library (limits: 64 images, 16 drafts, 64 neighbours, vocab 65536;
+    chains only: tree_parent / accept_path are refused).  Calls on one device share that array
+    and must not overlap on the GPU."""
     a = _args(n_images, 1, 1, n_draft_max, None, n_draft, None, None, 0, None, None, draft_probs,
-              uniforms, 1.0, 1.0, mode, nbr_k, delta)
-    o = _out(accept_len, next_token, None, None, accept_mask, None, None, margins)
+              uniforms, 1.0, 1.0, mode, nbr_k, delta, tree_parent)
+    o = _out(accept_len, next_token, None, None, accept_mask, None, None, margins, accept_path)
     _check(lib.vvs_decide_noalloc(_ptr(target_probs), int(vocab), int(vocab_offset), int(n_rows_per_seq),
                                   int(first_row), _ptr(drafts), _ptr(nbr_row_ptr), _ptr(nbr_col),
                                   C.byref(a), C.byref(o), _ptr(status_bits), _stream(stream)),
            "vvs_decide_noalloc")
+
+
+def vvs_selftest_bounded_wait(ctx: int, stream=None):
+    """Runs the bounded-wait self-test kernel; returns the two give-up flags."""
+    out = (C.c_int32 * 2)()
+    _check(lib.vvs_selftest_bounded_wait(ctx, _stream(stream), out), "vvs_selftest_bounded_wait")
+    return int(out[0]), int(out[1])
 
 
 def make_fcache(feat: torch.Tensor, fpos: torch.Tensor, newest: torch.Tensor) -> vvs_fcache:

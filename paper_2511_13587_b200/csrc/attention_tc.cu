@@ -359,20 +359,13 @@ int launch_attention_tc(const AttentionTcArgs& a, cudaStream_t s) {
   cfg.attrs = attr;
   cfg.numAttrs = a.pdl ? 1 : 0;
   cudaError_t e;
-  static bool configured64 = false, configured128 = false;
   if (a.hd == 64) {
-    if (!configured64) {
-      if (cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess)
-        return VVS_ERR_CUDA;
-      configured64 = true;
-    }
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(attention_tc_kernel<64>), smem_max) != cudaSuccess)
+      return VVS_ERR_CUDA;
     e = cudaLaunchKernelEx(&cfg, attention_tc_kernel<64>, p, *a.tm_q, *a.tm_k, *a.tm_v);
   } else {
-    if (!configured128) {
-      if (cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess)
-        return VVS_ERR_CUDA;
-      configured128 = true;
-    }
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(attention_tc_kernel<128>), smem_max) != cudaSuccess)
+      return VVS_ERR_CUDA;
     e = cudaLaunchKernelEx(&cfg, attention_tc_kernel<128>, p, *a.tm_q, *a.tm_k, *a.tm_v);
   }
   return e == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;

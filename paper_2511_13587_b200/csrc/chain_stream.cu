@@ -165,9 +165,10 @@ __device__ __forceinline__ size_t frag_off(int tok, int k, int span_bytes) {
 }
 
 // Bounded wait on an mbarrier phase; once the CTA is in abort mode every wait falls through.
-__device__ __noinline__ void wait_slow(uint64_t* bar, uint32_t parity, volatile int* s_abort, int32_t* status) {
+__device__ __noinline__ void wait_slow(uint64_t* bar, uint32_t parity, volatile int* s_abort, int32_t* status,
+                                       uint32_t limit = kParkedPolls) {
   if (*s_abort) return;
-  for (uint32_t i = 0; i < kParkedPolls; ++i) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait_parked(bar, parity, kParkNs)) return;
     if ((i & 15u) == 15u && *s_abort) return;
   }
@@ -1104,6 +1105,24 @@ chain_pack_kernel(PackLayer wl, const ChainCtaPlan* plans, uint8_t* out_layer, i
   if (pl.n[G_DOWN]) pack_task(G_DOWN, pl.t0[G_DOWN], pl.n[G_DOWN]);
 }
 
+// Self-test of the bounded waits: one thread waits, with a limit of a few hundred polls, on barriers
+// on which nobody ever arrives.  Both helpers must give up, record VVS_DEV_TIMEOUT and return.
+__global__ void bounded_wait_selftest_kernel(int32_t* status, int32_t* report) {
+  __shared__ __align__(8) uint64_t bar[2];
+  __shared__ volatile int s_abort;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar[0], 1);
+    mbar_init(&bar[1], 1);
+    s_abort = 0;
+    fence_barrier_init();
+    const bool got0 = mbar_wait_limited(&bar[0], 0u, 256u);   // the helper of the tcgen05 kernels
+    if (!got0) atomicOr(status, VVS_DEV_TIMEOUT);
+    wait_slow(&bar[1], 0u, &s_abort, status, 64u);            // the helper of the streaming chain kernel
+    report[0] = got0 ? 1 : 0;
+    report[1] = s_abort;
+  }
+}
+
 void geometry(int K, int& spans, int& gsz, int& ngroups) {
   spans = K / 32;
   ngroups = (spans + kGroupSpans - 1) / kGroupSpans;
@@ -1193,14 +1212,16 @@ int chain_stream_pack(const vvs_model_desc& md, const ChainStreamPlan& plan, con
 }
 
 // keys per attention block: K and V of a block share one 20 KB ring slot (8 KB each)
+void launch_bounded_wait_selftest(int32_t* status, int32_t* report, cudaStream_t s) {
+  bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(status, report);
+}
+
 int chain_stream_kb(const vvs_model_desc& md) { return md.head_dim == 64 ? 64 : 32; }
 size_t chain_stream_flag_words(const vvs_model_desc& md) { return (size_t)md.n_layers * N_ST + 2; }
 
 int chain_stream_configure() {
-  if (cudaFuncSetAttribute(chain_stream_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(3)) !=
-          cudaSuccess ||
-      cudaFuncSetAttribute(chain_stream_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(4)) !=
-          cudaSuccess)
+  if (ensure_dynamic_smem(reinterpret_cast<const void*>(chain_stream_kernel<3>), (int)smem_bytes(3)) != cudaSuccess ||
+      ensure_dynamic_smem(reinterpret_cast<const void*>(chain_stream_kernel<4>), (int)smem_bytes(4)) != cudaSuccess)
     return VVS_ERR_CUDA;
   return VVS_OK;
 }

@@ -1048,12 +1048,7 @@ int launch_fused_chain(const FusedChainArgs& a, cudaStream_t s) {
   const size_t smem = fused_chain_smem_bytes(md, a.t_len, &stages);
   if (stages < 3) return VVS_ERR_SHAPE;
   p.n_stages = stages;
-  static size_t configured = 0;
-  if (configured < smem) {
-    if (cudaFuncSetAttribute(fused_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return VVS_ERR_CUDA;
-    configured = smem;
-  }
+  if (ensure_dynamic_smem(reinterpret_cast<const void*>(fused_chain_kernel), (int)smem) != cudaSuccess) return VVS_ERR_CUDA;
   CUtensorMap tk = *a.tm_k, tv = *a.tm_v;
   void* args[] = {&p, &tk, &tv};
   // cooperative launch: all CTAs are resident together, which the grid barriers rely on

@@ -381,12 +381,9 @@ EncodeTiledFn encode_fn() {
 template <int EPI>
 cudaError_t launch_one(const GemmTcPlan& plan, const KernelParams& kp, const CUtensorMap& a, const CUtensorMap& a2,
                        const CUtensorMap& b, int tiles, bool pdl, cudaStream_t s) {
-  static int configured = 0;
-  if (configured < plan.smem_bytes) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         200 * 1024 + 1024);
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(gemm_tc_kernel<EPI>), 200 * 1024 + 1024);
     if (e != cudaSuccess) return e;
-    configured = 200 * 1024 + 1024;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(tiles, plan.splits, plan.passes);

@@ -290,11 +290,7 @@ void launch_attention(const T* q, const T* kv_k, const T* kv_v, const int32_t* c
                       cudaStream_t s) {
   constexpr int kWarps = 4;
   size_t smem = (size_t)kWarps * (md.s_max + md.head_dim) * sizeof(float);
-  static size_t configured = 0;
-  if (smem > 48 * 1024 && smem > configured) {
-    cudaFuncSetAttribute(attention_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    configured = smem;
-  }
+  if (smem > 48 * 1024) ensure_dynamic_smem(reinterpret_cast<const void*>(attention_kernel<T>), (int)smem);
   dim3 grid(md.n_heads, n_rows);
   attention_kernel<T><<<grid, kWarps * 32, smem, s>>>(q, kv_k, kv_v, cache_len, out, md.d_model,
                                                       md.n_heads, md.head_dim, md.s_max, layer,

@@ -273,12 +273,8 @@ int launch_lmhead_tc(const LmHeadArgs& a, cudaStream_t s) {
   while (cols < (uint32_t)nt) cols <<= 1;
   p.tmem_cols = cols;
   const size_t smem = (size_t)stages * stage_bytes + tile_bytes + 1024;
-  static size_t configured = 0;
-  if (configured < smem) {
-    if (cudaFuncSetAttribute(lmhead_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024) != cudaSuccess)
-      return VVS_ERR_CUDA;
-    configured = 226 * 1024;
-  }
+  if (smem > 226 * 1024) return VVS_ERR_SHAPE;
+  if (ensure_dynamic_smem(reinterpret_cast<const void*>(lmhead_tc_kernel), 226 * 1024) != cudaSuccess) return VVS_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((a.v + (int)kTileRows - 1) / (int)kTileRows, 1, 1);
   cfg.blockDim = dim3(128, 1, 1);

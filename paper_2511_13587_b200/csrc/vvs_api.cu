@@ -473,11 +473,19 @@ int enqueue_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out*
 // GPU needs to run them.  Each distinct argument set is therefore captured once into a CUDA graph
 // (on a private stream, so the caller may use the legacy default stream) and replayed afterwards.
 int verify_via_graph(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, cudaStream_t s) {
-  vvs_verify_args ka = *a;
-  ka.cache_len_host = nullptr;  // host-side validation only, not part of the device work
+  // the key is built field by field into zeroed storage: padding bytes of the caller's structs
+  // must not make two equal calls look different
+  vvs_verify_args ka;
+  std::memset(&ka, 0, sizeof(ka));
+  ka.n_images = a->n_images; ka.n_cfg = a->n_cfg; ka.n_forced = a->n_forced; ka.n_draft_max = a->n_draft_max;
+  ka.block = a->block; ka.n_draft = a->n_draft; ka.kv_k = a->kv_k; ka.kv_v = a->kv_v; ka.kv_rows = a->kv_rows;
+  ka.cache_len = a->cache_len;   // cache_len_host: host-side validation only, not part of the device work
+  ka.draft_probs = a->draft_probs; ka.uniforms = a->uniforms; ka.cfg_scale = a->cfg_scale;
+  ka.temperature = a->temperature; ka.mode = a->mode; ka.nbr_k = a->nbr_k; ka.delta = a->delta;
+  ka.tree_parent = a->tree_parent;
   std::vector<unsigned char> key(sizeof(ka) + sizeof(*o));
   std::memcpy(key.data(), &ka, sizeof(ka));
-  std::memcpy(key.data() + sizeof(ka), o, sizeof(*o));
+  std::memcpy(key.data() + sizeof(ka), o, sizeof(*o));   // nine pointers, no padding
   ++ctx->graph_clock;
   for (auto& g : ctx->graphs) {
     if (g.key == key) {
@@ -900,6 +908,21 @@ int vvs_device_status(vvs_ctx* ctx, void* stream, int32_t* out_bits) {
   if (bits & (VVS_DEV_BAD_TOKEN | VVS_DEV_CACHE_OVERFLOW | VVS_DEV_BAD_NEIGHBOUR | VVS_DEV_BAD_ARG))
     return VVS_ERR_DEVICE_BOUNDS;
   return VVS_OK;
+}
+
+int vvs_selftest_bounded_wait(vvs_ctx* ctx, void* stream, int32_t* gave_up) {
+  if (!ctx || !gave_up) return VVS_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // two report words at the end of the status line (the status word itself is the first)
+  int32_t* report = ctx->ws.status + 16;
+  VVS_CUDA_OK(cudaMemsetAsync(report, 0, 2 * sizeof(int32_t), s));
+  launch_bounded_wait_selftest(ctx->ws.status, report, s);
+  int32_t host[2] = {0, 0};
+  VVS_CUDA_OK(cudaMemcpyAsync(host, report, sizeof(host), cudaMemcpyDeviceToHost, s));
+  VVS_CUDA_OK(cudaStreamSynchronize(s));
+  gave_up[0] = host[0] == 0 ? 1 : 0;
+  gave_up[1] = host[1] != 0 ? 1 : 0;
+  return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
 }
 
 int vvs_last_launch_count(const vvs_ctx* ctx) { return ctx ? ctx->launches : 0; }

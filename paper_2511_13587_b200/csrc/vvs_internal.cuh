@@ -6,6 +6,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <map>
+#include <mutex>
+#include <utility>
 #include <vector>
 
 #include "vvs.h"
@@ -17,6 +20,23 @@
   } while (0)
 
 namespace vvs {
+
+// Raises a kernel's dynamic shared-memory limit to at least `bytes` on the CURRENT device.  The
+// attribute is per device: the table of what has been set is keyed by (device, kernel), so a
+// process that creates contexts on several GPUs configures each of them.
+inline cudaError_t ensure_dynamic_smem(const void* kernel, int bytes) {
+  static std::mutex mu;
+  static std::map<std::pair<int, const void*>, int> done;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(mu);
+  int& have = done[std::make_pair(dev, kernel)];
+  if (have >= bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) have = bytes;
+  return e;
+}
 
 // Scratch memory of a context.  Row index m of an activation matrix is r * T + t with
 // r = c * B + b (cond sequences first).  "Decision rows" are (b, t) pairs: index b * T + t.
@@ -321,6 +341,7 @@ int chain_stream_kb(const vvs_model_desc& md);
 size_t chain_stream_flag_words(const vvs_model_desc& md);
 int chain_stream_configure();
 int launch_chain_stream(const ChainStreamArgs& a, cudaStream_t s);
+void launch_bounded_wait_selftest(int32_t* status, int32_t* report, cudaStream_t s);
 
 // ---- decision stage, kernels_decide.cu -----------------------------------------------------
 struct DecideParams {

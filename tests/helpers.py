@@ -52,6 +52,35 @@ def build_case(ms: ModelShape, seed: int, n_images: int, n_cfg: int, n_forced: i
     return case
 
 
+def build_case_independent(ms: ModelShape, seed: int, n_images: int, n_cfg: int, n_forced: int, n_draft_max: int,
+                           fills, cfg_scale: float = 2.0, temperature: float = 1.0, mode: int = MODE_STRICT,
+                           nbr_k: int = 1, delta: float = float("inf"), logit_std: float = 1.0, w=None, kv=None,
+                           call_id: int = 0):
+    """Seeded inputs of one verify call with a drafter that does not look at the target
+    (q = softmax(N(0, logit_std^2)), drafts sampled from q): no teacher-forced oracle passes are
+    needed to build it, which is what makes the full-depth cases of the large workloads affordable.
+    `w` / `kv` may carry weights and caches generated elsewhere (stored bit patterns)."""
+    n_rows = n_images * n_cfg
+    t_len = n_forced + n_draft_max
+    w = gen.make_weights(ms, seed) if w is None else w
+    kv_k, kv_v = gen.make_kv_cache(ms, seed, n_rows) if kv is None else kv
+    fills = np.asarray(fills, dtype=np.int32)
+    cache_len = np.array([fills[r % n_images] for r in range(n_rows)], dtype=np.int32)
+    lo, hi = ms.vocab_offset, ms.vocab_offset + ms.vocab
+    block = np.zeros((n_images, t_len), dtype=np.int32)
+    block[:, :n_forced] = gen.random_tokens(seed, "forced", (n_images, n_forced), lo, hi)
+    q, drafts = gen.independent_draft(seed, call_id, n_images, n_draft_max, ms.vocab, logit_std)
+    block[:, n_forced:] = lo + drafts
+    u = philox.verify_uniforms(seed, call_id, n_images, n_draft_max)
+    case = dict(ms=ms, w=w, kv_k=kv_k, kv_v=kv_v, kv_rows=n_rows, cache_len=cache_len, block=block,
+                draft_probs=q, uniforms=u, n_draft=np.full(n_images, n_draft_max, np.int32), n_images=n_images,
+                n_cfg=n_cfg, n_forced=n_forced, n_draft_max=n_draft_max, cfg_scale=cfg_scale,
+                temperature=temperature, mode=mode, nbr_k=nbr_k, delta=delta, row_ptr=None, col=None)
+    if mode == MODE_RELAXED:
+        case["row_ptr"], case["col"] = gen.neighbour_csr(gen.make_codebook(seed, ms.vocab), nbr_k)
+    return case
+
+
 def run_oracle(case) -> dict:
     c = case
     n_rows = c["n_images"] * c["n_cfg"]
@@ -105,7 +134,7 @@ class GpuRunner:
     def close(self):
         self.vb.vvs_destroy(self.ctx)
 
-    def verify(self, case, want_probs=True, want_hidden=True) -> dict:
+    def verify(self, case, want_probs=True, want_hidden=True, kv_keep=None) -> dict:
         import torch
         vb, c, ms = self.vb, case, self.ms
         b, cfg, k, f = c["n_images"], c["n_cfg"], c["n_draft_max"], c["n_forced"]
@@ -135,7 +164,14 @@ class GpuRunner:
         res = {k_: (to_host(v) if v is not None else None) for k_, v in o.items()}
         res["status"] = status
         res["launches"] = vb.vvs_last_launch_count(self.ctx)
-        res["kv_k"], res["kv_v"] = to_host(kv_k), to_host(kv_v)
+        if kv_keep is None:
+            res["kv_k"], res["kv_v"] = to_host(kv_k), to_host(kv_v)
+        else:
+            # large caches: bring back only the first kv_keep slots, compare the rest on the device
+            res["kv_k"], res["kv_v"] = to_host(kv_k[:, :, :, :kv_keep]), to_host(kv_v[:, :, :, :kv_keep])
+            res["kv_rest_untouched"] = bool(
+                torch.equal(kv_k[:, :, :, kv_keep:], to_dev(c["kv_k"])[:, :, :, kv_keep:]) and
+                torch.equal(kv_v[:, :, :, kv_keep:], to_dev(c["kv_v"])[:, :, :, kv_keep:]))
         return res
 
 
@@ -147,7 +183,7 @@ def replay_decisions(case, gpu_probs: np.ndarray) -> dict:
     """Oracle decision stage on the float32 target probabilities the GPU emitted."""
     c = case
     ms = c["ms"]
-    out = dict(accept_len=[], next_token=[], accept_mask=[], margins=[])
+    out = dict(accept_len=[], next_token=[], accept_mask=[], margins=[], ratios=[])
     for b in range(c["n_images"]):
         d = O.decide(gpu_probs[b].astype(np.float32), c["block"][b, c["n_forced"]:] - ms.vocab_offset,
                      int(c["n_draft"][b]), c["n_forced"], c["draft_probs"][b], c["uniforms"][b],
@@ -156,6 +192,7 @@ def replay_decisions(case, gpu_probs: np.ndarray) -> dict:
         out["next_token"].append(d["next_token"] + ms.vocab_offset if d["next_token"] >= 0 else -1)
         out["accept_mask"].append(d["accept_mask"])
         out["margins"].append(d["margins"])
+        out["ratios"].append(d["ratios"])
     return {k: np.array(v) for k, v in out.items()}
 
 
@@ -182,11 +219,16 @@ def check_replay(case, gpu: dict, margin_tol: float = 1e-4, sample_tol: float = 
     return excluded
 
 
-def rel_err_rows(a: np.ndarray, ref: np.ndarray) -> float:
-    """max over rows of ||a - ref|| / ||ref||."""
+def rel_err_per_row(a: np.ndarray, ref: np.ndarray) -> np.ndarray:
+    """||a - ref|| / ||ref|| of every row (last axis)."""
     a2 = a.reshape(-1, a.shape[-1])
     r2 = ref.reshape(-1, ref.shape[-1])
-    return float(np.max(np.linalg.norm(a2 - r2, axis=1) / np.linalg.norm(r2, axis=1)))
+    return np.linalg.norm(a2 - r2, axis=1) / np.linalg.norm(r2, axis=1)
+
+
+def rel_err_rows(a: np.ndarray, ref: np.ndarray) -> float:
+    """max over rows of ||a - ref|| / ||ref||."""
+    return float(np.max(rel_err_per_row(a, ref)))
 
 
 def check_new_cache_rows(case, gpu: dict, ora: dict, rtol: float):

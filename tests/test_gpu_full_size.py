@@ -2,14 +2,18 @@
 
 configs[1]: the whole LlamaGen-XL shape (36 layers, d = 1280, V = 16384), batch 1 with guidance,
 K = 8: the oracle finishes one such step in seconds, so every output is compared.
-configs[3] / configs[2]: full width, head_dim, vocabulary slice and batch, at reduced depth (the
-layers repeat the same kernels with other weights; depth is covered by configs[1])."""
+configs[2] (16 images x guidance, relaxed acceptance, 36 layers) and configs[3] (the 7B shape, 32
+layers, fill 1500): one full-depth trial each with a target-independent drafter (no teacher-forced
+oracle passes; the oracle's single pass takes a minute or a few), every output compared, plus the
+quick two-layer versions with the target-aware drafter."""
 from dataclasses import replace
 
 import numpy as np
 import pytest
 
 import helpers as H
+from oracle import vvs_oracle as O
+from vvs_synth import gen
 from test_gpu_verify import _check_end_to_end
 from vvs_synth.configs import B7, CONFIGS, MODE_RELAXED, XL
 
@@ -96,4 +100,67 @@ def test_config1_full_shape_cache_edges(fill):
     gpu = run.verify(case)
     assert gpu["launches"] < 40
     _check_end_to_end(case, gpu, H.run_oracle(case))
+    run.close()
+
+
+def test_config2_full_depth_batch16_relaxed():
+    """configs[2] as the benchmark runs it: 36 layers, 16 images x guidance = 288 block rows through
+    the per-projection tensor-core kernels (two token passes, split-K sums, element-wise kernels),
+    fills drawn per image, relaxed acceptance over 64 latent neighbours."""
+    wl = CONFIGS[2]
+    ms = wl.shape
+    fills = [1, 575, 130, 288, 17, 400, 333, 128, 127, 129, 256, 500, 64, 9, 511, 200]
+    case = H.build_case_independent(ms, wl.seed, 16, 2, 1, 8, fills, cfg_scale=wl.cfg_scale, mode=MODE_RELAXED,
+                                    nbr_k=64, logit_std=1.0)
+    run = H.GpuRunner(ms, case["w"], 32, 9, max_nbr_k=64)
+    gpu = run.verify(case)
+    assert gpu["launches"] > 100           # one kernel per projection
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    print("configs[2] full depth: accept_len", gpu["accept_len"].tolist(), "oracle", ora["accept_len"].tolist())
+    run.close()
+
+
+@pytest.mark.parametrize("deterministic", [True, False])
+def test_config3_full_depth_7b(deterministic):
+    """configs[3] as the benchmark runs it: 32 layers of the 7B shape (d = 4096, 32 heads of 128, MLP
+    11008), 8192 codes inside a 65536-row head, fill 1500, one image with guidance, both whole-chain
+    kernels.  The 13 GB of weights are drawn on the GPU (seeded) and copied to the host for the
+    oracle, which widens one matrix at a time; the caches are cut to the slots the step can touch."""
+    import torch
+    wl = CONFIGS[3]
+    ms = wl.shape
+    fill, t_len = 1500, 9
+    g = torch.Generator(device="cuda").manual_seed(wl.seed + 7)
+    shp = gen.weight_shapes(ms)
+
+    def draw(name):
+        if name.startswith("norm"):
+            return (1.0 + 0.1 * torch.randn(shp[name], generator=g, device="cuda")).to(torch.bfloat16)
+        return (0.02 * torch.randn(shp[name], generator=g, device="cuda")).to(torch.bfloat16)
+
+    def bits(t):
+        return t.view(torch.int16).cpu().numpy().view(np.uint16)
+    wd = {n: draw(n) for n in ("tok_emb", "norm_f", "w_lm")}
+    wd["layers"] = [{n: draw(n) for n in gen.LAYER_TENSORS} for _ in range(ms.n_layers)]
+    w = {n: bits(wd[n]) for n in ("tok_emb", "norm_f", "w_lm")}
+    w["layers"] = {l: {n: bits(t) for n, t in wd["layers"][l].items()} for l in range(ms.n_layers)}
+    kv = [torch.randn((ms.n_layers, 2, ms.n_heads, ms.s_max, ms.head_dim), generator=g, device="cuda").to(torch.bfloat16)
+          for _ in range(2)]
+    case = H.build_case_independent(ms, wl.seed, 1, 2, 1, 8, [fill], cfg_scale=wl.cfg_scale, logit_std=1.0, w=w,
+                                    kv=(bits(kv[0]), bits(kv[1])))
+    from paper_2511_13587_b200 import binding as vb
+    run = H.GpuRunner.__new__(H.GpuRunner)       # weights are on the device already: no second copy
+    run.vb, run.ms, run.wd = vb, ms, wd
+    run.ctx = vb.vvs_create(vb.make_desc(ms, 2, t_len, 1, deterministic))
+    vb.vvs_bind_weights(run.ctx, wd)
+    gpu = run.verify(case, kv_keep=fill + t_len)
+    assert gpu["launches"] < 40            # a whole-chain kernel
+    assert gpu["kv_rest_untouched"]        # slots beyond the block, compared on the device
+    # the oracle only touches cache slots below fill + T: hand it that part (float64 copies of the
+    # whole 2384-slot caches would be 10 GB)
+    small = dict(case, kv_k=case["kv_k"][:, :, :, :fill + t_len], kv_v=case["kv_v"][:, :, :, :fill + t_len])
+    ora = H.run_oracle(small)
+    _check_end_to_end(small, gpu, ora)
+    print("configs[3] full depth: accept_len", gpu["accept_len"].tolist(), "oracle", ora["accept_len"].tolist())
     run.close()

@@ -3,11 +3,12 @@
 tolerate the synchronisation a cudaMalloc brings): its scratch is a fixed device array inside
 the library instead of a context's arena.  It must give exactly what vvs_decide gives, also on a
 second call that finds the first call's leftovers in the shared array, and it must refuse sizes
-beyond the array's stated capacity.  Collected last on purpose (file name)."""
+beyond the array's stated capacity.  Both entry points are also compared with the CPU oracle's
+decision stage on the same probabilities.  Collected last on purpose (file name)."""
 import numpy as np
 import pytest
 
-from test_gpu_decide import decide_case, gpu_decide
+from test_gpu_decide import compare_exact, decide_case, gpu_decide, oracle_decide
 from vvs_synth.configs import MODE_RELAXED, MODE_STRICT
 
 pytestmark = pytest.mark.gpu
@@ -25,8 +26,11 @@ def _both(c, vb):
                       draft_probs=d["draft_probs"], uniforms=d["uniforms"], mode=c["mode"],
                       nbr_k=c["nbr_k"], delta=c["delta"], **o)
 
+    import torch
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
     def no_alloc(d, o):
-        vb.vvs_decide_noalloc(target_probs=d["target_probs"], vocab=c["ms"].vocab,
+        vb.vvs_decide_noalloc(status_bits=status, target_probs=d["target_probs"], vocab=c["ms"].vocab,
                               vocab_offset=c["ms"].vocab_offset, n_rows_per_seq=rows,
                               first_row=first_row, drafts=d["drafts"], n_images=b, n_draft_max=k,
                               n_draft=d["n_draft"], draft_probs=d["draft_probs"],
@@ -35,7 +39,9 @@ def _both(c, vb):
                               delta=c["delta"], **o)
     want = gpu_decide(c, with_ctx)
     got = gpu_decide(c, no_alloc)
+    assert int(status.item()) == 0          # the caller-owned status word: no device-side complaint
     vb.vvs_destroy(ctx)
+    compare_exact(c, got, oracle_decide(c))  # the allocation-free entry point against the CPU oracle itself
     return got, want
 
 
@@ -71,3 +77,8 @@ def test_no_alloc_rejects_sizes_beyond_its_fixed_scratch():
         with pytest.raises(vb.VvsError) as e:
             vb.vvs_decide_noalloc(**dict(base, **bad))
         assert e.value.status == -2, bad
+    # a candidate tree needs scratch rows the fixed array does not have: refused, not decided as a chain
+    for bad in (dict(tree_parent=zi), dict(accept_path=zi)):
+        with pytest.raises(vb.VvsError) as e:
+            vb.vvs_decide_noalloc(**dict(base, **bad))
+        assert e.value.status == -1, bad
