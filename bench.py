@@ -519,18 +519,17 @@ def run_epilogue_sweep(args) -> None:
 
 def decoding_loops(ms, seed: int, runs, n_tokens: int = 576, k: int = 8, cfg_scale: float = 2.0,
                    latent_dim: int = 8, warm: bool = True):
-    """VVS decoding loop (Alg. 2) on model shape `ms` with a synthetic stand-in drafter: per
-    iteration a skip decision (vvs_skip_decide), then either a target verification of the K drafts
-    behind the still unverified tokens (vvs_verify with n_forced = 1 + gamma: post verification,
-    Sec. 4.1; feature-cache store) or a verification-free step (vvs_select_unverified; feature-cache
-    fetch of gamma stale features).  `runs` = [(name, threshold)].  Returns (device status,
-    {name: statistics incl. the per-iteration log}).  The drafter is synthetic (q = softmax(N(0,1)),
-    a random candidate tree whose paths share a stem), so tokens per forward says nothing about
-    image quality or real drafters."""
+    """Times the package's decoding loop (paper_2511_13587_b200.loop.DecodeLoop: Supp. Alg. 2 as a host
+    loop over the C-ABI entry points) on model shape `ms` with the synthetic stand-in drafter.
+    `runs` = [(name, schedule)], schedule = ("never",) | ("fixed", i) | ("dynamic", threshold, alpha).
+    Returns (device status, {name: statistics}).  The drafter is synthetic (q = softmax(N(0,1)), a
+    random candidate tree whose paths share a stem), so tokens per forward says nothing about image
+    quality or real drafters."""
     import torch
     from paper_2511_13587_b200 import binding as vb
+    from paper_2511_13587_b200.loop import DecodeLoop
+    from vvs_synth.drafter import SyntheticDrafter
     n_paths, depth, t_max = 12, 5, 1 + 5 + k
-    rng = gen.rng_for(seed, "loop")
 
     def dev(a):
         a = np.ascontiguousarray(a)
@@ -544,101 +543,23 @@ def decoding_loops(ms, seed: int, runs, n_tokens: int = 576, k: int = 8, cfg_sca
     del hw
     kv_k = torch.randn((ms.n_layers, 2, ms.n_heads, ms.s_max, ms.head_dim), device="cuda").to(torch.bfloat16)
     kv_v = torch.randn_like(kv_k)
-    ctx = vb.vvs_create(vb.make_desc(ms, 2, t_max, 1))
+    ctx = vb.vvs_create(vb.make_desc(ms, 2, t_max, 1, deterministic=False))
     vb.vvs_bind_weights(ctx, wd)
-    codebook_h = gen.make_codebook(seed, ms.vocab, latent_dim).astype(np.float32)
-    codebook = dev(codebook_h)
-    fc = vb.make_fcache(torch.zeros((2, 5 + t_max, ms.d_model), dtype=torch.bfloat16, device="cuda"),
-                        torch.zeros((2, 5 + t_max), dtype=torch.int32, device="cuda"),
-                        torch.zeros((2,), dtype=torch.int32, device="cuda"))
-    q_all, d_all = gen.independent_draft(seed, 0, 16, k, ms.vocab, DRAFT_LOGIT_STD)   # 16 draft sets, cycled
-    q_dev = [dev(q_all[i:i + 1]) for i in range(16)]
-    out = dict(accept_len=torch.zeros(1, dtype=torch.int32, device="cuda"),
-               next_token=torch.zeros(1, dtype=torch.int32, device="cuda"),
-               new_len=torch.zeros(2, dtype=torch.int32, device="cuda"),
-               n_commit=torch.zeros(2, dtype=torch.int32, device="cuda"),
-               hidden=torch.zeros((2, t_max, ms.d_model), dtype=torch.bfloat16, device="cuda"))
-    dec = torch.zeros(1, dtype=torch.uint8, device="cuda")
-    sim = torch.zeros(1, dtype=torch.float32, device="cuda")
-    sel_path = torch.zeros(1, dtype=torch.int32, device="cuda")
-    sel_gamma = torch.zeros(1, dtype=torch.int32, device="cuda")
-    sel_tok = torch.zeros((1, depth), dtype=torch.int32, device="cuda")
-    fetch_out = torch.zeros((2, 5, ms.d_model), dtype=torch.bfloat16, device="cuda")
-    fetch_pos = torch.zeros((2, 5), dtype=torch.int32, device="cuda")
-    skip_all = torch.ones(1, dtype=torch.uint8, device="cuda")
-    # fixed device buffers: the library replays a captured graph when a call repeats the same pointers
-    block_buf = torch.zeros(t_max, dtype=torch.int32, device="cuda")
-    cl_buf = torch.zeros(2, dtype=torch.int32, device="cuda")
-    u_buf = torch.zeros((1, k + 1), dtype=torch.float32, device="cuda")
-    q_buf = torch.zeros((1, k, ms.vocab), dtype=torch.float32, device="cuda")
-    hid_buf = {t: torch.zeros((2, t, ms.d_model), dtype=torch.bfloat16, device="cuda") for t in range(1 + k, t_max + 1)}
-    paths_buf = torch.zeros((1, n_paths, depth), dtype=torch.int32, device="cuda")
-    vlast_buf = torch.zeros(1, dtype=torch.uint8, device="cuda")
-    usel_buf = torch.zeros(1, dtype=torch.float32, device="cuda")
-    gam_buf = torch.zeros(2, dtype=torch.int32, device="cuda")
-
-    def one_image(threshold: float):
-        vb.vvs_feature_cache_reset(ctx, fc)
-        fill, generated, forwards, skips, it, stored = 1, 0, 0, 0, 0, 0
-        pending = []                                   # tokens accepted without verification, K/V not cached yet
-        last_tok, v_last = ms.vocab_offset + int(rng.integers(0, ms.vocab)), False      # Alg. 2 line 3
-        log = []
-        while generated < n_tokens and fill + t_max <= ms.s_max:
-            drafts = d_all[it % 16]
-            stem = int(rng.integers(1, depth + 1))     # synthetic tree: shared stem, then latent-space neighbours or noise
-            paths = np.tile(drafts[None, :depth], (n_paths, 1)).astype(np.int32)
-            noise = rng.integers(0, ms.vocab, size=(n_paths, depth))
-            paths[1:, stem:] = noise[1:, stem:]
-            paths_buf.copy_(torch.from_numpy(paths[None]))
-            vlast_buf.fill_(1 if v_last else 0)
-            vb.vvs_skip_decide(ctx, paths_buf, None, codebook, vlast_buf, 2, 0.8, threshold, dec, sim)
-            skip = bool(dec.item())
-            if not skip:
-                f = 1 + len(pending)
-                t_len = f + k
-                block_buf[:t_len].copy_(torch.tensor([last_tok] + pending + [ms.vocab_offset + int(x) for x in drafts],
-                                                     dtype=torch.int32))
-                cl_buf.fill_(fill)
-                u_buf.copy_(torch.from_numpy(philox.verify_uniforms(seed, it, 1, k)))
-                q_buf.copy_(q_dev[it % 16])
-                o = dict(out, hidden=hid_buf[t_len])
-                vb.vvs_verify(ctx, n_images=1, n_cfg=2, n_forced=f, n_draft_max=k, block=block_buf, n_draft=None,
-                              kv_k=kv_k, kv_v=kv_v, kv_rows=2, cache_len=cl_buf, draft_probs=q_buf, uniforms=u_buf,
-                              cfg_scale=cfg_scale, temperature=1.0, mode=0, nbr_k=1, delta=float("inf"), **o)
-                vb.vvs_feature_cache_store(ctx, fc, hid_buf[t_len], t_len, cl_buf, out["n_commit"])
-                n_acc, nxt = int(out["accept_len"].item()), int(out["next_token"].item())
-                fill += f + n_acc
-                stored += f + n_acc
-                generated += n_acc + 1
-                log.append(("verify", f, n_acc, int(out["new_len"][0].item())))
-                last_tok, pending, v_last = nxt, [], True
-                forwards += 1
-            else:
-                usel_buf.fill_(float(rng.random()))
-                vb.vvs_select_unverified(ctx, paths_buf, None, usel_buf, sel_path, sel_gamma, sel_tok)
-                gamma = int(sel_gamma.item())
-                if min(gamma, stored) > 0:               # the first steps have fewer cached features than gamma
-                    gam_buf.fill_(min(gamma, 5, stored))
-                    vb.vvs_feature_cache_fetch(ctx, fc, skip_all, 1, gam_buf, 5, 0, fetch_out, fetch_pos)
-                pending = pending + [ms.vocab_offset + t for t in sel_tok[0, :gamma].tolist()]
-                log.append(("skip", gamma, float(sim.item())))
-                generated += gamma
-                v_last = False
-                skips += 1
-            it += 1
-        torch.cuda.synchronize()
-        return generated, forwards, skips, it, fill, log
-
+    codebook = dev(gen.make_codebook(seed, ms.vocab, latent_dim).astype(np.float32))
+    drafter = SyntheticDrafter(seed, ms.vocab, k, n_paths=n_paths, depth=depth, logit_std=DRAFT_LOGIT_STD)
+    loop = DecodeLoop(ctx, ms, kv_k, kv_v, k, 2, cfg_scale, n_paths, depth, codebook=codebook)
+    u_of = lambda it: philox.verify_uniforms(seed, it, 1, k)
     results = {}
-    for name, thr in runs:
+    for name, schedule in runs:
         if warm:
-            one_image(thr)                               # captures the graphs of every block shape
+            loop.run(drafter.first_token(), drafter.propose, u_of, n_tokens, schedule)   # captures the graphs
         t0 = time.perf_counter()
-        gen_tok, fw, sk, its, fill, log = one_image(thr)
+        r = loop.run(drafter.first_token(), drafter.propose, u_of, n_tokens, schedule)
         dt = time.perf_counter() - t0
-        results[name] = {"tokens": gen_tok, "target_forwards": fw, "skipped_steps": sk, "iterations": its,
-                         "tokens_per_forward": gen_tok / max(fw, 1), "tokens_per_s": gen_tok / dt, "seconds": dt,
-                         "final_fill": fill, "log": log}
+        results[name] = {"tokens": r["generated"], "target_forwards": r["target_forwards"],
+                         "skipped_steps": r["skipped_steps"], "iterations": r["iterations"],
+                         "tokens_per_forward": r["generated"] / max(r["target_forwards"], 1),
+                         "tokens_per_s": r["generated"] / dt, "seconds": dt, "final_fill": r["fill"]}
     status = vb.vvs_device_status(ctx)
     vb.vvs_destroy(ctx)
     return status, results
@@ -650,11 +571,11 @@ def run_generation_loop(args) -> None:
     if int(os.environ.get("RANK", "0")) != 0:
         return
     wl = CONFIGS[1]
-    status, results = decoding_loops(wl.shape, wl.seed, (("never skip (plain speculative decoding)", 2.0),
-                                                         ("dynamic skip, threshold 0.65", 0.65)),
-                                     k=wl.n_draft_max, cfg_scale=wl.cfg_scale, latent_dim=wl.latent_dim)
-    for r in results.values():
-        r.pop("log")
+    runs = (("never skip (plain speculative decoding)", ("never",)),
+            ("VVS-U, fixed interval 4", ("fixed", 4)), ("VVS-U, fixed interval 3", ("fixed", 3)),
+            ("VVS-U, fixed interval 2", ("fixed", 2)), ("VVS-D, dynamic skip, threshold 0.65", ("dynamic", 0.65, 0.8)))
+    status, results = decoding_loops(wl.shape, wl.seed, runs, k=wl.n_draft_max, cfg_scale=wl.cfg_scale,
+                                     latent_dim=wl.latent_dim)
     print(json.dumps({"metric": "VVS decoding loop (Alg. 2), one 576-token image, LlamaGen-XL shape, synthetic drafter",
                       "unit": "generated tokens/s (host loop included)", "dtype": "bf16", "data": "synthetic",
                       "device_status": status, "runs": results}))

@@ -453,6 +453,86 @@ def select_unverified(paths: np.ndarray, path_len: np.ndarray, u: float):
 
 
 # ---------------------------------------------------------------------------------------
+# Skipped-step scheduling and the decoding loop (Sec. 4.4 first paragraph; Sec. 4.1; Supp. Alg. 2)
+
+
+def skip_schedule_fixed(step: int, interval: int) -> bool:
+    """VVS-U (Sec. 4.4): with a fixed interval i, after i - 1 normally verified steps the i-th
+    verification step is skipped.  Steps count from 0, so step t is skipped iff t mod i == i - 1;
+    an interval below 2 never skips (two skipped steps in a row are not allowed, Sec. 4.1)."""
+    return interval >= 2 and step % interval == interval - 1
+
+
+def decode_loop(ms, weights: dict, kv_k: np.ndarray, kv_v: np.ndarray, first_token: int, propose, uniforms_of,
+                n_tokens: int, k: int, n_cfg: int, cfg_scale: float, schedule, codebook=None, fill0: int = 1,
+                fcache_cap: int = 16, gamma_cap: int = 5) -> dict:
+    """Supp. Algorithm 2 for one image, with the drafter M_D replaced by the callable `propose`
+    (iteration -> drafts [K] codebook indices, q [K, V], candidate paths, path_len, u_select) and the
+    uniforms of iteration t given by uniforms_of(t) [1, K + 1].
+
+    Per iteration: Decision (schedule = ("never",) | ("fixed", i) | ("dynamic", threshold, alpha,
+    stride), the dynamic rule being Alg. 1 with its no-two-skips guard); if not skipped, ONE target
+    pass over [last committed token, the still unverified tokens, the K drafts] (post verification,
+    Sec. 4.1: n_forced = 1 + number of unverified tokens, their K/V restored, their features written
+    back), Verify, UpdateCache; otherwise UniformSample with truncation (Sec. 4.2) and a Retrieve of
+    the gamma most recent features for the drafter (Sec. 4.3).  V_last is read as "the last step was
+    verified" and starts False.  The loop ends once n_tokens tokens were generated or the KV cache
+    cannot take another block.
+
+    kv_k, kv_v: stored caches [n_layers, n_cfg, H, S, hd], filled to fill0 (the prefilled prompt).
+    Returns the generated tokens (embedding-table ids), the per-iteration log, the final fill, the
+    float64 caches and the feature cache."""
+    kc = [widen(kv_k[:, r]) for r in range(n_cfg)]
+    vc = [widen(kv_v[:, r]) for r in range(n_cfg)]
+    fc = FeatureCache(n_cfg, fcache_cap, ms.d_model)
+    t_max = 1 + gamma_cap + k
+    fill, generated, it, stored = fill0, 0, 0, 0
+    last_tok, pending, v_last = ms.vocab_offset + int(first_token), [], False
+    tokens, log = [], []
+    while generated < n_tokens and fill + t_max <= ms.s_max:
+        c = propose(it)
+        if schedule[0] == "never":
+            skip, sim = False, 0.0
+        elif schedule[0] == "fixed":
+            skip, sim = skip_schedule_fixed(it, int(schedule[1])), 0.0
+        else:
+            skip, sim = skip_decision(c["paths"], c["path_len"], codebook, schedule[2], schedule[1], v_last,
+                                      schedule[3] if len(schedule) > 3 else 2)
+        if skip and len(pending) + int(np.max(c["path_len"])) > gamma_cap:
+            skip = False      # the next block could not hold more unverified tokens
+        if not skip:
+            f = 1 + len(pending)
+            block = np.array([[last_tok] + pending + [ms.vocab_offset + int(x) for x in c["drafts"]]], dtype=np.int32)
+            hidden = np.zeros((n_cfg, f + k, ms.d_model))
+            for r in range(n_cfg):
+                hidden[r] = target_forward(ms, weights, block[0], kc[r], vc[r], fill)
+            out = epilogue(ms, weights, hidden, block[:, f:] - ms.vocab_offset, np.array([k]), f, c["q"][None],
+                           uniforms_of(it), n_cfg, cfg_scale)
+            n_acc = int(out["accept_len"][0])
+            nxt = int(out["next_token"][0]) + ms.vocab_offset
+            fc.store(hidden, np.full(n_cfg, fill), np.full(n_cfg, f + n_acc))
+            tokens += [int(t) for t in block[0, f:f + n_acc]] + [nxt]
+            log.append(("verify", f, n_acc, fill + f + n_acc))
+            fill += f + n_acc
+            stored += f + n_acc
+            generated += n_acc + 1
+            last_tok, pending, v_last = nxt, [], True
+        else:
+            idx, gamma, kept = select_unverified(c["paths"], c["path_len"], c["u_select"])
+            g_fetch = min(gamma, gamma_cap, stored)
+            feats = fc.fetch(np.ones(1, np.uint8), np.full(n_cfg, g_fetch), 0, gamma_cap) if g_fetch > 0 else None
+            pending = pending + [ms.vocab_offset + int(t) for t in kept]
+            tokens += [ms.vocab_offset + int(t) for t in kept]
+            log.append(("skip", idx, gamma, g_fetch))
+            generated += gamma
+            v_last = False
+            del feats
+        it += 1
+    return dict(tokens=tokens, log=log, fill=fill, last_token=last_tok, pending=pending, kc=kc, vc=vc, fcache=fc,
+                iterations=it)
+
+
+# ---------------------------------------------------------------------------------------
 # Tree verification (Sec. 2 / Sec. 5: the drafter proposes a candidate TREE, EAGLE-2 style; the
 # paper verifies it with the target in one pass and walks it with the sequential rule of Sec. 2)
 #
