@@ -12,6 +12,7 @@ and the max-over-ranks of the device time.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -27,15 +28,18 @@ sys.path.insert(0, ROOT)
 from vvs_synth import gen, philox  # noqa: E402
 from vvs_synth.configs import CONFIGS, MODE_RELAXED  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu
-# capture summarised under profiles/ (None until one has been taken for the current kernel).
-NCU_TRAFFIC = {1: 1.4825e9, 2: None, 3: None}   # fused_chain_kernel, capture of the current kernel
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the whole-chain kernel, from the ncu
+# captures summarised under profiles/.  Keyed by (workload, fixed-order sums); each entry names the
+# kernel's source file and the first 16 hex digits of that file's SHA-256 when the counters were
+# taken: the line reports null once the file has changed since.
+NCU_CAPTURES = {
+}
 N_TRIALS = 32           # distinct (fill, block, draft) inputs cycled through the steps
 DRAFT_LOGIT_STD = 1.0   # target-independent drafter: q = softmax(N(0, std^2))
 
 
 def metric_name(wl) -> str:
-    shape = "LlamaGen-XL" if wl.shape.name.startswith("llamagen") else "7B visual-AR"
+    shape = {"llamagen": "LlamaGen-XL", "visual_a": "7B visual-AR"}.get(wl.shape.name[:8], wl.shape.name)
     return f"verified draft tokens/sec ({shape}-shaped verify step)"
 
 
@@ -57,6 +61,19 @@ def max_over_ranks(values, world: int, device="cpu"):
 def aggregate_value(world: int, drafts_per_step: float, steps: int, ms_total: float) -> float:
     """Whole-job throughput: every replica verifies its own drafts in the (max over ranks) time."""
     return world * drafts_per_step * steps / (ms_total * 1e-3)
+
+
+def ncu_traffic(index: int, deterministic: bool, chain: bool):
+    """(bytes per launch, where they come from) for the dominant kernel, or (None, reason)."""
+    e = NCU_CAPTURES.get((index, deterministic))
+    if not chain or e is None:
+        return None, "no ncu capture of this kernel and workload under profiles/"
+    src, sha, nbytes, summary = e
+    with open(os.path.join(ROOT, src), "rb") as fh:
+        cur = hashlib.sha256(fh.read()).hexdigest()[:16]
+    if cur != sha:
+        return None, f"{summary} is stale: {src} has changed since the capture"
+    return nbytes, summary
 
 
 def peaks():
@@ -146,10 +163,239 @@ class ClockSampler:
 # the CUDA arm
 
 
+class VerifyBench:
+    """One workload resident on this process's GPU: weights, caches, a library context, the
+    seeded trials and the step function that the timed regions repeat."""
+
+    def __init__(self, index: int, rank: int = 0, deterministic: bool = False, n_trials: int = N_TRIALS):
+        import torch
+        from paper_2511_13587_b200 import binding as vb
+        from vvs_synth.configs import DTYPE_BF16
+        self.torch, self.vb, self.index = torch, vb, index
+        self.wl = wl = CONFIGS[index]
+        self.ms = ms = wl.shape
+        self.b, self.cfg, self.k, self.f = wl.n_images, wl.n_cfg, wl.n_draft_max, wl.n_forced
+        self.r, self.t_len = self.b * self.cfg, wl.block_len
+        self.relaxed = wl.mode == MODE_RELAXED
+        self.seed = seed = replica_seed(wl.seed, rank)
+        self.tdt = torch.bfloat16 if ms.dtype == DTYPE_BF16 else torch.float32
+        r, t_len, b = self.r, self.t_len, self.b
+        dev = self.dev
+
+        # resident state: weights, KV cache, neighbour table, feature cache
+        if index == 3:
+            # 13 GB of weights: drawn on the device (same distributions as the host generator; the
+            # benchmark compares nothing with the oracle, the full-size parity tests do)
+            g = torch.Generator(device="cuda").manual_seed(seed)
+            shp = gen.weight_shapes(ms)
+
+            def draw(name):
+                if name.startswith("norm"):
+                    return (1.0 + 0.1 * torch.randn(shp[name], generator=g, device="cuda")).to(torch.bfloat16)
+                return (0.02 * torch.randn(shp[name], generator=g, device="cuda")).to(torch.bfloat16)
+
+            wd = {n: draw(n) for n in ("tok_emb", "norm_f", "w_lm")}
+            wd["layers"] = [{n: draw(n) for n in gen.LAYER_TENSORS} for _ in range(ms.n_layers)]
+        else:
+            hw = gen.make_weights(ms, seed)
+            wd = {n: dev(v) for n, v in hw.items() if n != "layers"}
+            wd["layers"] = [{n: dev(v) for n, v in hw["layers"][l].items()} for l in range(ms.n_layers)]
+            del hw
+        # cache K/V ~ N(0, 1), drawn on the device (the host generator's distribution)
+        g = torch.Generator(device="cuda").manual_seed(seed + 1)
+        self.kv_k = torch.empty((ms.n_layers, r, ms.n_heads, ms.s_max, ms.head_dim), dtype=self.tdt, device="cuda")
+        self.kv_v = torch.empty_like(self.kv_k)
+        for l in range(ms.n_layers):
+            self.kv_k[l].copy_(torch.randn(self.kv_k[l].shape, generator=g, device="cuda"))
+            self.kv_v[l].copy_(torch.randn(self.kv_v[l].shape, generator=g, device="cuda"))
+        # the seeded cache, kept aside: set-up and statistics calls start from it, while the timed
+        # calls leave their block rows behind in the live cache like a decoding loop does
+        self.kv0_k, self.kv0_v = self.kv_k.clone(), self.kv_v.clone()
+        self.wd = wd
+        self.ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, wl.nbr_k, deterministic=deterministic))
+        vb.vvs_bind_weights(self.ctx, wd)
+        if self.relaxed:
+            rp, col = gen.neighbour_csr(gen.make_codebook(seed, ms.vocab, wl.latent_dim), wl.nbr_k)
+            self.rp_d, self.col_d = dev(rp), dev(col)
+            vb.vvs_bind_neighbors(self.ctx, self.rp_d, self.col_d)
+        cap = 5 + t_len
+        self.fc = vb.make_fcache(torch.zeros((r, cap, ms.d_model), dtype=self.tdt, device="cuda"),
+                                 torch.zeros((r, cap), dtype=torch.int32, device="cuda"),
+                                 torch.zeros((r,), dtype=torch.int32, device="cuda"))
+        vb.vvs_feature_cache_reset(self.ctx, self.fc)
+        self.out = dict(accept_len=torch.zeros(b, dtype=torch.int32, device="cuda"),
+                        next_token=torch.zeros(b, dtype=torch.int32, device="cuda"),
+                        new_len=torch.zeros(r, dtype=torch.int32, device="cuda"),
+                        n_commit=torch.zeros(r, dtype=torch.int32, device="cuda"),
+                        hidden=torch.zeros((r, t_len, ms.d_model), dtype=self.tdt, device="cuda"))
+        self.fetch_out = torch.zeros((r, 5, ms.d_model), dtype=self.tdt, device="cuda")
+        self.fetch_pos = torch.zeros((r, 5), dtype=torch.int32, device="cuda")
+        self.launches = 0
+        self.keys = ("cache_len", "block", "draft_probs", "uniforms", "n_draft", "skip_mask", "gamma")
+        self.trials = [host_trial(wl, t) for t in range(n_trials)]
+        self.dtr = [{n: dev(t[n]) for n in self.keys} for t in self.trials]
+        if index == 0:
+            self.drafter = f"independent softmax(N(0,{wl.q_noise_std}^2))"
+        else:
+            self._draft_from_target()
+            self.drafter = f"softmax(guided target logits + N(0,{wl.q_noise_std}^2)), position by position"
+
+    def dev(self, a):
+        torch = self.torch
+        a = np.ascontiguousarray(a)
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        return torch.from_numpy(a).cuda()
+
+    def _verify(self, inp, out, **extra):
+        wl = self.wl
+        self.vb.vvs_verify(self.ctx, n_images=self.b, n_cfg=self.cfg, n_forced=self.f, n_draft_max=self.k,
+                           block=inp["block"], n_draft=inp["n_draft"], kv_k=self.kv_k, kv_v=self.kv_v,
+                           kv_rows=self.r, cache_len=inp["cache_len"], draft_probs=inp["draft_probs"],
+                           uniforms=inp["uniforms"], cfg_scale=wl.cfg_scale, temperature=wl.temperature,
+                           mode=wl.mode, nbr_k=wl.nbr_k, delta=wl.delta, **out, **extra)
+
+    def _draft_from_target(self):
+        """Replaces every trial's drafter rows and draft tokens: the row for draft j is the softmax of
+        the library's own guided target logits for that position (given the forced tokens and
+        drafts 0..j-1) plus N(0, q_noise_std^2) noise, and draft j is sampled from it - K set-up
+        calls per trial, outside every timed region."""
+        torch, ms, wl = self.torch, self.ms, self.wl
+        b, k, f = self.b, self.k, self.f
+        g = torch.Generator(device="cuda").manual_seed(self.seed + 2)
+        probs = torch.zeros((b, self.t_len, ms.vocab), dtype=torch.float32, device="cuda")
+        for inp in self.dtr:
+            inp["block"][:, f:] = ms.vocab_offset
+            for j in range(k):
+                self.restore_cache()
+                self._verify(inp, self.out, target_probs=probs)
+                lg = torch.log(probs[:, f - 1 + j].clamp_min(1e-30))
+                lg = lg + wl.q_noise_std * torch.randn(lg.shape, generator=g, device="cuda")
+                qj = torch.softmax(lg, dim=-1)
+                inp["draft_probs"][:, j] = qj
+                tok = torch.multinomial(qj, 1, generator=g)[:, 0]
+                inp["block"][:, f + j] = (ms.vocab_offset + tok).to(torch.int32)
+        torch.cuda.synchronize()
+
+    def restore_cache(self):
+        self.kv_k.copy_(self.kv0_k)
+        self.kv_v.copy_(self.kv0_v)
+
+    def step(self, inp, out=None):
+        vb, ctx = self.vb, self.ctx
+        out = self.out if out is None else out
+        self._verify(inp, out)
+        if self.relaxed:   # the trials' fill levels are unrelated: start each from an empty feature cache
+            vb.vvs_feature_cache_reset(ctx, self.fc)
+            self.launches += 1
+        vb.vvs_feature_cache_store(ctx, self.fc, out["hidden"], self.t_len, inp["cache_len"], out["n_commit"])
+        self.launches += vb.vvs_last_launch_count(ctx) + 1
+        if self.relaxed:   # workload 2: skip-masked images reuse cached features
+            vb.vvs_feature_cache_fetch(ctx, self.fc, inp["skip_mask"], self.b, inp["gamma"], 5, 0,
+                                       self.fetch_out, self.fetch_pos)
+            self.launches += 1
+
+    def region(self, steps: int, fn=None) -> float:
+        """Device time (ms) of `steps` consecutive steps, events on the launching stream."""
+        torch = self.torch
+        fn = fn or (lambda i: self.step(self.dtr[i % len(self.dtr)]))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1)
+
+    def acceptance(self, seeded_cache: bool = True) -> dict:
+        """Untimed pass over the trials: accepted drafts, bonus-row samples and decisions whose
+        uniform lies within 1e-4 of the acceptance ratio.  With `seeded_cache` every call starts
+        from the seeded cache the drafter rows were made for; without it the calls see the cache
+        as the timed region leaves it (block rows of other trials inside their prefix), where the
+        drafter is further from the target."""
+        torch = self.torch
+        margins = torch.zeros((self.b, self.k + 1), dtype=torch.float32, device="cuda")
+        acc = drafted = bonus = near = judged = 0
+        for inp in self.dtr:
+            if seeded_cache:
+                self.restore_cache()
+            self._verify(inp, self.out, margins=margins)
+            a = self.out["accept_len"]
+            acc += int(a.sum().item())
+            drafted += int(inp["n_draft"].sum().item())
+            bonus += int((a == inp["n_draft"]).sum().item())
+            m = margins[:, :self.k]
+            judged += int(torch.isfinite(m).sum().item())
+            near += int((m < 1e-4).sum().item())
+        return {"acceptance_rate": acc / max(drafted, 1), "per_decision_acceptance": acc / max(judged, 1),
+                "mean_accept_len": acc / (len(self.dtr) * self.b),
+                "bonus_row_samples": bonus, "calls": len(self.dtr) * self.b, "judged": judged,
+                "near_threshold": near, "near_threshold_rule": "|u - ratio| < 1e-4"}
+
+    def class_times(self, n_prof: int):
+        vb = self.vb
+        vb.vvs_profile_enable(self.ctx, True)
+        for i in range(n_prof):
+            self.step(self.dtr[i % len(self.dtr)])
+        cls_ms, cls_n = vb.vvs_profile_read(self.ctx)
+        vb.vvs_profile_enable(self.ctx, False)
+        return cls_ms, cls_n
+
+    def drafts_per_step(self, steps: int) -> float:
+        return float(np.mean([self.trials[i % len(self.trials)]["n_draft"].sum() for i in range(steps)]))
+
+    def roofline(self, cls_ms, cls_n, n_prof: int, pk: dict, ms_step: float) -> dict:
+        """The roofline object of the kernel (or kernel set) that dominates the step."""
+        ms = self.ms
+        alg = algorithmic_bytes(self.wl, self.trials)
+        per_step = {"gemm": cls_ms[0] / n_prof, "attention": cls_ms[1] / n_prof,
+                    "other": cls_ms[2] / n_prof, "chain": cls_ms[3] / n_prof}
+        if cls_n[3] > 0:
+            # calls of at most 32 tokens: embedding + all decoder layers are ONE persistent kernel, which
+            # streams every layer weight once and reads the K/V rows (the LM head is a separate launch)
+            name = "whole-chain kernel (embedding + all decoder layers, one persistent launch)"
+            dom_ms = cls_ms[3] / cls_n[3]
+            dom_bytes = alg["total"] - ms.vocab * ms.d_model * 2
+            dom_launches = cls_n[3] / n_prof
+        else:
+            # wider calls: a launch per projection / attention / element-wise stage; no single kernel
+            # dominates, so the object describes the whole step (all launches of one verify call)
+            name = "whole step (per-projection GEMM, attention and element-wise launches together)"
+            dom_ms, dom_bytes, dom_launches = ms_step, alg["total"], sum(cls_n) / n_prof
+        achieved = dom_bytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
+        return {"kernel": name, "bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / pk["hbm_gbs"], "peak_source": pk["source"],
+                "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms,
+                "launches_per_step": dom_launches, "class_ms_per_step": per_step}
+
+    def close(self):
+        self.vb.vvs_destroy(self.ctx)
+        self.ctx = None
+        self.wd = self.kv_k = self.kv_v = self.kv0_k = self.kv0_v = self.dtr = self.fc = self.out = None
+        self.torch.cuda.empty_cache()
+
+
+def timed_regions(fn_region, steps: int, world: int, barrier, min_ms: float = 500.0, max_repeats: int = 400,
+                  device="cuda"):
+    """Repeats a `steps`-long timed region (each one bracketed by barrier + synchronize, its device
+    time taken as the maximum over ranks) until at least `min_ms` of device time has been
+    measured.  Returns the list of region times (ms)."""
+    times = []
+    target = None
+    while True:
+        barrier()
+        t = max_over_ranks([fn_region(steps)], world, device=device)[0]
+        barrier()
+        times.append(t)
+        if target is None:     # every rank derives the same repeat count from the same number
+            target = int(min(max_repeats, max(1, np.ceil(min_ms / max(t, 1e-3)))))
+        if len(times) >= target:
+            return times
+
+
 def run_ours(args) -> None:
     import torch
     import torch.distributed as dist
-    from paper_2511_13587_b200 import binding as vb
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -157,108 +403,27 @@ def run_ours(args) -> None:
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    wl = CONFIGS[args.workload]
-    ms = wl.shape
-    b, cfg, k, f = wl.n_images, wl.n_cfg, wl.n_draft_max, wl.n_forced
-    r, t_len = b * cfg, wl.block_len
-    relaxed = wl.mode == MODE_RELAXED
-    seed = replica_seed(wl.seed, rank)
-
-    def dev(a):
-        a = np.ascontiguousarray(a)
-        if a.dtype == np.uint16:
-            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
-        return torch.from_numpy(a).cuda()
-
-    # resident state: weights, KV cache, neighbour table, feature cache
-    if args.workload == 3:
-        # 13 GB of weights: drawn on the device (same distributions as the host generator; the
-        # benchmark compares nothing with the oracle, the full-size parity tests do)
-        g = torch.Generator(device="cuda").manual_seed(seed)
-        shp = gen.weight_shapes(ms)
-
-        def draw(name):
-            if name.startswith("norm"):
-                return (1.0 + 0.1 * torch.randn(shp[name], generator=g, device="cuda")).to(torch.bfloat16)
-            return (0.02 * torch.randn(shp[name], generator=g, device="cuda")).to(torch.bfloat16)
-
-        wd = {n: draw(n) for n in ("tok_emb", "norm_f", "w_lm")}
-        wd["layers"] = [{n: draw(n) for n in gen.LAYER_TENSORS} for _ in range(ms.n_layers)]
-        kv_k = torch.randn((ms.n_layers, r, ms.n_heads, ms.s_max, ms.head_dim), generator=g,
-                           device="cuda").to(torch.bfloat16)
-        kv_v = torch.randn((ms.n_layers, r, ms.n_heads, ms.s_max, ms.head_dim), generator=g,
-                           device="cuda").to(torch.bfloat16)
-    else:
-        hw = gen.make_weights(ms, seed)
-        wd = {n: dev(v) for n, v in hw.items() if n != "layers"}
-        wd["layers"] = [{n: dev(v) for n, v in hw["layers"][l].items()} for l in range(ms.n_layers)]
-        del hw
-        kv_k = torch.empty((ms.n_layers, r, ms.n_heads, ms.s_max, ms.head_dim), dtype=torch.bfloat16, device="cuda")
-        kv_v = torch.empty_like(kv_k)
-        for row in range(r):
-            hk, hv = gen.make_kv_row(ms, seed, row)
-            kv_k[:, row].copy_(dev(hk))
-            kv_v[:, row].copy_(dev(hv))
-    ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, wl.nbr_k, deterministic=bool(args.deterministic)))
-    vb.vvs_bind_weights(ctx, wd)
-    if relaxed:
-        rp, col = gen.neighbour_csr(gen.make_codebook(seed, ms.vocab, wl.latent_dim), wl.nbr_k)
-        rp_d, col_d = dev(rp), dev(col)
-        vb.vvs_bind_neighbors(ctx, rp_d, col_d)
-    cap = 5 + t_len
-    fc = vb.make_fcache(torch.zeros((r, cap, ms.d_model), dtype=torch.bfloat16, device="cuda"),
-                        torch.zeros((r, cap), dtype=torch.int32, device="cuda"),
-                        torch.zeros((r,), dtype=torch.int32, device="cuda"))
-    vb.vvs_feature_cache_reset(ctx, fc)
-
-    trials = [host_trial(wl, t) for t in range(N_TRIALS)]
-    keys = ("cache_len", "block", "draft_probs", "uniforms", "n_draft", "skip_mask", "gamma")
-    dtr = [{n: dev(t[n]) for n in keys} for t in trials]
-    out = dict(accept_len=torch.zeros(b, dtype=torch.int32, device="cuda"),
-               next_token=torch.zeros(b, dtype=torch.int32, device="cuda"),
-               new_len=torch.zeros(r, dtype=torch.int32, device="cuda"),
-               n_commit=torch.zeros(r, dtype=torch.int32, device="cuda"),
-               hidden=torch.zeros((r, t_len, ms.d_model), dtype=torch.bfloat16, device="cuda"))
-    fetch_out = torch.zeros((r, 5, ms.d_model), dtype=torch.bfloat16, device="cuda")
-    fetch_pos = torch.zeros((r, 5), dtype=torch.int32, device="cuda")
-    launches = [0]
-
-    def step(inp, out=out):
-        vb.vvs_verify(ctx, n_images=b, n_cfg=cfg, n_forced=f, n_draft_max=k, block=inp["block"],
-                      n_draft=inp["n_draft"], kv_k=kv_k, kv_v=kv_v, kv_rows=r, cache_len=inp["cache_len"],
-                      draft_probs=inp["draft_probs"], uniforms=inp["uniforms"], cfg_scale=wl.cfg_scale,
-                      temperature=wl.temperature, mode=wl.mode, nbr_k=wl.nbr_k, delta=wl.delta, **out)
-        if relaxed:   # the trials' fill levels are unrelated: start each from an empty feature cache
-            vb.vvs_feature_cache_reset(ctx, fc)
-            launches[0] += 1
-        vb.vvs_feature_cache_store(ctx, fc, out["hidden"], t_len, inp["cache_len"], out["n_commit"])
-        launches[0] += vb.vvs_last_launch_count(ctx) + 1
-        if relaxed:   # workload 2: skip-masked images reuse cached features
-            vb.vvs_feature_cache_fetch(ctx, fc, inp["skip_mask"], b, inp["gamma"], 5, 0, fetch_out, fetch_pos)
-            launches[0] += 1
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
+    S = VerifyBench(args.workload, rank, bool(args.deterministic))
+    wl, ms, vb = S.wl, S.ms, S.vb
+    warm = max(args.warmup, 3)
+
     # ---- device-resident timing ---------------------------------------------------------------
-    for i in range(max(args.warmup, 3)):
-        step(dtr[i % N_TRIALS])
+    for i in range(warm):
+        S.step(S.dtr[i % len(S.dtr)])
     barrier()
-    launches[0] = 0
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    S.launches = 0
     with ClockSampler(local) as clocks:
-        barrier()
-        e0.record()
-        for i in range(args.steps):
-            step(dtr[i % N_TRIALS])
-        e1.record()
-        barrier()
-    ms_total = e0.elapsed_time(e1)
-    gpu_launches = launches[0]
-    status = vb.vvs_device_status(ctx)
-    drafts_per_step = float(np.mean([trials[i % N_TRIALS]["n_draft"].sum() for i in range(args.steps)]))
+        regions = timed_regions(S.region, args.steps, world, barrier)
+    gpu_launches = S.launches // len(regions)
+    ms_region = float(np.median(regions))
+    status = vb.vvs_device_status(S.ctx)
+    drafts_per_step = S.drafts_per_step(args.steps)
 
     # ---- end to end: host buffers in, host results out, every step ------------------------------
     # The step's inputs sit in ONE pinned host buffer and its results come back in one: a call
@@ -271,101 +436,126 @@ def run_ours(args) -> None:
         buf = torch.empty(off, dtype=torch.uint8).pin_memory() if pinned else torch.empty(off, dtype=torch.uint8, device="cuda")
         return buf, {n: buf[o:o + nb].view(dt).view(shape) for n, (o, nb, shape, dt) in views.items()}
 
-    in_shapes = {n: (tuple(dtr[0][n].shape), dtr[0][n].dtype) for n in keys}
+    in_shapes = {n: (tuple(S.dtr[0][n].shape), S.dtr[0][n].dtype) for n in S.keys}
     res_names = ("accept_len", "next_token", "new_len")
-    out_shapes = {n: (tuple(out[n].shape), out[n].dtype) for n in res_names}
+    out_shapes = {n: (tuple(S.out[n].shape), S.out[n].dtype) for n in res_names}
     pin = []
-    for t in trials[:8]:
+    for t in S.dtr[:8]:
         buf, views = packed(in_shapes, True)
-        for n in keys:
-            views[n].copy_(torch.from_numpy(np.ascontiguousarray(t[n])))
+        for n in S.keys:
+            views[n].copy_(t[n].cpu())
         pin.append(buf)
     stage_buf, stage = packed(in_shapes, False)
     res_dev_buf, res_dev = packed(out_shapes, False)
     res_host_buf, res_host = packed(out_shapes, True)
-    out_e2e = dict(out, **res_dev)
+    out_e2e = dict(S.out, **res_dev)
     h2d = stage_buf.numel()
     d2h = res_host_buf.numel()
 
     def step_e2e(i):
         stage_buf.copy_(pin[i % len(pin)], non_blocking=True)
-        step(stage, out_e2e)
+        S.step(stage, out_e2e)
         res_host_buf.copy_(res_dev_buf, non_blocking=True)
         torch.cuda.current_stream().synchronize()
 
     for i in range(3):
         step_e2e(i)
-    barrier()
-    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e2.record()
-    for i in range(args.steps):
-        step_e2e(i)
-    e3.record()
-    barrier()
-    ms_e2e = e2.elapsed_time(e3)
+    regions_e2e = timed_regions(lambda n: S.region(n, step_e2e), args.steps, world, barrier)
+    ms_e2e = float(np.median(regions_e2e))
 
     # ---- per-kernel-class timing for the roofline (separate pass, not the headline) -----------
-    vb.vvs_profile_enable(ctx, True)
     n_prof = min(args.steps, 8)
-    for i in range(n_prof):
-        step(dtr[i % N_TRIALS])
-    cls_ms, cls_n = vb.vvs_profile_read(ctx)
-    vb.vvs_profile_enable(ctx, False)
+    cls_ms, cls_n = S.class_times(n_prof)
+    accept_live = S.acceptance(seeded_cache=False)
+    accept = S.acceptance()
+    accept["live_cache"] = {n: accept_live[n] for n in ("acceptance_rate", "per_decision_acceptance", "mean_accept_len",
+                                                        "bonus_row_samples", "near_threshold")}
+    status |= vb.vvs_device_status(S.ctx)
 
-    # ---- reduce over ranks ----------------------------------------------------------------------
-    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     pk = peaks()
-    alg = algorithmic_bytes(wl, trials)
-    if cls_n[3] > 0:
-        # calls of at most 32 tokens: embedding + all decoder layers are ONE persistent kernel, which
-        # streams every layer weight once and reads the K/V rows (the LM head is a separate launch)
-        dom_name = "fused_chain_kernel (embedding + all decoder layers, one persistent launch)"
-        dom_ms = cls_ms[3] / cls_n[3]
-        dom_bytes = alg["total"] - ms.vocab * ms.d_model * 2
-        dom_launches = cls_n[3] / n_prof
-    else:
-        dom_name = "gemm_tc_kernel (projection / LM-head GEMMs, weight streaming)"
-        dom_ms = cls_ms[0] / max(cls_n[0], 1)
-        dom_bytes = alg["weights"] * n_prof / max(cls_n[0], 1)
-        dom_launches = cls_n[0] / n_prof
-    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
-    ms_step = ms_total / args.steps
+    alg = algorithmic_bytes(wl, S.trials)
+    ms_step = ms_region / args.steps
+    roof = S.roofline(cls_ms, cls_n, n_prof, pk, ms_step)
+    roof["traffic"], roof["traffic_source"] = ncu_traffic(args.workload, bool(args.deterministic), cls_n[3] > 0)
+    b, cfg, k, t_len = S.b, S.cfg, S.k, S.t_len
     line = {
         "metric": metric_name(wl),
-        "value": aggregate_value(world, drafts_per_step, args.steps, ms_total),
-        "unit": "drafts/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_step, "verify_latency_us": ms_step * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "value": aggregate_value(world, drafts_per_step, args.steps, ms_region),
+        "unit": "drafts/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
+        "repeats": len(regions), "timed_ms": float(np.sum(regions)),
+        "ms_per_step": ms_step, "ms_per_step_min": float(np.min(regions)) / args.steps,
+        "ms_per_step_max": float(np.max(regions)) / args.steps, "verify_latency_us": ms_step * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if S.tdt == torch.bfloat16 else "f32",
         "data": "synthetic",
         "config": {"workload": f"configs[{args.workload}] {wl.name}", "n_images": b, "n_cfg": cfg,
                    "n_draft": k, "block_rows": t_len, "fill": f"U[{wl.fill_lo},{wl.fill_hi}] per trial",
-                   "trials": N_TRIALS, "draft": f"independent softmax(N(0,{DRAFT_LOGIT_STD}^2))",
-                   "l2": f"weights streamed per step ({alg['weights'] / 1e9:.2f} GB) exceed the 126 MB L2; no flush needed",
+                   "trials": len(S.trials), "draft": S.drafter,
+                   "sums": "fixed order (bitwise repeatable)" if args.deterministic else "arrival order (split-K adds in L2)",
+                   "timing": "median over `repeats` regions of `steps` steps each, every region bracketed by barrier + synchronize",
+                   "l2": f"weights streamed per step ({alg['weights'] / 1e9:.2f} GB) exceed the 126 MB L2; no flush needed"
+                         if alg["weights"] > 126e6 else "weights fit in L2: a latency case, not a bandwidth case",
                    "parallelism": "replicas only (no collective)"},
+        "acceptance": accept,
         "step_hbm": {"algorithmic_bytes": alg["total"], "achieved_gbs": alg["total"] / (ms_step * 1e-3) / 1e9,
                      "frac_of_measured": alg["total"] / (ms_step * 1e-3) / 1e9 / pk["hbm_gbs"],
                      "frac_of_8tbs": alg["total"] / (ms_step * 1e-3) / 1e9 / 8000.0},
-        "roofline": {"kernel": dom_name, "bound": "hbm",
-                     "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / pk["hbm_gbs"], "peak_source": pk["source"],
-                     "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms,
-                     "traffic": NCU_TRAFFIC.get(args.workload), "launches_per_step": dom_launches,
-                     "class_ms_per_step": {"gemm": cls_ms[0] / n_prof, "attention": cls_ms[1] / n_prof,
-                                           "other": cls_ms[2] / n_prof, "chain": cls_ms[3] / n_prof}},
+        "roofline": roof,
         "e2e": {"value": aggregate_value(world, drafts_per_step, args.steps, ms_e2e), "unit": "drafts/s",
-                "ms_per_step": ms_e2e / args.steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "ms_per_step": ms_e2e / args.steps, "repeats": len(regions_e2e),
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": gpu_launches, "device_status": status, "clocks": clocks.summary(),
     }
+    S.close()
+    if world == 1 and not args.no_other and args.workload == 1:
+        line["other_workloads"] = other_workloads(args, pk)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, steps=args.cpu_steps)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def quick_measure(index: int, deterministic: bool, steps: int, pk: dict, min_ms: float = 300.0) -> dict:
+    """A short device-resident measurement of one workload (one GPU): median step time over
+    repeated regions, the step's algorithmic bytes and roofline fraction, acceptance statistics."""
+    import torch
+    S = VerifyBench(index, 0, deterministic, n_trials=16)
+    for i in range(3):
+        S.step(S.dtr[i % len(S.dtr)])
+    torch.cuda.synchronize()
+    S.launches = 0
+    regions = timed_regions(S.region, steps, 1, torch.cuda.synchronize, min_ms=min_ms)
+    launches = S.launches // (len(regions) * steps)
+    ms_step = float(np.median(regions)) / steps
+    n_prof = min(steps, 8)
+    cls_ms, cls_n = S.class_times(n_prof)
+    roof = S.roofline(cls_ms, cls_n, n_prof, pk, ms_step)
+    alg = algorithmic_bytes(S.wl, S.trials)
+    res = {"workload": f"configs[{index}] {S.wl.name}", "ms_per_step": ms_step, "steps": steps, "repeats": len(regions),
+           "drafts_per_s": S.drafts_per_step(steps) / (ms_step * 1e-3), "launches_per_step": launches,
+           "sums": "fixed order" if deterministic else "arrival order",
+           "algorithmic_bytes": alg["total"], "step_frac_of_measured_hbm": alg["total"] / (ms_step * 1e-3) / 1e9 / pk["hbm_gbs"],
+           "roofline": {n: roof[n] for n in ("kernel", "achieved", "frac", "ms_per_launch", "class_ms_per_step")},
+           "acceptance": S.acceptance(), "device_status": S.vb.vvs_device_status(S.ctx)}
+    S.close()
+    return res
+
+
+def other_workloads(args, pk: dict) -> dict:
+    """The workloads beside the headline one, each measured briefly on this GPU."""
+    out = {"configs[1] fixed-order sums": quick_measure(1, True, 64, pk),
+           "configs[0]": quick_measure(0, False, 256, pk, min_ms=100.0),
+           "configs[2]": quick_measure(2, False, 16, pk),
+           "configs[3]": quick_measure(3, False, 16, pk),
+           "configs[3] fixed-order sums": quick_measure(3, True, 16, pk),
+           "configs[4]": epilogue_sweep(steps=20, pk=pk)}
+    return out
 
 
 # ---------------------------------------------------------------------------------------------
@@ -426,24 +616,33 @@ def run_reference(args) -> None:
 # ---------------------------------------------------------------------------------------------
 # configs[4]: the acceptance epilogue in isolation (LM head + guidance + softmax + decisions)
 
+# (d, V, B, K, C, mode, neighbour k, drafter noise scale, temperature): every value of every axis
+# of the sweep appears at least once; the noise scale skews the drafter against the target so that
+# the measured acceptance rates run from a few per cent to above 90 %
+SWEEP_POINTS = (
+    (1280, 16384, 1, 8, 2, 0, 1, 1.0, 1.0), (1280, 16384, 1, 4, 1, 0, 1, 0.15, 0.5),
+    (1280, 16384, 8, 8, 2, 1, 1, 0.5, 1.0), (1280, 16384, 16, 8, 2, 1, 64, 1.0, 1.0),
+    (1280, 16384, 32, 8, 2, 0, 1, 2.0, 1.5), (1280, 16384, 8, 16, 2, 1, 1000, 1.5, 1.0),
+    (1280, 4096, 64, 16, 2, 1, 64, 3.0, 1.0), (1280, 65536, 32, 4, 2, 0, 1, 0.3, 0.7),
+    (4096, 4096, 8, 4, 2, 0, 1, 0.15, 1.0), (4096, 16384, 32, 8, 2, 0, 1, 1.0, 1.2),
+    (4096, 65536, 8, 8, 2, 0, 1, 2.0, 1.0), (4096, 65536, 64, 16, 2, 0, 1, 0.5, 1.0),
+    (4096, 65536, 64, 16, 1, 0, 1, 1.0, 1.0),
+)
 
-def run_epilogue_sweep(args) -> None:
-    """A few points of the configs[4] sweep through vvs_epilogue, inputs drawn on the device.
-    One JSON line; every point carries its time, the LM-head TFLOP/s (2 M d V over the whole call,
-    which runs the LM head, the decision kernels and the one-row-per-image second pass) and the
-    bytes-per-second of the codebook stream, each as a fraction of the measured peak."""
+
+def epilogue_sweep(steps: int, pk: dict) -> dict:
+    """Points of the acceptance-epilogue sweep through vvs_epilogue (LM head + guidance + softmax +
+    decisions on given features), inputs drawn on the device.  Every point carries its time, the
+    LM-head TFLOP/s (2 M d V over the whole call, which runs the LM head, the decision kernels and
+    the one-row-per-image second pass), the bytes per second of the codebook stream, each as a
+    fraction of the measured peak, and the measured acceptance rate.  The drafter row of a
+    position is softmax(log p + scale * Gumbel noise), p the library's own target row."""
     import torch
     from paper_2511_13587_b200 import binding as vb
-    from vvs_synth.configs import ModelShape, MODE_STRICT
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-    if int(os.environ.get("RANK", "0")) != 0:
-        return
-    pk = peaks()
+    from vvs_synth.configs import ModelShape
     points = []
-    for d, v, b, k, c, mode, nbr_k in ((1280, 16384, 1, 8, 2, MODE_STRICT, 1), (1280, 16384, 16, 8, 2, MODE_RELAXED, 64),
-                                       (1280, 16384, 32, 8, 2, MODE_STRICT, 1), (4096, 16384, 32, 8, 2, MODE_STRICT, 1),
-                                       (4096, 65536, 8, 8, 2, MODE_STRICT, 1), (4096, 65536, 64, 16, 2, MODE_STRICT, 1),
-                                       (4096, 65536, 64, 16, 1, MODE_STRICT, 1), (1280, 4096, 64, 16, 2, MODE_RELAXED, 64)):
+    csr = {}
+    for d, v, b, k, c, mode, nbr_k, noise, temp in SWEEP_POINTS:
         ms = ModelShape("epilogue", 0, d, 0, 0, 0, v)
         rows = k + 1
         ctx = vb.vvs_create(vb.make_desc(ms, b * c, rows, max(1, nbr_k)))
@@ -451,40 +650,60 @@ def run_epilogue_sweep(args) -> None:
         w_lm = (torch.randn((v, d), generator=g, device="cuda") * (2.0 / d ** 0.5)).to(torch.bfloat16)
         vb.vvs_bind_weights(ctx, {"w_lm": w_lm, "layers": []})
         if mode == MODE_RELAXED:
-            rp, col = gen.neighbour_csr(gen.make_codebook(0x56565304, v), nbr_k)
-            rp_d, col_d = torch.from_numpy(rp).cuda(), torch.from_numpy(col).cuda()
-            vb.vvs_bind_neighbors(ctx, rp_d, col_d)
+            if (v, nbr_k) not in csr:
+                rp, col = gen.neighbour_csr(gen.make_codebook(0x56565304, v), nbr_k)
+                csr[(v, nbr_k)] = (torch.from_numpy(rp).cuda(), torch.from_numpy(col).cuda())
+            vb.vvs_bind_neighbors(ctx, *csr[(v, nbr_k)])
         hidden = torch.randn((b * c, rows, d), generator=g, device="cuda").to(torch.bfloat16)
-        q = torch.softmax(torch.randn((b, k, v), generator=g, device="cuda"), -1).contiguous()
-        drafts = torch.randint(0, v, (b, k), generator=g, device="cuda", dtype=torch.int32)
+        q = torch.full((b, k, v), 1.0 / v, dtype=torch.float32, device="cuda")
+        drafts = torch.zeros((b, k), dtype=torch.int32, device="cuda")
         u = torch.rand((b, k + 1), generator=g, device="cuda").clamp_(1e-6, 1 - 1e-6)
         nd = torch.full((b,), k, dtype=torch.int32, device="cuda")
         o = dict(accept_len=torch.zeros(b, dtype=torch.int32, device="cuda"),
                  next_token=torch.zeros(b, dtype=torch.int32, device="cuda"))
+        kw = dict(hidden_in=hidden, n_rows_per_seq=rows, first_row=0, drafts=drafts, n_images=b, n_cfg=c,
+                  n_draft_max=k, n_draft=nd, draft_probs=q, cfg_scale=2.0, temperature=temp, mode=mode,
+                  nbr_k=nbr_k, delta=float("inf"))
+        # set-up: the target rows of this point, then the skewed drafter and its tokens
+        probs = torch.zeros((b, rows, v), dtype=torch.float32, device="cuda")
+        vb.vvs_epilogue(ctx, uniforms=u, target_probs=probs, **kw, **o)
+        gum = -torch.log(-torch.log(torch.rand((b, k, v), generator=g, device="cuda").clamp_(1e-9, 1 - 1e-9)))
+        q.copy_(torch.softmax(torch.log(probs[:, :k].clamp_min(1e-30)) + noise * gum, dim=-1))
+        drafts.copy_(torch.multinomial(q.view(b * k, v), 1, generator=g).view(b, k).to(torch.int32))
+        del probs, gum
 
-        def call():
-            vb.vvs_epilogue(ctx, hidden_in=hidden, n_rows_per_seq=rows, first_row=0, drafts=drafts, n_images=b,
-                            n_cfg=c, n_draft_max=k, n_draft=nd, draft_probs=q, uniforms=u, cfg_scale=2.0,
-                            temperature=1.0, mode=mode, nbr_k=nbr_k, delta=float("inf"), **o)
+        def call(uu=u):
+            vb.vvs_epilogue(ctx, uniforms=uu, **kw, **o)
 
         for _ in range(3):
             call()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for _ in range(args.steps):
+        for _ in range(steps):
             call()
         e1.record()
         torch.cuda.synchronize()
-        ms_call = e0.elapsed_time(e1) / args.steps
+        ms_call = e0.elapsed_time(e1) / steps
+        acc = first = calls = 0                      # acceptance statistics, untimed, fresh uniforms per call
+        for _ in range(max(1, 256 // b)):
+            uu = torch.rand((b, k + 1), generator=g, device="cuda").clamp_(1e-6, 1 - 1e-6)
+            call(uu)
+            acc += int(o["accept_len"].sum().item())
+            first += int((o["accept_len"] >= 1).sum().item())
+            calls += b
         m_rows = b * c * rows
         flops, byts = 2.0 * m_rows * d * v, d * v * 2 + m_rows * d * 2 + b * v * 4
         points.append({"d": d, "V": v, "B": b, "K": k, "C": c, "M": m_rows, "relaxed_k": nbr_k if mode else 0,
+                       "temperature": temp, "drafter_noise": noise,
                        "us": ms_call * 1e3, "tflops": flops / ms_call / 1e9,
                        "frac_tensor": flops / ms_call / 1e9 / pk["bf16_tflops"],
                        "gbs": byts / ms_call / 1e6, "frac_hbm": byts / ms_call / 1e6 / pk["hbm_gbs"],
+                       "first_draft_acceptance": first / calls, "acceptance_rate": acc / (calls * k),
                        "device_status": vb.vvs_device_status(ctx)})
         vb.vvs_destroy(ctx)
+        del w_lm, hidden, q
+        torch.cuda.empty_cache()
     # the dynamic skip decision (Alg. 1 / Eq. 2): 16 images, 24 candidate paths of depth 5 each,
     # the 8-dim latent codebook of 16384 codes; latency-bound (one CTA per image, a few hundred
     # dependent-load-limited cosine terms), reported as time per call
@@ -506,11 +725,19 @@ def run_epilogue_sweep(args) -> None:
     torch.cuda.synchronize()
     skip_us = e0.elapsed_time(e1) * 10.0
     vb.vvs_destroy(ctx)
-    print(json.dumps({"metric": "acceptance epilogue in isolation (configs[4] sweep points)", "unit": "us per call",
-                      "skip_decide": {"images": 16, "paths": 24, "depth": 5, "codebook": [16384, 8], "stride": 2,
-                                      "us_per_call": skip_us, "bound": "latency (launch + one chain of L2 loads)"},
-                      "steps": args.steps, "dtype": "bf16", "data": "synthetic", "peak_source": pk["source"],
-                      "points": points}))
+    return {"metric": "acceptance epilogue in isolation (configs[4] sweep points)", "unit": "us per call",
+            "skip_decide": {"images": 16, "paths": 24, "depth": 5, "codebook": [16384, 8], "stride": 2,
+                            "us_per_call": skip_us, "bound": "latency (launch + one chain of L2 loads)"},
+            "steps": steps, "dtype": "bf16", "data": "synthetic", "peak_source": pk["source"],
+            "points": points}
+
+
+def run_epilogue_sweep(args) -> None:
+    import torch
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    print(json.dumps(epilogue_sweep(args.steps, peaks())))
 
 
 # ---------------------------------------------------------------------------------------------
@@ -670,11 +897,13 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=512)     # ~0.7 s timed region at configs[1]: several clock samples
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3, 4, 5, 6])
+    ap.add_argument("--workload", type=int, default=1, choices=[0, 1, 2, 3, 4, 5, 6])
     ap.add_argument("--deterministic", type=int, default=0, choices=[0, 1],
                     help="1: fixed-order sums (bitwise repeatable), 0: arrival-order split-K sums (faster)")
     ap.add_argument("--cpu-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other", action="store_true",
+                    help="skip the short measurements of the other workloads that the default line carries")
     args = ap.parse_args()
     if args.workload == 4:
         run_epilogue_sweep(args)

@@ -28,9 +28,19 @@ def main() -> None:
     # the slowest rank decides the time of the whole job
     ms_total, ms_e2e = bench.max_over_ranks([10.0 + rank, 20.0 - rank], world)
     drafts = float(trial["n_draft"].sum())
+    # repeated timed regions: the rank-dependent region times must give every rank the same repeat
+    # count (it follows from the maximum over ranks of the first region), or the barriers deadlock
+    calls = []
+
+    def region(steps):
+        calls.append(steps)
+        return 40.0 + 30.0 * rank + len(calls)      # rank 1 is slower: 71, 72, ...
+
+    regions = bench.timed_regions(region, 4, world, dist.barrier, min_ms=500.0, device="cpu")
     if rank == 0:
         out = {"fills": [int(f[0]) for f in all_fills], "ms_total": ms_total, "ms_e2e": ms_e2e,
-               "value": bench.aggregate_value(world, drafts, 4, ms_total), "drafts": drafts, "world": world}
+               "value": bench.aggregate_value(world, drafts, 4, ms_total), "drafts": drafts, "world": world,
+               "regions": regions, "region_calls": calls}
         with open(os.environ["VVS_RANK_TEST_OUT"], "w") as f:
             json.dump(out, f)
     dist.destroy_process_group()

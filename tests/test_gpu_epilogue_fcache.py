@@ -76,6 +76,12 @@ def _run_epilogue(case):
     (320, 4096 + 136, 8, 2, 8, False, MODE_RELAXED, 64, float("inf"), 0.5),
     (512, 2048, 3, 2, 16, True, MODE_RELAXED, 1000, 0.2, 1.5),
     (512, 1000, 5, 1, 8, True, MODE_RELAXED, 1, float("inf"), 1.0),
+    # points of the epilogue sweep at its own sizes (d in {1280, 4096}, V in {4096, 16384, 65536})
+    (1280, 16384, 8, 2, 8, True, MODE_RELAXED, 64, float("inf"), 1.0),
+    (1280, 16384, 1, 1, 4, True, MODE_RELAXED, 1000, 0.3, 0.5),
+    (4096, 4096, 32, 2, 16, True, MODE_STRICT, 1, float("inf"), 1.5),
+    (4096, 65536, 8, 2, 4, True, MODE_STRICT, 1, float("inf"), 1.0),
+    (1280, 65536, 64, 1, 4, False, MODE_STRICT, 1, float("inf"), 0.7),
 ])
 def test_epilogue_sweep_points(d, v, n_images, n_cfg, k, bonus, mode, nbr_k, delta, tau):
     rows = k + 1 if bonus else k
