@@ -22,7 +22,14 @@ is silent or garbled:
   entries whose cumulative target mass (not counting p(x)) stays <= delta; acceptance
   probability min(1, sum_{x' in A} p(x') / q(x)).  **parity unpinned** by the paper beyond
   "k = 1 or delta = 0 is strict" and the bounds p(x) <= P_A <= p(x) + delta.
-* residual after a relaxed rejection: the plain norm(max(0, p - q)).  **parity unpinned**.
+* residual after a relaxed rejection: the plain norm(max(0, p - q)) by default.  Flag
+  `adjusted_residual`: norm(max(0, p~ - q)) with p~ the adjusted target of the rejected draft x
+  (the pooled mass of A sits on x, the other members of A carry none): the distribution under
+  which the relaxed test of x is the plain speculative test.  **parity unpinned** by the paper
+  for the choice; mass conservation, the hand example and k = 1 = strict are pinned.
+* relaxed acceptance on a candidate tree (not printed): the chain's relaxed rule with the
+  current residual p_res in the place of p at every sibling round.  **parity unpinned** by the
+  paper; pinned here by k = 1 = the strict walk and by a chain-shaped tree = the chain rule.
 * classifier-free guidance is not in the paper: l = l_u + s (l_c - l_u) on logits before the
   softmax; rows ordered [cond_0..cond_{B-1}, uncond_0..uncond_{B-1}].
 * architecture (not in the paper): pre-norm RMSNorm (eps inside the square root, learned
@@ -198,6 +205,35 @@ def pooled_mass(p_row: np.ndarray, x: int, row_ptr: np.ndarray, col: np.ndarray,
     return float(p_row[x]) + cum
 
 
+def pooled_neighbours(p_row: np.ndarray, x: int, row_ptr: np.ndarray, col: np.ndarray, k: int,
+                      delta: float) -> list:
+    """The neighbours of x (x itself excluded) whose mass pooled_mass adds to p(x): the same
+    distance-ordered prefix, as a list of codebook indices."""
+    nb = col[row_ptr[x]:row_ptr[x + 1]][:k]
+    cum, taken = 0.0, []
+    for xn in nb[1:]:
+        pn = float(p_row[xn])
+        if cum + pn > delta:
+            break
+        cum += pn
+        taken.append(int(xn))
+    return taken
+
+
+def adjusted_target(p_row: np.ndarray, x: int, row_ptr: np.ndarray, col: np.ndarray, k: int,
+                    delta: float) -> np.ndarray:
+    """Target row under which the relaxed test of draft x is the plain speculative test (the
+    adjusted distribution of the relaxed-acceptance construction the paper takes over in Sec. 2):
+    the pooled neighbours' mass sits on x, the pooled neighbours carry none, every other code keeps
+    its probability.  Same dtype as p_row (the moved mass is rounded to it)."""
+    out = np.array(p_row, copy=True)
+    mass = pooled_mass(p_row, x, row_ptr, col, k, delta)
+    for xn in pooled_neighbours(p_row, x, row_ptr, col, k, delta):
+        out[xn] = 0
+    out[x] = mass
+    return out
+
+
 def acceptance_ratio(p_mass: float, q_x: float) -> float:
     """min(1, P / q(x)); a draft with q(x) = 0 is accepted iff P > 0."""
     if q_x > 0.0:
@@ -221,13 +257,15 @@ def inverse_cdf(r: np.ndarray, u: float):
 
 def decide(p32: np.ndarray, drafts: np.ndarray, n_draft: int, n_forced: int, q32: np.ndarray,
            u32: np.ndarray, mode: int = MODE_STRICT, row_ptr=None, col=None, k: int = 1,
-           delta: float = float("inf")) -> dict:
+           delta: float = float("inf"), adjusted_residual: bool = False) -> dict:
     """Sequential verification of one image's drafts against float32 target rows p32 [T, V].
 
     Draft i (token drafts[i], draft row q32[i]) is judged against p32[n_forced-1+i] with
     uniform u32[i]; verification stops at the first rejection.  The next token comes from
     norm(max(0, p - q)) of the rejecting position, or from the following target row if every
-    draft was accepted (-1 if p32 has no such row); it uses the last uniform u32[-1]."""
+    draft was accepted (-1 if p32 has no such row); it uses the last uniform u32[-1].
+    With `adjusted_residual` (relaxed mode only; off by default) the p of the residual is the
+    adjusted target of the rejected draft instead of the plain row."""
     p32 = np.asarray(p32, dtype=np.float32)
     q32 = np.asarray(q32, dtype=np.float32)
     k_max = len(u32) - 1
@@ -255,6 +293,8 @@ def decide(p32: np.ndarray, drafts: np.ndarray, n_draft: int, n_forced: int, q32
     else:
         row = p32[src]
         if n < n_draft:
+            if adjusted_residual and mode == MODE_RELAXED:
+                row = adjusted_target(row, int(drafts[n]), row_ptr, col, k, delta)
             r = np.maximum(np.float32(0.0), row - q32[n])       # IEEE float32 subtraction
             if not np.any(r > 0):
                 r = row                                          # p == q numerically
@@ -271,7 +311,8 @@ def decide(p32: np.ndarray, drafts: np.ndarray, n_draft: int, n_forced: int, q32
 
 def epilogue(ms, weights: dict, hidden: np.ndarray, drafts, n_draft, n_forced: int, draft_probs,
              uniforms, n_cfg: int, cfg_scale: float, temperature: float = 1.0, mode: int = MODE_STRICT,
-             row_ptr=None, col=None, k: int = 1, delta: float = float("inf")) -> dict:
+             row_ptr=None, col=None, k: int = 1, delta: float = float("inf"),
+             adjusted_residual: bool = False) -> dict:
     """LM head + guidance + softmax + decisions on given features.
 
     hidden [R, T, d] with R = n_cfg*B rows ordered cond images then uncond images (n_cfg = 2
@@ -291,7 +332,7 @@ def epilogue(ms, weights: dict, hidden: np.ndarray, drafts, n_draft, n_forced: i
         logits[b] = guided_logits(l_c, l_u, cfg_scale)
         probs[b] = guided_probs(l_c, l_u, cfg_scale, temperature)
         dec = decide(probs[b].astype(np.float32), drafts[b], int(n_draft[b]), n_forced,
-                     draft_probs[b], uniforms[b], mode, row_ptr, col, k, delta)
+                     draft_probs[b], uniforms[b], mode, row_ptr, col, k, delta, adjusted_residual)
         for key in ("accept_len", "next_token", "accept_mask", "margins", "ratios"):
             out[key][b] = dec[key]
     out["target_probs"] = probs
@@ -303,7 +344,7 @@ def verify(ms, weights: dict, block: np.ndarray, n_forced: int, n_draft: np.ndar
            kv_k: np.ndarray, kv_v: np.ndarray, cache_len: np.ndarray, draft_probs: np.ndarray,
            uniforms: np.ndarray, n_cfg: int, cfg_scale: float, temperature: float = 1.0,
            mode: int = MODE_STRICT, row_ptr=None, col=None, k: int = 1,
-           delta: float = float("inf")) -> dict:
+           delta: float = float("inf"), adjusted_residual: bool = False) -> dict:
     """One verification step for B images.
 
     block int [B, T] = n_forced committed tokens whose K/V is not yet cached, then K drafts,
@@ -328,7 +369,7 @@ def verify(ms, weights: dict, block: np.ndarray, n_forced: int, n_draft: np.ndar
         v_new[:, r] = vc[:, :, fill:fill + t_len]
     drafts = block[:, n_forced:] - ms.vocab_offset            # embedding id -> codebook index
     out = epilogue(ms, weights, hidden, drafts, n_draft, n_forced, draft_probs, uniforms,
-                   n_cfg, cfg_scale, temperature, mode, row_ptr, col, k, delta)
+                   n_cfg, cfg_scale, temperature, mode, row_ptr, col, k, delta, adjusted_residual)
     out["next_token"] = np.where(out["next_token"] >= 0, out["next_token"] + ms.vocab_offset,
                                  -1).astype(np.int32)
     out["hidden"] = hidden
@@ -576,12 +617,18 @@ def tree_forward(ms, weights: dict, tokens: np.ndarray, parent: np.ndarray, kc: 
 
 
 def tree_decide(p32: np.ndarray, draft_tokens: np.ndarray, parent: np.ndarray, n_forced: int,
-                q32: np.ndarray, u32: np.ndarray) -> dict:
+                q32: np.ndarray, u32: np.ndarray, mode: int = MODE_STRICT, row_ptr=None, col=None,
+                k: int = 1, delta: float = float("inf"), adjusted_residual: bool = False) -> dict:
     """Walk of one image's candidate tree.  p32 [T, V] float32 target rows (row t = distribution
     of the token after node t); draft node i = block row n_forced + i carries codebook token
     draft_tokens[i], was drawn from q32[i] (the drafter's distribution at its parent) and is judged
     with u32[i]; u32[K] drives the final sample.  The first residual is the float32 difference (as
-    in the chain rule); later rounds work in float64."""
+    in the chain rule); later rounds work in float64.
+    Relaxed mode: the numerator of a child's ratio is the pooled mass of the child and its
+    neighbours in the CURRENT residual p_res (the chain's relaxed rule with p_res in the place
+    of p); with `adjusted_residual` a rejection subtracts q from the adjusted p_res of the
+    rejected child, otherwise from p_res itself."""
+    relaxed = mode == MODE_RELAXED
     p32 = np.asarray(p32, dtype=np.float32)
     q32 = np.asarray(q32, dtype=np.float32)
     t_len, k_max = p32.shape[0], len(u32) - 1
@@ -597,15 +644,19 @@ def tree_decide(p32: np.ndarray, draft_tokens: np.ndarray, parent: np.ndarray, n
         for c in children:
             i = c - n_forced
             x = int(draft_tokens[i])
-            ratio = acceptance_ratio(float(p_res[x]), float(q32[i, x]))
+            mass = pooled_mass(p_res, x, row_ptr, col, k, delta) if relaxed else float(p_res[x])
+            ratio = acceptance_ratio(mass, float(q32[i, x]))
             margins[i] = abs(float(u32[i]) - ratio)
             if float(u32[i]) < ratio:
                 accepted = c
                 break
+            adjust = relaxed and adjusted_residual
             if first_round:
-                r = np.maximum(np.float32(0.0), p32[cur] - q32[i]).astype(np.float64)   # IEEE float32
+                row = adjusted_target(p32[cur], x, row_ptr, col, k, delta) if adjust else p32[cur]
+                r = np.maximum(np.float32(0.0), row - q32[i]).astype(np.float64)        # IEEE float32
             else:
-                r = np.maximum(0.0, p_res - q32[i].astype(np.float64))
+                row = adjusted_target(p_res, x, row_ptr, col, k, delta) if adjust else p_res
+                r = np.maximum(0.0, row - q32[i].astype(np.float64))
             z = float(np.sum(r))
             if z > 0.0:                                          # p_res == q numerically: keep p_res
                 p_res, sample_from = r / z, r
@@ -621,7 +672,9 @@ def tree_decide(p32: np.ndarray, draft_tokens: np.ndarray, parent: np.ndarray, n
 
 def tree_verify(ms, weights: dict, block: np.ndarray, parent: np.ndarray, n_forced: int,
                 kv_k: np.ndarray, kv_v: np.ndarray, cache_len: np.ndarray, draft_probs: np.ndarray,
-                uniforms: np.ndarray, n_cfg: int, cfg_scale: float, temperature: float = 1.0) -> dict:
+                uniforms: np.ndarray, n_cfg: int, cfg_scale: float, temperature: float = 1.0,
+                mode: int = MODE_STRICT, row_ptr=None, col=None, k: int = 1, delta: float = float("inf"),
+                adjusted_residual: bool = False) -> dict:
     """One verification step over candidate trees: tree_forward per sequence, guidance and
     softmax per image as in `epilogue`, then tree_decide.  block [B, T] embedding-table ids,
     parent [B, T].  Returns accept_len, accept_path (list per image, block rows), next_token
@@ -644,7 +697,8 @@ def tree_verify(ms, weights: dict, block: np.ndarray, parent: np.ndarray, n_forc
         l_u = lm_head_logits(ms, weights, widen(hidden[n_images + b])) if n_cfg == 2 else None
         out["target_probs"][b] = guided_probs(l_c, l_u, cfg_scale, temperature)
         dec = tree_decide(out["target_probs"][b].astype(np.float32), block[b, n_forced:] - ms.vocab_offset,
-                          parent[b], n_forced, draft_probs[b], uniforms[b])
+                          parent[b], n_forced, draft_probs[b], uniforms[b], mode, row_ptr, col, k, delta,
+                          adjusted_residual)
         out["accept_len"][b] = dec["accept_len"]
         out["accept_path"].append(dec["accept_path"])
         out["next_token"][b] = dec["next_token"] + ms.vocab_offset
