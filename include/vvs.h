@@ -193,9 +193,20 @@ typedef struct vvs_verify_args {
                                node are tried in index order, child x passes iff
                                u < min(1, p_res(x) / q(x)), a rejection replaces p_res by
                                norm(max(0, p_res - q)); when no child is left the next token is drawn
-                               from p_res (from the node's own target row if it is a leaf).  Tree
-                               calls need a bf16 context, strict mode, n_draft == NULL and
+                               from p_res (from the node's own target row if it is a leaf).  In
+                               relaxed mode the numerator of a child's ratio is the pooled mass of
+                               the child and its neighbours in the CURRENT p_res (the chain's relaxed
+                               rule with p_res in the place of p; the paper prints no tree rule).
+                               Tree calls need a bf16 context, n_draft == NULL and
                                out->target_probs (the walk reads whole target rows). */
+  int32_t adjusted_residual; /* relaxed mode only, 0 (default) or 1.  0: after a rejection the next
+                               token is drawn from norm(max(0, p - q)) with the plain target row p.
+                               1: from norm(max(0, p~ - q)), p~ the adjusted target of the rejected
+                               draft x - the pooled mass of the accepted set A sits on x, the other
+                               members of A carry none, all other codes keep their probability (the
+                               distribution under which the relaxed test is the plain speculative
+                               test; Sec. 2 cites the relaxed rule without printing its residual).
+                               Ignored in strict mode; must be 0 or 1. */
 } vvs_verify_args;
 
 /* Outputs, device memory allocated by the caller.  Optional ones may be NULL and are then
@@ -266,7 +277,8 @@ int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, 
  * Capacity (larger sizes return VVS_ERR_SHAPE): n_images <= 64, n_draft_max <= 16,
  * nbr_k <= 64, vocab <= 65536.
  *
- * Chains only: args->tree_parent and out->accept_path must be NULL (VVS_ERR_INVALID_ARG).
+ * Chains only: args->tree_parent and out->accept_path must be NULL, and args->adjusted_residual
+ * must be 0 (it needs a writable copy of the sampled row): VVS_ERR_INVALID_ARG otherwise.
  *
  * Arguments are those of vvs_decide, with what a context would carry passed explicitly: vocab,
  * vocab_offset, and the CSR neighbour table (device int32, may be NULL in strict mode).

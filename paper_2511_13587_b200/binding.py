@@ -50,7 +50,7 @@ class vvs_verify_args(C.Structure):
                 ("cache_len", C.c_void_p), ("cache_len_host", C.c_void_p),
                 ("draft_probs", C.c_void_p), ("uniforms", C.c_void_p), ("cfg_scale", C.c_float),
                 ("temperature", C.c_float), ("mode", C.c_int32), ("nbr_k", C.c_int32),
-                ("delta", C.c_float), ("tree_parent", C.c_void_p)]
+                ("delta", C.c_float), ("tree_parent", C.c_void_p), ("adjusted_residual", C.c_int32)]
 
 
 class vvs_verify_out(C.Structure):
@@ -188,11 +188,12 @@ def vvs_bind_neighbors(ctx: int, row_ptr: torch.Tensor, col: torch.Tensor) -> No
 
 def _args(n_images, n_cfg, n_forced, n_draft_max, block, n_draft, kv_k, kv_v, kv_rows, cache_len,
           cache_len_host, draft_probs, uniforms, cfg_scale, temperature, mode, nbr_k, delta,
-          tree_parent=None):
+          tree_parent=None, adjusted_residual=False):
     return vvs_verify_args(int(n_images), int(n_cfg), int(n_forced), int(n_draft_max), _ptr(block),
                            _ptr(n_draft), _ptr(kv_k), _ptr(kv_v), int(kv_rows), _ptr(cache_len),
                            _ptr(cache_len_host), _ptr(draft_probs), _ptr(uniforms), float(cfg_scale),
-                           float(temperature), int(mode), int(nbr_k), float(delta), _ptr(tree_parent))
+                           float(temperature), int(mode), int(nbr_k), float(delta), _ptr(tree_parent),
+                           int(adjusted_residual))
 
 
 def _out(accept_len, next_token, new_len, n_commit, accept_mask, target_probs, hidden, margins,
@@ -205,9 +206,10 @@ def vvs_verify(ctx: int, *, n_images, n_cfg, n_forced, n_draft_max, block, kv_k,
                cache_len, draft_probs, uniforms, accept_len, next_token, new_len, n_draft=None,
                cache_len_host=None, cfg_scale=1.0, temperature=1.0, mode=VVS_MODE_STRICT, nbr_k=1,
                delta=float("inf"), n_commit=None, accept_mask=None, target_probs=None, hidden=None,
-               margins=None, tree_parent=None, accept_path=None, stream=None) -> None:
+               margins=None, tree_parent=None, accept_path=None, adjusted_residual=False, stream=None) -> None:
     a = _args(n_images, n_cfg, n_forced, n_draft_max, block, n_draft, kv_k, kv_v, kv_rows, cache_len,
-              cache_len_host, draft_probs, uniforms, cfg_scale, temperature, mode, nbr_k, delta, tree_parent)
+              cache_len_host, draft_probs, uniforms, cfg_scale, temperature, mode, nbr_k, delta, tree_parent,
+              adjusted_residual)
     o = _out(accept_len, next_token, new_len, n_commit, accept_mask, target_probs, hidden, margins, accept_path)
     _check(lib.vvs_verify(ctx, C.byref(a), C.byref(o), _stream(stream)), "vvs_verify")
 
@@ -215,9 +217,10 @@ def vvs_verify(ctx: int, *, n_images, n_cfg, n_forced, n_draft_max, block, kv_k,
 def vvs_epilogue(ctx: int, *, hidden_in, n_rows_per_seq, first_row, drafts, n_images, n_cfg,
                  n_draft_max, draft_probs, uniforms, accept_len, next_token, n_draft=None,
                  cfg_scale=1.0, temperature=1.0, mode=VVS_MODE_STRICT, nbr_k=1, delta=float("inf"),
-                 accept_mask=None, target_probs=None, margins=None, stream=None) -> None:
+                 accept_mask=None, target_probs=None, margins=None, adjusted_residual=False,
+                 stream=None) -> None:
     a = _args(n_images, n_cfg, 1, n_draft_max, None, n_draft, None, None, 0, None, None, draft_probs,
-              uniforms, cfg_scale, temperature, mode, nbr_k, delta)
+              uniforms, cfg_scale, temperature, mode, nbr_k, delta, None, adjusted_residual)
     o = _out(accept_len, next_token, None, None, accept_mask, target_probs, None, margins)
     _check(lib.vvs_epilogue(ctx, _ptr(hidden_in), int(n_rows_per_seq), int(first_row), _ptr(drafts),
                             C.byref(a), C.byref(o), _stream(stream)), "vvs_epilogue")
@@ -226,9 +229,9 @@ def vvs_epilogue(ctx: int, *, hidden_in, n_rows_per_seq, first_row, drafts, n_im
 def vvs_decide(ctx: int, *, target_probs, n_rows_per_seq, first_row, drafts, n_images, n_draft_max,
                draft_probs, uniforms, accept_len, next_token, n_draft=None, mode=VVS_MODE_STRICT,
                nbr_k=1, delta=float("inf"), accept_mask=None, margins=None, tree_parent=None,
-               accept_path=None, stream=None) -> None:
+               accept_path=None, adjusted_residual=False, stream=None) -> None:
     a = _args(n_images, 1, 1, n_draft_max, None, n_draft, None, None, 0, None, None, draft_probs,
-              uniforms, 1.0, 1.0, mode, nbr_k, delta, tree_parent)
+              uniforms, 1.0, 1.0, mode, nbr_k, delta, tree_parent, adjusted_residual)
     o = _out(accept_len, next_token, None, None, accept_mask, None, None, margins, accept_path)
     _check(lib.vvs_decide(ctx, _ptr(target_probs), int(n_rows_per_seq), int(first_row), _ptr(drafts),
                           C.byref(a), C.byref(o), _stream(stream)), "vvs_decide")
@@ -238,13 +241,13 @@ def vvs_decide_noalloc(*, target_probs, vocab, vocab_offset, n_rows_per_seq, fir
                        n_images, n_draft_max, draft_probs, uniforms, accept_len, next_token,
                        nbr_row_ptr=None, nbr_col=None, n_draft=None, mode=VVS_MODE_STRICT, nbr_k=1,
                        delta=float("inf"), accept_mask=None, margins=None, status_bits=None,
-                       tree_parent=None, accept_path=None, stream=None) -> None:
+                       tree_parent=None, accept_path=None, adjusted_residual=False, stream=None) -> None:
     """vvs_decide for callers that must not allocate device memory: no context, scratch in a fixed
     device array inside the library (limits: 64 images, 16 drafts, 64 neighbours, vocab 65536;
     chains only: tree_parent / accept_path are refused).  Calls on one device share that array
     and must not overlap on the GPU."""
     a = _args(n_images, 1, 1, n_draft_max, None, n_draft, None, None, 0, None, None, draft_probs,
-              uniforms, 1.0, 1.0, mode, nbr_k, delta, tree_parent)
+              uniforms, 1.0, 1.0, mode, nbr_k, delta, tree_parent, adjusted_residual)
     o = _out(accept_len, next_token, None, None, accept_mask, None, None, margins, accept_path)
     _check(lib.vvs_decide_noalloc(_ptr(target_probs), int(vocab), int(vocab_offset), int(n_rows_per_seq),
                                   int(first_row), _ptr(drafts), _ptr(nbr_row_ptr), _ptr(nbr_col),

@@ -22,6 +22,31 @@ __device__ __forceinline__ double warp_incl_scan_d(double v, int lane) {
   return v;
 }
 
+// Relaxed numerator (Sec. 2): the longest distance-ordered prefix of neighbour entries 1 .. kk-1
+// whose cumulative mass stays <= delta.  One warp; pn(j) gives the mass of entry j.  Returns the
+// pooled mass (the same value in every lane) and the first entry NOT pooled in *j_end.
+template <typename F>
+__device__ __forceinline__ double pooled_prefix(int kk, double delta, int lane, F pn_of, int* j_end) {
+  double cum = 0.0;
+  int end = kk;
+  for (int j0 = 1; j0 < kk; j0 += 32) {
+    const int j = j0 + lane;
+    const double pn = (j < kk) ? pn_of(j) : 0.0;
+    const double tot = cum + warp_incl_scan_d(pn, lane);
+    const unsigned over = __ballot_sync(0xffffffffu, (j < kk) && (tot > delta));
+    if (over) {
+      const int first = __ffs(over) - 1;
+      const double prev = __shfl_sync(0xffffffffu, tot, first > 0 ? first - 1 : 0);
+      if (first > 0) cum = prev;
+      end = j0 + first;
+      break;
+    }
+    cum = __shfl_sync(0xffffffffu, tot, 31);
+  }
+  *j_end = end;
+  return cum;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Combine per-tile softmax partials: M = max_t m_t, S = sum_t s_t exp(m_t - M), fixed order.
 __global__ void finalize_stats_kernel(const float* __restrict__ part_m, const float* __restrict__ part_s,
@@ -109,22 +134,9 @@ __global__ void accept_kernel(Workspace ws, DecideParams p) {
           if (len < 1 && lane == 0) atomicOr(ws.status, VVS_DEV_BAD_NEIGHBOUR);
           int kk = min(p.nbr_k, len);
           const float* ln = ws.l_nbr + ((size_t)b * K + i) * p.kmax;
-          double cum = 0.0;
-          bool stop = false;
-          for (int j0 = 1; j0 < kk && !stop; j0 += 32) {
-            int j = j0 + lane;
-            double pn = (j < kk) ? (double)(direct ? ln[j] : prob_of(ln[j], m, inv)) : 0.0;
-            double tot = cum + warp_incl_scan_d(pn, lane);
-            unsigned over = __ballot_sync(0xffffffffu, (j < kk) && (tot > (double)p.delta));
-            if (over) {
-              int first = __ffs(over) - 1;
-              double prev = __shfl_sync(0xffffffffu, tot, first > 0 ? first - 1 : 0);
-              if (first > 0) cum = prev;
-              stop = true;
-            } else {
-              cum = __shfl_sync(0xffffffffu, tot, 31);
-            }
-          }
+          int j_end;
+          const double cum = pooled_prefix(kk, (double)p.delta, lane, [&](int j) {
+            return (double)(direct ? ln[j] : prob_of(ln[j], m, inv)); }, &j_end);
           mass += cum;
         }
         double qx = (double)p.draft_probs[((size_t)b * K + i) * V + x];
@@ -205,6 +217,49 @@ void launch_select_p_row(const float* logits, const Workspace& ws, int n_images,
 }
 
 // ---------------------------------------------------------------------------------------------
+// Adjusted target of a relaxed rejection (flag adjusted_residual): in the row image b samples
+// from, the pooled neighbours of the rejected draft x give their mass to x.  The row lives in
+// ws.p_row (copied there first when the caller's probabilities are used directly); the pooled
+// prefix is found again from the row's own float32 values, by the rule of accept_kernel.
+// grid B, 256 threads.
+__global__ void adjust_target_kernel(Workspace ws, DecideParams p) {
+  const int b = blockIdx.x, V = p.vocab;
+  const int sel = ws.sel_row[b];
+  if (sel < 0) return;
+  float* row = ws.p_row + (size_t)b * V;
+  if (p.direct_probs) {
+    const float* src = p.direct_probs + (size_t)sel * V;
+    for (int j = threadIdx.x; j < V; j += blockDim.x) row[j] = src[j];
+    __syncthreads();
+  }
+  if (ws.sel_kind[b] != 0 || threadIdx.x >= 32) return;    // bonus row: nothing was rejected
+  const int lane = threadIdx.x;
+  const int n = p.accept_len[b];
+  const int x = p.drafts[(size_t)b * p.drafts_ld + n] - p.vocab_offset;
+  if (x < 0 || x >= V) return;                             // reported by the acceptance kernel
+  const int beg = p.row_ptr[x], len = p.row_ptr[x + 1] - beg;
+  const int kk = min(p.nbr_k, len);
+  auto mass_of = [&](int j) {
+    const int c = p.col[beg + j];
+    return (c >= 0 && c < V) ? (double)row[c] : 0.0;
+  };
+  int j_end;
+  const double cum = pooled_prefix(kk, (double)p.delta, lane, mass_of, &j_end);
+  const double mass = (double)row[x] + cum;
+  __syncwarp();
+  for (int j = 1 + lane; j < j_end; j += 32) {
+    const int c = p.col[beg + j];
+    if (c >= 0 && c < V) row[c] = 0.f;
+  }
+  __syncwarp();
+  if (lane == 0) row[x] = (float)mass;
+}
+
+void launch_adjust_target(const Workspace& ws, const DecideParams& p, cudaStream_t s) {
+  adjust_target_kernel<<<p.n_images, 256, 0, s>>>(ws, p);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Residual distribution (Sec. 2): r = max(0, p - q_n) at the first rejected draft n, or r = p for
 // the bonus token; float32 difference, float64 accumulation.
 __device__ __forceinline__ float residual_value(float pr, const float* q_row, int j, int kind) {
@@ -222,7 +277,7 @@ __global__ void residual_mass_kernel(Workspace ws, DecideParams p, int n_chunks)
   const float* q_row = p.draft_probs + ((size_t)b * K + (kind == 0 ? n : 0)) * V;
   const int sel = ws.sel_row[b];
   if (sel < 0) return;  // no row to sample from: sample_kernel reports -1
-  const float* p_row = p.direct_probs ? p.direct_probs + (size_t)sel * V : ws.p_row + (size_t)b * V;
+  const float* p_row = (p.direct_probs && !p.adjusted) ? p.direct_probs + (size_t)sel * V : ws.p_row + (size_t)b * V;
   double sr = 0.0, sp = 0.0;
   int end = min(V, (c + 1) * kSampleChunk);
   for (int j = c * kSampleChunk + threadIdx.x; j < end; j += blockDim.x) {
@@ -308,8 +363,8 @@ __global__ void sample_kernel(Workspace ws, DecideParams p, int n_chunks) {
   int n = p.accept_len[b];
   int eff_kind = s_use_p ? 1 : kind;
   const float* q_row = p.draft_probs + ((size_t)b * K + (eff_kind == 0 ? n : 0)) * V;
-  const float* p_row = p.direct_probs ? p.direct_probs + (size_t)ws.sel_row[b] * V
-                                      : ws.p_row + (size_t)b * V;
+  const float* p_row = (p.direct_probs && !p.adjusted) ? p.direct_probs + (size_t)ws.sel_row[b] * V
+                                                       : ws.p_row + (size_t)b * V;
   int j = s_chunk * kSampleChunk + threadIdx.x;
   double val = 0.0;
   if (j < V) val = (double)residual_value(p_row[j], q_row, j, eff_kind);

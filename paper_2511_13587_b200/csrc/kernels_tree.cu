@@ -5,6 +5,9 @@
 // child is left the next token is drawn from the last residual.  A chain-shaped tree reduces to
 // the chain rule of Sec. 2 bit for bit: the first residual is the float32 difference of the two
 // float32 rows, later rounds (which a chain never reaches) work in float64.
+// Relaxed mode: the numerator is the pooled mass of x and its neighbours in the current p_res
+// (the chain's relaxed rule with p_res in the place of p); with the adjusted-residual flag a
+// rejection subtracts q from p_res after the pooled neighbours' mass has been moved onto x.
 //
 // One CTA per image; the walk is sequential over tree depth and siblings, each residual update
 // and the final inverse-CDF draw are block-wide passes over the V codes.  Sums run in a fixed
@@ -33,6 +36,30 @@ __device__ __forceinline__ double tw_warp_scan(double v, int lane) {
   return v;
 }
 
+// Longest distance-ordered prefix of neighbour entries 1 .. kk-1 whose cumulative mass stays
+// <= delta (one warp; the pooled mass in every lane, the first entry not pooled in *j_end).
+template <typename F>
+__device__ __forceinline__ double tw_pooled_prefix(int kk, double delta, int lane, F pn_of, int* j_end) {
+  double cum = 0.0;
+  int end = kk;
+  for (int j0 = 1; j0 < kk; j0 += 32) {
+    const int j = j0 + lane;
+    const double pn = (j < kk) ? pn_of(j) : 0.0;
+    const double tot = cum + tw_warp_scan(pn, lane);
+    const unsigned over = __ballot_sync(0xffffffffu, (j < kk) && (tot > delta));
+    if (over) {
+      const int first = __ffs(over) - 1;
+      const double prev = __shfl_sync(0xffffffffu, tot, first > 0 ? first - 1 : 0);
+      if (first > 0) cum = prev;
+      end = j0 + first;
+      break;
+    }
+    cum = __shfl_sync(0xffffffffu, tot, 31);
+  }
+  *j_end = end;
+  return cum;
+}
+
 // Sum over the block, the same value in every thread (two barriers).
 __device__ double tw_block_sum(double v, double* s_warp) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -48,7 +75,8 @@ __device__ double tw_block_sum(double v, double* s_warp) {
 __global__ void __launch_bounds__(kTreeThreads) tree_walk_kernel(TreeParams p) {
   __shared__ double s_warp[kTreeThreads / 32];
   __shared__ int s_child[32];
-  __shared__ int s_n, s_pass, s_first, s_last;
+  __shared__ int s_n, s_pass, s_first, s_last, s_jend;
+  __shared__ double s_mass;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int F = p.n_forced, K = p.n_draft_max, T = p.t_len, V = p.vocab;
   const int32_t* par = p.parent + (size_t)b * T;
@@ -88,19 +116,34 @@ __global__ void __launch_bounds__(kTreeThreads) tree_walk_kernel(TreeParams p) {
       const float* qrow = p.draft_probs + ((size_t)b * K + i) * V;
       const int x = p.drafts[(size_t)b * p.drafts_ld + i] - p.vocab_offset;
       const bool x_ok = x >= 0 && x < V;
-      if (tid == 0) {
+      if (warp == 0) {
         int pass = 0;
         if (!x_ok) {
-          atomicOr(p.status, VVS_DEV_BAD_TOKEN);
+          if (lane == 0) atomicOr(p.status, VVS_DEV_BAD_TOKEN);
         } else {
-          const double px = first_round ? (double)prow[x] : buf[src][x] / z;
+          double px = first_round ? (double)prow[x] : buf[src][x] / z;
+          int j_end = 1;
+          if (p.relaxed) {
+            const int beg = p.row_ptr[x], len = p.row_ptr[x + 1] - beg;
+            if (len < 1 && lane == 0) atomicOr(p.status, VVS_DEV_BAD_NEIGHBOUR);
+            const int kk = min(p.nbr_k, len);
+            const double* cur_res = first_round ? nullptr : buf[src];
+            px += tw_pooled_prefix(kk, (double)p.delta, lane, [&](int j) {
+              const int cc = p.col[beg + j];
+              if (cc < 0 || cc >= V) return 0.0;
+              return cur_res ? cur_res[cc] / z : (double)prow[cc]; }, &j_end);
+          }
           const double qx = (double)qrow[x];
           const double ratio = qx > 0.0 ? fmin(1.0, px / qx) : (px > 0.0 ? 1.0 : 0.0);
           const double u = (double)p.uniforms[(size_t)b * (K + 1) + i];
-          if (p.margins) p.margins[(size_t)b * (K + 1) + i] = (float)fabs(u - ratio);
+          if (lane == 0 && p.margins) p.margins[(size_t)b * (K + 1) + i] = (float)fabs(u - ratio);
           pass = u < ratio ? 1 : 0;
+          if (lane == 0) {
+            s_mass = px;
+            s_jend = j_end;
+          }
         }
-        s_pass = pass;
+        if (lane == 0) s_pass = pass;
       }
       __syncthreads();
       const int pass = s_pass;
@@ -126,6 +169,24 @@ __global__ void __launch_bounds__(kTreeThreads) tree_walk_kernel(TreeParams p) {
           dst[v] = r;
           local += r;
         }
+      }
+      if (p.adjusted) {
+        // adjusted target of the rejected child: its pooled neighbours carry no mass, the child
+        // carries the pooled mass; the touched entries are rewritten and the sum is taken again
+        __syncthreads();
+        const int beg = p.row_ptr[x];
+        const int j_end = s_jend;
+        for (int j = 1 + tid; j < j_end; j += kTreeThreads) {
+          const int cc = p.col[beg + j];
+          if (cc >= 0 && cc < V) dst[cc] = 0.0;
+        }
+        __syncthreads();
+        if (tid == 0)
+          dst[x] = first_round ? (double)fmaxf(0.f, __fsub_rn((float)s_mass, qrow[x]))
+                               : fmax(0.0, __dsub_rn(s_mass, (double)qrow[x]));
+        __syncthreads();
+        local = 0.0;
+        for (int v = tid; v < V; v += kTreeThreads) local += dst[v];
       }
       const double z_new = tw_block_sum(local, s_warp);
       if (z_new > 0.0) {                          // else p_res == q numerically: keep p_res

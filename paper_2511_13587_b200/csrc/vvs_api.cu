@@ -143,6 +143,7 @@ DecideParams decide_params(const vvs_ctx* ctx, int rows_per_seq, int first_row, 
   p.n_draft_max = a->n_draft_max; p.vocab = md.vocab; p.vocab_offset = md.vocab_offset;
   p.mode = a->mode; p.nbr_k = a->mode == VVS_MODE_RELAXED ? a->nbr_k : 1; p.kmax = md.max_nbr_k;
   p.delta = a->delta;
+  p.adjusted = (a->mode == VVS_MODE_RELAXED && a->nbr_k > 1 && a->adjusted_residual) ? 1 : 0;
   p.drafts = drafts; p.drafts_ld = drafts_ld; p.n_draft = a->n_draft;
   p.draft_probs = a->draft_probs; p.uniforms = a->uniforms;
   p.row_ptr = ctx->nbr_row_ptr; p.col = ctx->nbr_col;
@@ -196,6 +197,7 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
       VVS_LAUNCH(VVS_PROF_OTHER, launch_select_p_row(lbuf, ws, B, V, s));
       if (o->target_probs)
         VVS_LAUNCH(VVS_PROF_OTHER, launch_probs_from_logits(o->target_probs, ws, o->target_probs, BT, V, s));
+      if (p.adjusted) VVS_LAUNCH(VVS_PROF_OTHER, launch_adjust_target(ws, p, s));
       VVS_LAUNCH(VVS_PROF_OTHER, launch_residual_mass(ws, p, s));
       VVS_LAUNCH(VVS_PROF_OTHER, launch_sample(ws, p, s));
       return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
@@ -207,6 +209,7 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
     lr.row_mode = 1; lr.sel_row = ws.sel_row; lr.stat_m = ws.stat_m; lr.stat_inv = ws.stat_inv; lr.p_row = ws.p_row;
     VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_lmhead_tc(lr, s));
     if (rc != VVS_OK) return rc;
+    if (p.adjusted) VVS_LAUNCH(VVS_PROF_OTHER, launch_adjust_target(ws, p, s));
     VVS_LAUNCH(VVS_PROF_OTHER, launch_residual_mass(ws, p, s));
     VVS_LAUNCH(VVS_PROF_OTHER, launch_sample(ws, p, s));
     return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
@@ -221,6 +224,7 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
   if (o->target_probs)
     VVS_LAUNCH(VVS_PROF_OTHER, launch_probs_from_logits(ws.logits, ws, o->target_probs, BT, V, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_select_p_row(ws.logits, ws, B, V, s));
+  if (p.adjusted) VVS_LAUNCH(VVS_PROF_OTHER, launch_adjust_target(ws, p, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_residual_mass(ws, p, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_sample(ws, p, s));
   return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
@@ -295,6 +299,8 @@ int run_tree_decisions(vvs_ctx* ctx, const __nv_bfloat16* hid, const vvs_verify_
   tp.drafts_ld = Tn;
   tp.probs = o->target_probs; tp.draft_probs = a->draft_probs; tp.uniforms = a->uniforms; tp.cache_len = a->cache_len;
   tp.res = ws.tree_res; tp.accept_len = o->accept_len;
+  tp.relaxed = (a->mode == VVS_MODE_RELAXED && a->nbr_k > 1) ? 1 : 0; tp.nbr_k = a->nbr_k; tp.delta = a->delta;
+  tp.adjusted = (tp.relaxed && a->adjusted_residual) ? 1 : 0; tp.row_ptr = ctx->nbr_row_ptr; tp.col = ctx->nbr_col;
   tp.accept_path = o->accept_path ? o->accept_path : ws.tree_path;
   tp.next_token = o->next_token; tp.new_len = o->new_len; tp.n_commit = o->n_commit;
   tp.accept_mask = o->accept_mask; tp.margins = o->margins; tp.status = ws.status;
@@ -482,7 +488,7 @@ int verify_via_graph(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_ou
   ka.cache_len = a->cache_len;   // cache_len_host: host-side validation only, not part of the device work
   ka.draft_probs = a->draft_probs; ka.uniforms = a->uniforms; ka.cfg_scale = a->cfg_scale;
   ka.temperature = a->temperature; ka.mode = a->mode; ka.nbr_k = a->nbr_k; ka.delta = a->delta;
-  ka.tree_parent = a->tree_parent;
+  ka.tree_parent = a->tree_parent; ka.adjusted_residual = a->adjusted_residual;
   std::vector<unsigned char> key(sizeof(ka) + sizeof(*o));
   std::memcpy(key.data(), &ka, sizeof(ka));
   std::memcpy(key.data() + sizeof(ka), o, sizeof(*o));   // nine pointers, no padding
@@ -543,6 +549,7 @@ int check_decision_args(const vvs_ctx* ctx, const vvs_verify_args* a, const vvs_
   if (!(a->temperature > 0.f) || !std::isfinite(a->temperature) || !std::isfinite(a->cfg_scale))
     return VVS_ERR_INVALID_ARG;
   if (a->mode != VVS_MODE_STRICT && a->mode != VVS_MODE_RELAXED) return VVS_ERR_INVALID_ARG;
+  if (a->adjusted_residual != 0 && a->adjusted_residual != 1) return VVS_ERR_INVALID_ARG;
   if (a->mode == VVS_MODE_RELAXED) {
     if (a->nbr_k < 1 || a->nbr_k > md.max_nbr_k) return VVS_ERR_SHAPE;
     if (!(a->delta >= 0.f)) return VVS_ERR_INVALID_ARG;  // also rejects NaN
@@ -749,7 +756,7 @@ int vvs_verify(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* o, 
   if (!a->block || !a->kv_k || !a->kv_v || !a->cache_len || !o->new_len) return VVS_ERR_INVALID_ARG;
   if (a->kv_rows < R) return VVS_ERR_SHAPE;
   if (a->tree_parent) {
-    if (a->mode != VVS_MODE_STRICT || a->n_draft || !o->target_probs) return VVS_ERR_INVALID_ARG;
+    if (a->n_draft || !o->target_probs) return VVS_ERR_INVALID_ARG;
     if (!ctx->tensor_core_path) return VVS_ERR_SHAPE;     // Tn <= 32 = max_block holds for every call
   } else if (o->accept_path) {
     return VVS_ERR_INVALID_ARG;
@@ -806,13 +813,15 @@ int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, 
   Workspace& ws = ctx->ws;
   if (a->tree_parent) {
     // the tree walk on the caller's rows: block rows 0 .. first_row are the forced chain
-    if (a->mode != VVS_MODE_STRICT || a->n_draft || !ws.tree_res) return VVS_ERR_INVALID_ARG;
+    if (a->n_draft || !ws.tree_res) return VVS_ERR_INVALID_ARG;
     if (first_row + 1 + a->n_draft_max != n_rows_per_seq) return VVS_ERR_SHAPE;
     TreeParams tp{};
     tp.n_images = a->n_images; tp.n_cfg = 1; tp.n_forced = first_row + 1; tp.n_draft_max = a->n_draft_max;
     tp.t_len = n_rows_per_seq; tp.vocab = ctx->desc.vocab; tp.vocab_offset = ctx->desc.vocab_offset;
     tp.parent = a->tree_parent; tp.drafts = drafts; tp.drafts_ld = a->n_draft_max; tp.probs = target_probs;
     tp.draft_probs = a->draft_probs; tp.uniforms = a->uniforms; tp.res = ws.tree_res;
+    tp.relaxed = (a->mode == VVS_MODE_RELAXED && a->nbr_k > 1) ? 1 : 0; tp.nbr_k = a->nbr_k; tp.delta = a->delta;
+    tp.adjusted = (tp.relaxed && a->adjusted_residual) ? 1 : 0; tp.row_ptr = ctx->nbr_row_ptr; tp.col = ctx->nbr_col;
     tp.accept_len = o->accept_len; tp.accept_path = o->accept_path ? o->accept_path : ws.tree_path;
     tp.next_token = o->next_token; tp.accept_mask = o->accept_mask; tp.margins = o->margins; tp.status = ws.status;
     VVS_LAUNCH(VVS_PROF_OTHER, launch_tree_walk(tp, s));
@@ -822,6 +831,7 @@ int vvs_decide(vvs_ctx* ctx, const float* target_probs, int32_t n_rows_per_seq, 
   p.direct_probs = target_probs;
   if (p.n_draft_max > 0) VVS_LAUNCH(VVS_PROF_OTHER, launch_gather_logits(target_probs, ws, p, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_accept(ws, p, s));
+  if (p.adjusted) VVS_LAUNCH(VVS_PROF_OTHER, launch_adjust_target(ws, p, s));   // copies the row, then adjusts it
   VVS_LAUNCH(VVS_PROF_OTHER, launch_residual_mass(ws, p, s));
   VVS_LAUNCH(VVS_PROF_OTHER, launch_sample(ws, p, s));
   return cudaGetLastError() == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;

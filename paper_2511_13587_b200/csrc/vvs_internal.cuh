@@ -299,6 +299,9 @@ struct TreeParams {
   const float* uniforms;      // [B, K+1]
   const int32_t* cache_len;
   double* res;                // [2][B, V]
+  int relaxed, nbr_k, adjusted;   // relaxed acceptance on the current residual; adjusted-residual flag
+  float delta;
+  const int32_t* row_ptr; const int32_t* col;
   int32_t* accept_len; int32_t* accept_path; int32_t* next_token; int32_t* new_len; int32_t* n_commit;
   uint8_t* accept_mask; float* margins;
   int32_t* status;
@@ -348,6 +351,7 @@ struct DecideParams {
   int n_images, n_cfg, rows_per_seq, first_row, n_draft_max, vocab, vocab_offset;
   int mode, nbr_k, kmax;
   float delta;
+  int adjusted;               // relaxed mode: the residual's p is the adjusted target of the rejected draft
   const int32_t* drafts;      // [B, drafts_ld] embedding ids
   int drafts_ld;
   const int32_t* n_draft;     // [B] or null
@@ -372,6 +376,7 @@ void launch_accept(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_probs_from_logits(const float* logits, const Workspace& ws, float* probs, int n_rows,
                               int v, cudaStream_t s);
 void launch_select_p_row(const float* logits, const Workspace& ws, int n_images, int v, cudaStream_t s);
+void launch_adjust_target(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_residual_mass(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 void launch_sample(const Workspace& ws, const DecideParams& p, cudaStream_t s);
 

@@ -80,6 +80,7 @@ extern "C" int vvs_decide_noalloc(const float* target_probs, int32_t vocab, int3
   if (o->new_len || o->n_commit || o->hidden || o->target_probs) return VVS_ERR_INVALID_ARG;
   // chains only: a candidate tree would need the walk's float64 scratch rows, which this array has not
   if (a->tree_parent || o->accept_path) return VVS_ERR_INVALID_ARG;
+  if (a->adjusted_residual != 0) return VVS_ERR_INVALID_ARG;   // needs a writable copy of the sampled row
   if (!aligned16(target_probs) || !aligned16(a->draft_probs)) return VVS_ERR_ALIGN;
 
   unsigned char* base = nullptr;

@@ -87,7 +87,7 @@ def run_oracle(case) -> dict:
     return O.verify(c["ms"], c["w"], c["block"], c["n_forced"], c["n_draft"], c["kv_k"][:, :n_rows],
                     c["kv_v"][:, :n_rows], c["cache_len"], c["draft_probs"], c["uniforms"],
                     c["n_cfg"], c["cfg_scale"], c["temperature"], c["mode"], c["row_ptr"], c["col"],
-                    c["nbr_k"], c["delta"])
+                    c["nbr_k"], c["delta"], c.get("adjusted_residual", False))
 
 
 # ---------------------------------------------------------------------------------------
@@ -159,7 +159,8 @@ class GpuRunner:
                       kv_rows=c["kv_rows"], cache_len=cache_len,
                       draft_probs=to_dev(c["draft_probs"]), uniforms=to_dev(c["uniforms"]),
                       cfg_scale=c["cfg_scale"], temperature=c["temperature"], mode=c["mode"],
-                      nbr_k=c["nbr_k"], delta=c["delta"], **o)
+                      nbr_k=c["nbr_k"], delta=c["delta"],
+                      adjusted_residual=c.get("adjusted_residual", False), **o)
         status = vb.vvs_device_status(self.ctx)
         res = {k_: (to_host(v) if v is not None else None) for k_, v in o.items()}
         res["status"] = status
@@ -187,7 +188,7 @@ def replay_decisions(case, gpu_probs: np.ndarray) -> dict:
     for b in range(c["n_images"]):
         d = O.decide(gpu_probs[b].astype(np.float32), c["block"][b, c["n_forced"]:] - ms.vocab_offset,
                      int(c["n_draft"][b]), c["n_forced"], c["draft_probs"][b], c["uniforms"][b],
-                     c["mode"], c["row_ptr"], c["col"], c["nbr_k"], c["delta"])
+                     c["mode"], c["row_ptr"], c["col"], c["nbr_k"], c["delta"], c.get("adjusted_residual", False))
         out["accept_len"].append(d["accept_len"])
         out["next_token"].append(d["next_token"] + ms.vocab_offset if d["next_token"] >= 0 else -1)
         out["accept_mask"].append(d["accept_mask"])
@@ -302,7 +303,9 @@ def run_tree_oracle(case) -> dict:
     n_rows = c["n_images"] * c["n_cfg"]
     return O.tree_verify(c["ms"], c["w"], c["block"], c["parent"], c["n_forced"], c["kv_k"][:, :n_rows],
                          c["kv_v"][:, :n_rows], c["cache_len"], c["draft_probs"], c["uniforms"],
-                         c["n_cfg"], c["cfg_scale"], c["temperature"])
+                         c["n_cfg"], c["cfg_scale"], c["temperature"], c.get("mode", MODE_STRICT), c.get("row_ptr"),
+                         c.get("col"), c.get("nbr_k", 1), c.get("delta", float("inf")),
+                         c.get("adjusted_residual", False))
 
 
 def run_tree_gpu(runner: "GpuRunner", case) -> dict:
@@ -320,10 +323,15 @@ def run_tree_gpu(runner: "GpuRunner", case) -> dict:
              margins=torch.zeros((b, k + 1), dtype=torch.float32, device="cuda"),
              target_probs=torch.zeros((b, t_len, ms.vocab), dtype=torch.float32, device="cuda"),
              hidden=torch.zeros((r, t_len, ms.d_model), dtype=torch.bfloat16, device="cuda"))
+    if c.get("row_ptr") is not None:
+        rp, col = to_dev(c["row_ptr"]), to_dev(c["col"])
+        vb.vvs_bind_neighbors(runner.ctx, rp, col)
     vb.vvs_verify(runner.ctx, n_images=b, n_cfg=cfg, n_forced=f, n_draft_max=k, block=to_dev(c["block"]),
                   kv_k=kv_k, kv_v=kv_v, kv_rows=c["kv_rows"], cache_len=to_dev(c["cache_len"]),
                   draft_probs=to_dev(c["draft_probs"]), uniforms=to_dev(c["uniforms"]),
-                  cfg_scale=c["cfg_scale"], temperature=c["temperature"], tree_parent=to_dev(c["parent"]), **o)
+                  cfg_scale=c["cfg_scale"], temperature=c["temperature"], tree_parent=to_dev(c["parent"]),
+                  mode=c.get("mode", MODE_STRICT), nbr_k=c.get("nbr_k", 1), delta=c.get("delta", float("inf")),
+                  adjusted_residual=c.get("adjusted_residual", False), **o)
     res = {k_: to_host(v) for k_, v in o.items()}
     res["status"] = vb.vvs_device_status(runner.ctx)
     res["launches"] = vb.vvs_last_launch_count(runner.ctx)

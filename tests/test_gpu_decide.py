@@ -41,7 +41,7 @@ def oracle_decide(c):
     for b in range(c["n_images"]):
         d = O.decide(c["probs"][b], c["drafts"][b] - off, int(c["n_draft"][b]), c["first_row"] + 1,
                      c["draft_probs"][b], c["uniforms"][b], c["mode"], c["row_ptr"], c["col"],
-                     c["nbr_k"], c["delta"])
+                     c["nbr_k"], c["delta"], c.get("adjusted_residual", False))
         res["accept_len"].append(d["accept_len"])
         res["next_token"].append(d["next_token"] + off if d["next_token"] >= 0 else -1)
         res["accept_mask"].append(d["accept_mask"])
@@ -110,6 +110,38 @@ def test_decide_is_bit_exact_with_oracle(v, n_images, k, rows, first_row, mode, 
     vb.vvs_destroy(ctx)
 
 
+@pytest.mark.parametrize("v,n_images,k,rows,first_row,mode,nbr_k,delta,tau,gumbel,off",
+                         [c for c in CASES if c[5] == MODE_RELAXED])
+def test_adjusted_residual_is_bit_exact_with_oracle(v, n_images, k, rows, first_row, mode, nbr_k, delta, tau,
+                                                    gumbel, off):
+    """The adjusted-residual flag: same acceptances as the plain relaxed call, the sample drawn
+    from the adjusted target's residual; on some image the two samples must differ."""
+    from paper_2511_13587_b200 import binding as vb
+    c = decide_case(v + k, v, n_images, k, rows, first_row, mode, nbr_k, delta, tau, gumbel, off)
+    ctx = vb.vvs_create(vb.make_desc(c["ms"], n_images, rows, nbr_k))
+
+    def call(flag):
+        def run(d, o):
+            vb.vvs_bind_neighbors(ctx, d["row_ptr"], d["col"])
+            vb.vvs_decide(ctx, target_probs=d["target_probs"], n_rows_per_seq=rows, first_row=first_row,
+                          drafts=d["drafts"], n_images=n_images, n_draft_max=k, n_draft=d["n_draft"],
+                          draft_probs=d["draft_probs"], uniforms=d["uniforms"], mode=mode, nbr_k=nbr_k,
+                          delta=delta, adjusted_residual=flag, **o)
+        return run
+    plain = gpu_decide(c, call(False))
+    adj = gpu_decide(c, call(True))
+    assert vb.vvs_device_status(ctx) == 0
+    want = oracle_decide(dict(c, adjusted_residual=True))
+    compare_exact(c, adj, want)
+    np.testing.assert_array_equal(adj["accept_len"], plain["accept_len"])
+    rejected = adj["accept_len"] < c["n_draft"]
+    print("rejections", int(rejected.sum()), "of", n_images)
+    if rejected.sum() >= 3:
+        assert (adj["next_token"][rejected] != plain["next_token"][rejected]).any()
+    np.testing.assert_array_equal(adj["next_token"][~rejected], plain["next_token"][~rejected])
+    vb.vvs_destroy(ctx)
+
+
 # ---------------------------------------------------------------------------------------
 # candidate trees: the walk of vvs_verify's tree calls on given probabilities
 
@@ -143,10 +175,15 @@ def tree_decide_case(seed, v, n_images, k, n_forced, tau, gumbel, off=0):
                 rows=rows, n_forced=n_forced)
 
 
+@pytest.mark.parametrize("mode,nbr_k,delta,adjusted", [(MODE_STRICT, 1, float("inf"), False),
+                                                       (MODE_RELAXED, 16, float("inf"), False),
+                                                       (MODE_RELAXED, 64, 0.1, True),
+                                                       (MODE_RELAXED, 8, float("inf"), True)])
 @pytest.mark.parametrize("v,n_images,k,n_forced,tau,gumbel,off",
                          [(1000, 64, 12, 1, 1.0, 0.5, 0), (16384, 32, 15, 3, 0.5, 1.5, 100),
                           (4096 + 40, 16, 31, 1, 1.0, 2.5, 0), (512, 64, 6, 2, 2.0, 3.0, 7)])
-def test_tree_walk_is_exact_on_random_trees(v, n_images, k, n_forced, tau, gumbel, off):
+def test_tree_walk_is_exact_on_random_trees(v, n_images, k, n_forced, tau, gumbel, off, mode, nbr_k, delta,
+                                            adjusted):
     """Same float32 inputs on both sides: accepted paths and sampled tokens must be equal; only
     decisions within 1e-12 of their threshold (float64 summation order of a later-round
     normaliser, or of the sampling CDF) are left out."""
@@ -154,7 +191,12 @@ def test_tree_walk_is_exact_on_random_trees(v, n_images, k, n_forced, tau, gumbe
     from paper_2511_13587_b200 import binding as vb
     c = tree_decide_case(v + k, v, n_images, k, n_forced, tau, gumbel, off)
     rows = c["rows"]
-    ctx = vb.vvs_create(vb.make_desc(c["ms"], n_images, rows, 1))
+    ctx = vb.vvs_create(vb.make_desc(c["ms"], n_images, rows, nbr_k))
+    row_ptr = col = None
+    if mode == MODE_RELAXED:
+        row_ptr, col = gen.neighbour_csr(gen.make_codebook(v + k, v), nbr_k)
+        rp_d, col_d = H.to_dev(row_ptr), H.to_dev(col)
+        vb.vvs_bind_neighbors(ctx, rp_d, col_d)
     o = dict(accept_len=torch.full((n_images,), -7, dtype=torch.int32, device="cuda"),
              next_token=torch.full((n_images,), -7, dtype=torch.int32, device="cuda"),
              accept_mask=torch.full((n_images, k), 9, dtype=torch.uint8, device="cuda"),
@@ -163,14 +205,15 @@ def test_tree_walk_is_exact_on_random_trees(v, n_images, k, n_forced, tau, gumbe
     vb.vvs_decide(ctx, target_probs=H.to_dev(c["probs"]), n_rows_per_seq=rows, first_row=n_forced - 1,
                   drafts=H.to_dev(c["drafts"]), n_images=n_images, n_draft_max=k,
                   draft_probs=H.to_dev(c["draft_probs"]), uniforms=H.to_dev(c["uniforms"]),
-                  tree_parent=H.to_dev(c["parent"]), **o)
+                  tree_parent=H.to_dev(c["parent"]), mode=mode, nbr_k=nbr_k, delta=delta,
+                  adjusted_residual=adjusted, **o)
     torch.cuda.synchronize()
     assert vb.vvs_device_status(ctx) == 0
     got = {k_: H.to_host(t) for k_, t in o.items()}
     judged = rejected_rounds = 0
     for b in range(n_images):
         d = O.tree_decide(c["probs"][b], c["drafts"][b] - off, c["parent"][b], n_forced, c["draft_probs"][b],
-                          c["uniforms"][b])
+                          c["uniforms"][b], mode, row_ptr, col, nbr_k, delta, adjusted)
         if np.any(d["margins"][:k] < 1e-12):
             continue
         n = int(got["accept_len"][b])

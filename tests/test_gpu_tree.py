@@ -12,6 +12,7 @@ import pytest
 import helpers as H
 from oracle import vvs_oracle as O
 from test_gpu_verify import _tols
+from vvs_synth import gen
 from vvs_synth.configs import B7_SMALL, MODE_RELAXED, XL_SMALL
 
 pytestmark = pytest.mark.gpu
@@ -30,7 +31,9 @@ def _replay(case, gpu):
     for b in range(c["n_images"]):
         out.append(O.tree_decide(gpu["target_probs"][b].astype(np.float32),
                                  c["block"][b, c["n_forced"]:] - ms.vocab_offset, c["parent"][b],
-                                 c["n_forced"], c["draft_probs"][b], c["uniforms"][b]))
+                                 c["n_forced"], c["draft_probs"][b], c["uniforms"][b],
+                                 c.get("mode", 0), c.get("row_ptr"), c.get("col"), c.get("nbr_k", 1),
+                                 c.get("delta", float("inf")), c.get("adjusted_residual", False)))
     return out
 
 
@@ -102,6 +105,24 @@ def test_tree_parity_xl_small(parent, n_forced, n_images, fills, q_noise):
     run.close()
 
 
+@pytest.mark.parametrize("nbr_k,delta,adjusted", [(64, float("inf"), False), (16, 0.05, True), (64, float("inf"), True)])
+def test_relaxed_tree_parity_xl_small(nbr_k, delta, adjusted):
+    """Relaxed acceptance on a candidate tree (the pooled mass is taken in the current residual),
+    with and without the adjusted-residual flag, through vvs_verify against the oracle's walk."""
+    ms = XL_SMALL
+    case = H.build_tree_case(ms, 52, 2, 2, 1, TREE_C, [40, 311], q_noise=1.5)
+    case.update(mode=MODE_RELAXED, nbr_k=nbr_k, delta=delta, adjusted_residual=adjusted)
+    case["row_ptr"], case["col"] = gen.neighbour_csr(gen.make_codebook(52, ms.vocab), nbr_k)
+    run = H.GpuRunner(ms, case["w"], 4, len(TREE_C), max_nbr_k=nbr_k)
+    gpu = H.run_tree_gpu(run, case)
+    ora = H.run_tree_oracle(case)
+    _check_tree(case, gpu, ora)
+    strict = _replay(dict(case, mode=0), gpu)
+    print("relaxed tree paths", [list(g[:n]) for g, n in zip(gpu["accept_path"], gpu["accept_len"])],
+          "strict walk on the same rows", [r["accept_path"] for r in strict])
+    run.close()
+
+
 def test_tree_parity_7b_small_1d_rope():
     """1-D rope: a node's position is fill + depth, not fill + index."""
     ms = B7_SMALL
@@ -150,7 +171,8 @@ def test_tree_argument_errors():
     bad = dict(case, parent=np.array([[-1, 0, 0, 1, 1, 1, 2, 8, 7]], dtype=np.int32))   # parent after child
     gpu = H.run_tree_gpu(run, bad)
     assert gpu["status"] & vb.VVS_DEV_BAD_ARG
-    # relaxed acceptance and a missing probability buffer are refused before any launch
+    # a missing probability buffer, a relaxed call without a neighbour table and a flag value other
+    # than 0 / 1 are refused before any launch
     b, r, k, t_len = 1, 2, 8, 9
     common = dict(n_images=b, n_cfg=2, n_forced=1, n_draft_max=k, block=H.to_dev(case["block"]),
                   kv_k=H.to_dev(case["kv_k"]), kv_v=H.to_dev(case["kv_v"]), kv_rows=case["kv_rows"],
@@ -163,7 +185,9 @@ def test_tree_argument_errors():
         vb.vvs_verify(run.ctx, **common)
     probs = torch.zeros((b, t_len, ms.vocab), dtype=torch.float32, device="cuda")
     with pytest.raises(vb.VvsError):
-        vb.vvs_verify(run.ctx, mode=MODE_RELAXED, nbr_k=1, target_probs=probs, **common)
+        vb.vvs_verify(run.ctx, mode=MODE_RELAXED, nbr_k=2, target_probs=probs, **common)
+    with pytest.raises(vb.VvsError):
+        vb.vvs_verify(run.ctx, adjusted_residual=2, target_probs=probs, **common)
     run.close()
 
 

@@ -119,6 +119,38 @@ def test_xl_shape_small_bf16_cfg(n_images, fills, deterministic):
     run.close()
 
 
+@pytest.mark.parametrize("n_images,want_probs", [(4, True), (4, False), (12, False)])
+def test_relaxed_acceptance_adjusted_residual_bf16(n_images, want_probs):
+    """The adjusted-residual flag through vvs_verify on all three decision routes: probabilities
+    written out, guided logits in scratch (at most 64 decision rows), and the second LM-head pass
+    that recomputes the sampled row (more than 64 decision rows)."""
+    ms = XL_SMALL
+    fills = [10, 200, 333, 574, 55, 123, 400, 9, 77, 501, 268, 31][:n_images]
+    case = H.build_case_independent(ms, 29, n_images, 2, 1, 8, fills, mode=MODE_RELAXED, nbr_k=16,
+                                    logit_std=2.5)
+    case["adjusted_residual"] = True
+    run = H.GpuRunner(ms, case["w"], 2 * n_images, 9, max_nbr_k=16)
+    gpu = run.verify(case, want_probs=True)
+    if not want_probs:                                  # the route under test emits no probabilities:
+        gpu2 = run.verify(case, want_probs=False)       # its integers must equal the checked route's
+        m = H.replay_decisions(case, gpu["target_probs"])["margins"]   # (two runs differ in the last bits)
+        clear = (m[:, :8] > 1e-2).all(axis=1)
+        np.testing.assert_array_equal(gpu2["accept_len"][clear], gpu["accept_len"][clear])
+        # the sampled code sits in a CDF bin about 1/V wide; run-to-run differences of the rows
+        # may move a sample point across an edge now and then
+        assert clear.sum() >= n_images // 2
+        assert (gpu2["next_token"][clear] != gpu["next_token"][clear]).sum() <= max(1, n_images // 4)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    plain = run.verify(dict(case, adjusted_residual=False))
+    m = H.replay_decisions(case, gpu["target_probs"])["margins"]
+    clear = (m[:, :8] > 1e-2).all(axis=1)
+    np.testing.assert_array_equal(plain["accept_len"][clear], gpu["accept_len"][clear])
+    rejected = clear & (gpu["accept_len"] < 8)
+    assert rejected.any() and (plain["next_token"][rejected] != gpu["next_token"][rejected]).any()
+    run.close()
+
+
 @pytest.mark.parametrize("delta", [float("inf"), 0.1, 0.0])
 def test_relaxed_acceptance_bf16(delta):
     ms = XL_SMALL
