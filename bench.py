@@ -93,7 +93,7 @@ def host_trial(wl, trial: int) -> dict:
     ms = wl.shape
     b, k, f = wl.n_images, wl.n_draft_max, wl.n_forced
     fills = gen.make_fills(wl.seed, b, wl.fill_lo, wl.fill_hi, trial)
-    q, drafts = gen.independent_draft(wl.seed, trial, b, k, ms.vocab, DRAFT_LOGIT_STD)
+    q, drafts = gen.independent_draft(wl.seed, trial, b, k, ms.vocab, wl.q_noise_std)
     forced = gen.random_tokens(wl.seed, f"forced.{trial}", (b, f), ms.vocab_offset,
                                ms.vocab_offset + ms.vocab)
     block = np.concatenate([forced, drafts + ms.vocab_offset], axis=1).astype(np.int32)
@@ -167,7 +167,8 @@ class VerifyBench:
     """One workload resident on this process's GPU: weights, caches, a library context, the
     seeded trials and the step function that the timed regions repeat."""
 
-    def __init__(self, index: int, rank: int = 0, deterministic: bool = False, n_trials: int = N_TRIALS):
+    def __init__(self, index: int, rank: int = 0, deterministic: bool = False, n_trials: int = N_TRIALS,
+                 draft: str = "target"):
         import torch
         from paper_2511_13587_b200 import binding as vb
         from vvs_synth.configs import DTYPE_BF16
@@ -210,7 +211,9 @@ class VerifyBench:
             self.kv_v[l].copy_(torch.randn(self.kv_v[l].shape, generator=g, device="cuda"))
         # the seeded cache, kept aside: set-up and statistics calls start from it, while the timed
         # calls leave their block rows behind in the live cache like a decoding loop does
-        self.kv0_k, self.kv0_v = self.kv_k.clone(), self.kv_v.clone()
+        self.kv0_k = self.kv0_v = None
+        if index != 0 and draft == "target":
+            self.kv0_k, self.kv0_v = self.kv_k.clone(), self.kv_v.clone()
         self.wd = wd
         self.ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, wl.nbr_k, deterministic=deterministic))
         vb.vvs_bind_weights(self.ctx, wd)
@@ -234,7 +237,7 @@ class VerifyBench:
         self.keys = ("cache_len", "block", "draft_probs", "uniforms", "n_draft", "skip_mask", "gamma")
         self.trials = [host_trial(wl, t) for t in range(n_trials)]
         self.dtr = [{n: dev(t[n]) for n in self.keys} for t in self.trials]
-        if index == 0:
+        if index == 0 or draft == "independent":
             self.drafter = f"independent softmax(N(0,{wl.q_noise_std}^2))"
         else:
             self._draft_from_target()
@@ -278,8 +281,9 @@ class VerifyBench:
         torch.cuda.synchronize()
 
     def restore_cache(self):
-        self.kv_k.copy_(self.kv0_k)
-        self.kv_v.copy_(self.kv0_v)
+        if self.kv0_k is not None:
+            self.kv_k.copy_(self.kv0_k)
+            self.kv_v.copy_(self.kv0_v)
 
     def step(self, inp, out=None):
         vb, ctx = self.vb, self.ctx
@@ -409,7 +413,7 @@ def run_ours(args) -> None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    S = VerifyBench(args.workload, rank, bool(args.deterministic))
+    S = VerifyBench(args.workload, rank, bool(args.deterministic), n_trials=args.trials, draft=args.draft)
     wl, ms, vb = S.wl, S.ms, S.vb
     warm = max(args.warmup, 3)
 
@@ -902,6 +906,10 @@ def main() -> None:
                     help="1: fixed-order sums (bitwise repeatable), 0: arrival-order split-K sums (faster)")
     ap.add_argument("--cpu-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--trials", type=int, default=N_TRIALS, help="distinct seeded inputs cycled through the steps")
+    ap.add_argument("--draft", default="target", choices=["target", "independent"],
+                    help="target: drafter rows from the library's own target logits plus noise (K set-up calls per "
+                         "trial); independent: rows that ignore the target (no set-up calls: short profiler runs)")
     ap.add_argument("--no-other", action="store_true",
                     help="skip the short measurements of the other workloads that the default line carries")
     args = ap.parse_args()

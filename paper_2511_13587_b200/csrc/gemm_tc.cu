@@ -435,7 +435,9 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
   for (int s = 1; s <= max_splits; ++s) {
     const long long per_cta = (pl.kb_total + s - 1) / s;
     const long long waves = ((long long)pl.tiles * s * pl.passes + slots - 1) / slots;
-    const long long cost = per_cta * waves * 64 + s;  // mild preference for fewer splits
+    // mild preference for fewer splits.  (Measured at 288 tokens: charging a split for its extra atomic
+    // adds, i.e. fewer and longer CTAs, made every projection slower, not faster.)
+    const long long cost = per_cta * waves * 64 + s;
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
       best = s;

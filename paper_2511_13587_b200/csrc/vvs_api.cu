@@ -349,6 +349,12 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
       make_tmap_bf16_2d(&tm_act, act, (uint64_t)M, (uint64_t)ff, (uint32_t)p_down.nt) != VVS_OK)
     return VVS_ERR_CUDA;
 
+  const bool rows_attention = wide && attention_rows_applicable(md, Tn);
+  AttentionRowsArgs ar{};
+  ar.qkv = ws.qkv; ar.kv_k = kv_k; ar.kv_v = kv_v; ar.cache_len = a->cache_len; ar.rope_cos = ws.rope_cos;
+  ar.rope_sin = ws.rope_sin; ar.anc_mask = ws.anc_mask; ar.out = attn; ar.d = d; ar.n_heads = md.n_heads;
+  ar.hd = md.head_dim; ar.s_max = md.s_max; ar.kv_rows = a->kv_rows; ar.t_len = Tn; ar.n_rows = R; ar.pdl = ctx->use_pdl;
+
   GemmTcArgs base{};
   base.m = M; base.pdl = ctx->use_pdl; base.status = ws.status;
   base.scratch = ws.sk_scratch; base.counters = ws.sk_counters;
@@ -425,16 +431,22 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
       GemmTcArgs g = base;
       g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.out = ws.qkv; g.ldo = 3 * d;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_qkv, g, s));
-      VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_append<T>(ws.qkv, ws.rope_inv_freq, q, kv_k, kv_v, a->cache_len, md,
-                                                       l, a->kv_rows, R, Tn, ws.status, s,
-                                                       a->tree_parent ? ws.rope_cos : nullptr,
-                                                       a->tree_parent ? ws.rope_sin : nullptr, true));
+      if (rows_attention) {
+        // rotation, rounding, cache append and attention of each (sequence, head) in one kernel
+        ar.layer = l;
+        if (rc == VVS_OK) VVS_LAUNCH(VVS_PROF_ATTENTION, rc = launch_attention_rows(ar, s));
+      } else {
+        VVS_LAUNCH(VVS_PROF_OTHER, launch_rope_append<T>(ws.qkv, ws.rope_inv_freq, q, kv_k, kv_v, a->cache_len, md,
+                                                         l, a->kv_rows, R, Tn, ws.status, s,
+                                                         a->tree_parent ? ws.rope_cos : nullptr,
+                                                         a->tree_parent ? ws.rope_sin : nullptr, true));
+      }
     } else {
       GemmTcArgs g = base;
       g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.ld_scratch = 3 * d; g.layer = l;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_QKV, p_qkv, g, s));
     }
-    if (rc == VVS_OK) {
+    if (rc == VVS_OK && !(wide && rows_attention)) {
       at.layer = l;
       VVS_LAUNCH(VVS_PROF_ATTENTION, rc = launch_attention_tc(at, s));
     }

@@ -249,6 +249,22 @@ struct AttentionTcArgs {
 };
 int launch_attention_tc(const AttentionTcArgs& a, cudaStream_t s);
 
+// ---- row-batched attention with fused rotation / cache append, attention_rows.cu ----------------------
+struct AttentionRowsArgs {
+  float* qkv;                  // [M, 3 d] fp32 split-K sums of the QKV projection; read, then cleared
+  __nv_bfloat16* kv_k;         // cache [layers][kv_rows][heads][s_max][hd]; slots fill .. fill + T - 1 are written
+  __nv_bfloat16* kv_v;
+  const int32_t* cache_len;    // [R]
+  const float* rope_cos;       // [M, hd / 2] rotation table of the step
+  const float* rope_sin;
+  const uint32_t* anc_mask;    // [M] visible block rows per block row
+  __nv_bfloat16* out;          // [M, d]
+  int d, n_heads, hd, s_max, layer, kv_rows, t_len, n_rows;
+  bool pdl;
+};
+bool attention_rows_applicable(const vvs_model_desc& md, int t_len);
+int launch_attention_rows(const AttentionRowsArgs& a, cudaStream_t s);
+
 // ---- LM head with fused decision epilogue, lmhead_tc.cu -------------------------------------------
 struct LmHeadArgs {
   int v, k, bt, n_cfg;           // codebook size, d_model, decision rows, 1 or 2 feature rows per decision row
