@@ -106,9 +106,61 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const T* __restrict_
   for (int i = threadIdx.x; i < d; i += blockDim.x) o[i] = from_f<T>(row[i] * rs * to_f(scale[i]));
 }
 
+// The same for many rows of a bf16 context: one warp per row, 16-byte loads, no shared memory; as a
+// programmatic dependent of the projection before it (the row is read after griddepcontrol.wait).
+__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* __restrict__ x,
+                                                           const __nv_bfloat16* __restrict__ scale,
+                                                           __nv_bfloat16* __restrict__ out, int m, int d, float eps) {
+  const int lane = threadIdx.x & 31, row_i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (row_i >= m) return;
+  const float* row = x + (size_t)row_i * d;
+  float ss = 0.f;
+  for (int i = lane * 4; i < d; i += 128) {
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(row + i));
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float rs = rsqrtf(ss / (float)d + eps);
+  __nv_bfloat16* o = out + (size_t)row_i * d;
+  for (int i = lane * 4; i < d; i += 128) {
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(row + i));
+    const uint2 g = *reinterpret_cast<const uint2*>(scale + i);
+    const __nv_bfloat162 g0 = *reinterpret_cast<const __nv_bfloat162*>(&g.x);
+    const __nv_bfloat162 g1 = *reinterpret_cast<const __nv_bfloat162*>(&g.y);
+    __nv_bfloat162 r0 = __floats2bfloat162_rn(v.x * rs * __bfloat162float(g0.x), v.y * rs * __bfloat162float(g0.y));
+    __nv_bfloat162 r1 = __floats2bfloat162_rn(v.z * rs * __bfloat162float(g1.x), v.w * rs * __bfloat162float(g1.y));
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&r0);
+    pk.y = *reinterpret_cast<uint32_t*>(&r1);
+    *reinterpret_cast<uint2*>(o + i) = pk;
+  }
+}
+
 template <typename T>
 void launch_rmsnorm(const float* x, const T* scale, T* out, int m, int d, float eps, cudaStream_t s) {
   rmsnorm_kernel<T><<<m, 256, 0, s>>>(x, scale, out, d, eps);
+}
+
+static cudaError_t launch_dependent(const void* fn, dim3 grid, dim3 block, void** args, bool pdl, cudaStream_t s) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelExC(&cfg, fn, args);
+}
+
+void launch_rmsnorm_rows(const float* x, const __nv_bfloat16* scale, __nv_bfloat16* out, int m, int d, float eps,
+                         bool pdl, cudaStream_t s) {
+  void* args[] = {&x, &scale, &out, &m, &d, &eps};
+  launch_dependent(reinterpret_cast<const void*>(rmsnorm_rows_kernel), dim3((m + 7) / 8), dim3(256), args, pdl, s);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -304,6 +356,8 @@ __global__ void silu_mul_kernel(float* __restrict__ gu, T* __restrict__ act, int
   float* row = gu + (size_t)blockIdx.y * 2 * ff;
   T* o = act + (size_t)blockIdx.y * ff;
   const int j = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // returns at once unless launched as a programmatic dependent
   if (j >= ff) return;                       // ff is a multiple of 8
   const float4 g = *reinterpret_cast<const float4*>(row + j);
   const float4 u = *reinterpret_cast<const float4*>(row + ff + j);
@@ -319,8 +373,11 @@ __global__ void silu_mul_kernel(float* __restrict__ gu, T* __restrict__ act, int
 }
 
 template <typename T>
-void launch_silu_mul(float* gu, T* act, int m, int ff, cudaStream_t s, bool clear_src) {
-  silu_mul_kernel<T><<<dim3((ff + 1023) / 1024, m), 256, 0, s>>>(gu, act, ff, clear_src ? 1 : 0);
+void launch_silu_mul(float* gu, T* act, int m, int ff, cudaStream_t s, bool clear_src, bool pdl) {
+  int clear = clear_src ? 1 : 0;
+  void* args[] = {&gu, &act, &ff, &clear};
+  launch_dependent(reinterpret_cast<const void*>(silu_mul_kernel<T>), dim3((ff + 1023) / 1024, m), dim3(256), args,
+                   pdl, s);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -380,7 +437,7 @@ void launch_row_stats(const float* logits, float* part_m, float* part_s, int n_r
                                       cudaStream_t, const float*, const float*, bool);               \
   template void launch_attention<T>(const T*, const T*, const T*, const int32_t*, T*,                \
                                     const vvs_model_desc&, int, int, int, int, cudaStream_t);        \
-  template void launch_silu_mul<T>(float*, T*, int, int, cudaStream_t, bool);
+  template void launch_silu_mul<T>(float*, T*, int, int, cudaStream_t, bool, bool);
 VVS_INSTANTIATE(float)
 VVS_INSTANTIATE(__nv_bfloat16)
 

@@ -424,7 +424,12 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   for (int l = 0; l < md.n_layers && rc == VVS_OK; ++l) {
     const Layer& L = ctx->layers[l];
     const LayerMaps& W = ctx->layer_maps[l];
-    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm1), xn, M, d, md.rms_eps, s));
+    // many rows: the warp-per-row norm, launched as a programmatic dependent of the projection before it
+    const bool rows_norm = wide && d % 8 == 0;
+    if (rows_norm)
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm_rows(ws.x, static_cast<const __nv_bfloat16*>(L.norm1), xn, M, d, md.rms_eps, ctx->use_pdl && l > 0, s));
+    else
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm1), xn, M, d, md.rms_eps, s));
     if (wide) {
       // many tokens: a per-thread epilogue over hundreds of tokens is slower than a plain split-K
       // sum into fp32 followed by one thread per element for rotation, rounding and cache append
@@ -455,14 +460,17 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
       g.n = d; g.k = d; g.tm_a = &W.w_o; g.tm_b = &tm_attn; g.out = ws.x; g.ldo = d;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_o, g, s));
     }
-    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm2), xn, M, d, md.rms_eps, s));
+    if (rows_norm)
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm_rows(ws.x, static_cast<const __nv_bfloat16*>(L.norm2), xn, M, d, md.rms_eps, ctx->use_pdl, s));
+    else
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(L.norm2), xn, M, d, md.rms_eps, s));
     if (rc == VVS_OK && wide) {
       GemmTcArgs g = base;
       g.n = ff; g.k = d; g.tm_a = &W.w_gate; g.tm_b = &tm_xn; g.out = ws.gu; g.ldo = 2 * ff;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_g1, g, s));
       g.tm_a = &W.w_up; g.out = ws.gu + ff;
       if (rc == VVS_OK) VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_g1, g, s));
-      VVS_LAUNCH(VVS_PROF_OTHER, launch_silu_mul<T>(ws.gu, act, M, ff, s, true));
+      VVS_LAUNCH(VVS_PROF_OTHER, launch_silu_mul<T>(ws.gu, act, M, ff, s, true, ctx->use_pdl));
     } else if (rc == VVS_OK) {
       GemmTcArgs g = base;
       g.n = ff; g.k = d; g.tm_a = &W.w_gate; g.tm_a2 = &W.w_up; g.tm_b = &tm_xn; g.ld_scratch = 2 * ff;
@@ -475,7 +483,10 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     }
   }
   if (rc != VVS_OK) return rc;
-  VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
+  if (wide && d % 8 == 0)
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm_rows(ws.x, static_cast<const __nv_bfloat16*>(ctx->norm_f), hid, M, d, md.rms_eps, ctx->use_pdl, s));
+  else
+    VVS_LAUNCH(VVS_PROF_OTHER, launch_rmsnorm<T>(ws.x, static_cast<const T*>(ctx->norm_f), hid, M, d, md.rms_eps, s));
   if (cudaGetLastError() != cudaSuccess) return VVS_ERR_CUDA;
   if (a->tree_parent) return run_tree_decisions(ctx, hid, a, o, s);
   return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);

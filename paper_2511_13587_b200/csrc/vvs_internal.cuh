@@ -203,7 +203,9 @@ void launch_attention(const T* q, const T* kv_k, const T* kv_v, const int32_t* c
                       const vvs_model_desc& md, int layer, int kv_rows, int n_rows, int t_len,
                       cudaStream_t s);
 template <typename T>
-void launch_silu_mul(float* gu, T* act, int m, int ff, cudaStream_t s, bool clear_src = false);
+void launch_silu_mul(float* gu, T* act, int m, int ff, cudaStream_t s, bool clear_src = false, bool pdl = false);
+void launch_rmsnorm_rows(const float* x, const __nv_bfloat16* scale, __nv_bfloat16* out, int m, int d, float eps,
+                         bool pdl, cudaStream_t s);
 void launch_guide(const float* raw, float* logits, int n_images, int n_cfg, int rows_per_seq, int v,
                   float cfg_scale, float inv_temp, cudaStream_t s);
 void launch_row_stats(const float* logits, float* part_m, float* part_s, int n_rows, int v,
