@@ -197,6 +197,23 @@ def test_per_projection_kernels_head_dims_and_long_blocks(ms, n_images, n_forced
     run.close()
 
 
+@pytest.mark.parametrize("ms,n_forced,k,fills",
+                         [(XL_SMALL, 1, 8, [0, 63, 64, 65, 128, 583]),    # empty cache, 64-key block edges, block fills the cache
+                          (XL_SMALL, 2, 30, [129, 500]),                  # 32 rows per sequence: two full m-tiles
+                          (B7_SMALL, 1, 8, [0, 64, 191, 391])])           # head_dim 128; 391 + 9 rows = capacity
+def test_row_batched_attention_edges(ms, n_forced, k, fills):
+    """More than 64 block tokens: rotation, cache append and attention run per (sequence, head) in one
+    kernel that streams the cached keys in 64-key blocks."""
+    n_images = len(fills)
+    case = H.build_case_independent(ms, 83 + k, n_images, 2, n_forced, k, fills, logit_std=0.5)
+    assert n_images * 2 * (n_forced + k) > 64
+    run = H.GpuRunner(ms, case["w"], 2 * n_images, n_forced + k)
+    gpu = run.verify(case)
+    ora = H.run_oracle(case)
+    _check_end_to_end(case, gpu, ora)
+    run.close()
+
+
 @pytest.mark.parametrize("deterministic", [True, False])
 def test_ragged_drafts_forced_prefix_and_cache_edges(deterministic):
     """n_draft below K (including 0), two forced rows, an empty cache and a cache that the block
