@@ -33,6 +33,10 @@ from vvs_synth.configs import CONFIGS, MODE_RELAXED  # noqa: E402
 # kernel's source file and the first 16 hex digits of that file's SHA-256 when the counters were
 # taken: the line reports null once the file has changed since.
 NCU_CAPTURES = {
+    (1, False): ("paper_2511_13587_b200/csrc/fused_chain.cu", "76919ebd16cc78e6", 1.4800e9,
+                 "profiles/fused_chain_kernel_configs1_ncu_full.txt"),
+    (1, True): ("paper_2511_13587_b200/csrc/chain_stream.cu", "59094e79f0fee11d", 1.4597e9,
+                "profiles/chain_stream_kernel_configs1_ncu_full.txt"),
 }
 N_TRIALS = 32           # distinct (fill, block, draft) inputs cycled through the steps
 DRAFT_LOGIT_STD = 1.0   # target-independent drafter: q = softmax(N(0, std^2))
@@ -423,7 +427,7 @@ def run_ours(args) -> None:
     barrier()
     S.launches = 0
     with ClockSampler(local) as clocks:
-        regions = timed_regions(S.region, args.steps, world, barrier)
+        regions = timed_regions(S.region, args.steps, world, barrier, min_ms=args.min_ms)
     gpu_launches = S.launches // len(regions)
     ms_region = float(np.median(regions))
     status = vb.vvs_device_status(S.ctx)
@@ -464,7 +468,7 @@ def run_ours(args) -> None:
 
     for i in range(3):
         step_e2e(i)
-    regions_e2e = timed_regions(lambda n: S.region(n, step_e2e), args.steps, world, barrier)
+    regions_e2e = timed_regions(lambda n: S.region(n, step_e2e), args.steps, world, barrier, min_ms=args.min_ms)
     ms_e2e = float(np.median(regions_e2e))
 
     # ---- per-kernel-class timing for the roofline (separate pass, not the headline) -----------
@@ -906,6 +910,9 @@ def main() -> None:
                     help="1: fixed-order sums (bitwise repeatable), 0: arrival-order split-K sums (faster)")
     ap.add_argument("--cpu-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-ms", type=float, default=500.0,
+                    help="the --steps-long timed region is repeated until this much device time has been measured "
+                         "(the line reports the median region); profiler runs pass a small value")
     ap.add_argument("--trials", type=int, default=N_TRIALS, help="distinct seeded inputs cycled through the steps")
     ap.add_argument("--draft", default="target", choices=["target", "independent"],
                     help="target: drafter rows from the library's own target logits plus noise (K set-up calls per "
