@@ -846,7 +846,7 @@ def run_tree_step(args) -> None:
     kv_k = torch.randn((ms.n_layers, r, ms.n_heads, ms.s_max, ms.head_dim), generator=g,
                        device="cuda").to(torch.bfloat16)
     kv_v = torch.randn_like(kv_k)
-    ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, 1))
+    ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, 1, deterministic=bool(args.deterministic)))
     vb.vvs_bind_weights(ctx, wd)
     trials = []
     for t in range(N_TRIALS):
@@ -908,7 +908,7 @@ def main() -> None:
     ap.add_argument("--workload", type=int, default=1, choices=[0, 1, 2, 3, 4, 5, 6])
     ap.add_argument("--deterministic", type=int, default=0, choices=[0, 1],
                     help="1: fixed-order sums (bitwise repeatable), 0: arrival-order split-K sums (faster)")
-    ap.add_argument("--cpu-steps", type=int, default=4)
+    ap.add_argument("--cpu-steps", type=int, default=2)   # 5-16 s of host time at configs[1], depending on the host
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--min-ms", type=float, default=500.0,
                     help="the --steps-long timed region is repeated until this much device time has been measured "
