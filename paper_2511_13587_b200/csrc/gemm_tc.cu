@@ -33,7 +33,7 @@ constexpr uint32_t kATileBytes = kTileRows * kBlockK * 2;
 
 struct KernelParams {
   int m, n, k;
-  int nt, passes, kb_total, splits, stages;
+  int nt, passes, kb_total, splits, stages, wide_add;
   uint32_t tmem_cols;
   float* scratch;
   int ld_scratch;
@@ -257,7 +257,36 @@ gemm_tc_kernel(const KernelParams p, const __grid_constant__ CUtensorMap tm_a,
       do_final = s_last != 0;
       if (do_final) __threadfence();
     }
-    if (do_final) {
+    if (EPI == GEMM_EPI_ADD && p.wide_add) {
+      // Many tokens: the tile goes through shared memory (token-major, the ring is free once the
+      // accumulator is complete) so that each thread adds four consecutive output columns of one
+      // token with ONE vector reduction: a quarter of the reduction instructions, 512 contiguous
+      // bytes per warp.
+      float* sT = reinterpret_cast<float*>(smem);
+      constexpr int kLd = (int)kTileRows + 4;
+      const int ntok = min(p.nt, p.m - tok0);
+      for (int c0 = 0; c0 < ntok; c0 += 16) {
+        float v[16];
+        tmem_ld16(t_row + c0, v);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) sT[(c0 + j) * kLd + (int)threadIdx.x] = v[j];
+      }
+      __syncthreads();
+      const int n_base = tile * (int)kTileRows;
+      for (int idx = threadIdx.x; idx < ntok * (int)(kTileRows / 4); idx += blockDim.x) {
+        const int tk = idx >> 5, g4 = (idx & 31) * 4;
+        const float4 val = *reinterpret_cast<const float4*>(sT + tk * kLd + g4);
+        float* dst = p.out + (size_t)(tok0 + tk) * p.ldo + n_base + g4;
+        if (n_base + g4 + 3 < p.n) {
+          asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(val.x), "f"(val.y), "f"(val.z),
+                       "f"(val.w) : "memory");
+        } else {
+          if (n_base + g4 < p.n) atomicAdd(dst, val.x);
+          if (n_base + g4 + 1 < p.n) atomicAdd(dst + 1, val.y);
+          if (n_base + g4 + 2 < p.n) atomicAdd(dst + 2, val.z);
+        }
+      }
+    } else if (do_final) {
       for (int c0 = 0; c0 < p.nt && tok0 + c0 < p.m; c0 += 16) {
         float v[16], v2[16];
         if (fixup) {
@@ -451,7 +480,10 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
   if (stages > per_cta) stages = per_cta;
   if (stages < 1) stages = 1;
   pl.stages = stages;
-  pl.smem_bytes = stages * (int)stage_bytes + 1024;
+  pl.smem_bytes = stages * (int)stage_bytes;
+  // calls of many tokens stage the accumulator tile for vector reductions: nt rows of 132 floats
+  if (pl.nt > 32 && !dual && pl.smem_bytes < pl.nt * ((int)kTileRows + 4) * 4) pl.smem_bytes = pl.nt * ((int)kTileRows + 4) * 4;
+  pl.smem_bytes += 1024;
   uint32_t cols = 32;
   while (cols < (uint32_t)pl.nt * (dual ? 2u : 1u)) cols <<= 1;
   pl.tmem_cols = (int)cols;
@@ -463,6 +495,8 @@ int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStr
   kp.m = g.m; kp.n = g.n; kp.k = g.k;
   kp.nt = plan.nt; kp.passes = plan.passes; kp.kb_total = plan.kb_total; kp.splits = plan.splits;
   kp.stages = plan.stages; kp.tmem_cols = (uint32_t)plan.tmem_cols;
+  kp.wide_add = (epi == GEMM_EPI_ADD && plan.nt > 32 && g.ldo % 4 == 0 &&
+                 (reinterpret_cast<uintptr_t>(g.out) & 15) == 0) ? 1 : 0;
   kp.scratch = g.scratch; kp.ld_scratch = g.ld_scratch; kp.counters = g.counters; kp.status = g.status;
   kp.out = g.out; kp.ldo = g.ldo;
   kp.q = g.q; kp.kv_k = g.kv_k; kp.kv_v = g.kv_v; kp.slot_pos = g.slot_pos;
