@@ -560,6 +560,7 @@ def other_workloads(args, pk: dict) -> dict:
     out = {"configs[1] fixed-order sums": quick_measure(1, True, 64, pk),
            "configs[0]": quick_measure(0, False, 256, pk, min_ms=100.0),
            "configs[2]": quick_measure(2, False, 16, pk),
+           "configs[2] fixed-order sums": quick_measure(2, True, 16, pk),
            "configs[3]": quick_measure(3, False, 16, pk),
            "configs[3] fixed-order sums": quick_measure(3, True, 16, pk),
            "configs[4]": epilogue_sweep(steps=20, pk=pk)}

@@ -98,7 +98,7 @@ typedef struct vvs_model_desc {
   int32_t max_nbr_k;     /* largest neighbour count k in relaxed mode (>= 1) */
   float rms_eps;
   float rope_base;
-  int32_t deterministic; /* bf16 contexts, calls of at most 32 block tokens (n_images * n_cfg * T):
+  int32_t deterministic; /* bf16 contexts:
                             1 = every sum of the decoder is taken in a fixed order, so the same call
                                 gives the same bits every time (target_probs, hidden, the appended
                                 K / V rows and hence next_token); vvs_bind_weights then keeps a private
@@ -107,8 +107,11 @@ typedef struct vvs_model_desc {
                                 the measured numbers in the repository's notes), the last bits of the
                                 logits differ from run to run, and a residual sample over many nearly
                                 equally likely codes need not repeat.
-                            Calls of more than 32 block tokens use arrival-order sums in either mode;
-                            float32 contexts are always repeatable. */
+                            With 1, calls of at most 32 block tokens (n_images * n_cfg * T) run the
+                            streaming whole-chain kernel; larger calls split each projection's K range
+                            over a thread-block cluster that adds its partial tiles in rank order through
+                            distributed shared memory (about a quarter slower than the arrival-order
+                            reductions).  float32 contexts are always repeatable. */
 } vvs_model_desc;
 
 /* Per-layer weights, device, type T.  Projection matrices are [out_features, in_features]

@@ -33,7 +33,7 @@ constexpr uint32_t kATileBytes = kTileRows * kBlockK * 2;
 
 struct KernelParams {
   int m, n, k;
-  int nt, passes, kb_total, splits, stages, wide_add;
+  int nt, passes, kb_total, splits, stages, wide_add, cluster_mode;
   uint32_t tmem_cols;
   float* scratch;
   int ld_scratch;
@@ -104,6 +104,18 @@ __device__ __forceinline__ void final_chunk(const KernelParams& p, int n, int to
       }
     }
   }
+}
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t local_addr, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+  return v;
 }
 
 template <int EPI>
@@ -222,6 +234,10 @@ gemm_tc_kernel(const KernelParams p, const __grid_constant__ CUtensorMap tm_a,
     if (!got) s_abort = 1;
     if (__syncthreads_or(got ? 0 : 1)) {
       if (threadIdx.x == 0) atomicOr(p.status, VVS_DEV_TIMEOUT);
+      if (EPI == GEMM_EPI_ADD && p.cluster_mode) {   // the other CTAs of the cluster wait on these two barriers
+        cluster_sync_all();
+        cluster_sync_all();
+      }
       alive = false;
       break;
     }
@@ -273,6 +289,39 @@ gemm_tc_kernel(const KernelParams p, const __grid_constant__ CUtensorMap tm_a,
       }
       __syncthreads();
       const int n_base = tile * (int)kTileRows;
+      if (p.cluster_mode) {
+        // The K splits of this (tile, token pass) are the CTAs of one cluster (cluster rank = split).
+        // Rank r sums token rows r, r + splits, ... over all ranks' staged tiles in rank order and is
+        // the only writer of those outputs.
+        cluster_sync_all();
+        const uint32_t rank = (uint32_t)split, nrank = (uint32_t)p.splits;
+        const int mine = ntok > (int)rank ? (ntok - (int)rank + (int)nrank - 1) / (int)nrank : 0;
+        const uint32_t sT_addr = smem_u32(sT);
+        for (int idx = threadIdx.x; idx < mine * (int)(kTileRows / 4); idx += blockDim.x) {
+          const int tk = (int)rank + (idx >> 5) * (int)nrank, g4 = (idx & 31) * 4;
+          float4 part[8];                                   // all remote loads in flight, then summed in rank order
+#pragma unroll
+          for (uint32_t q = 0; q < 8; ++q)
+            if (q < nrank) part[q] = ld_cluster_f4(sT_addr + (uint32_t)(tk * kLd + g4) * 4u, q);
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (uint32_t q = 0; q < 8; ++q)
+            if (q < nrank) { acc.x += part[q].x; acc.y += part[q].y; acc.z += part[q].z; acc.w += part[q].w; }
+          float* dst = p.out + (size_t)(tok0 + tk) * p.ldo + n_base + g4;
+          if (n_base + g4 + 3 < p.n) {
+            if (p.cluster_mode == 2) {
+              const float4 o = *reinterpret_cast<const float4*>(dst);
+              acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+            }
+            *reinterpret_cast<float4*>(dst) = acc;
+          } else {
+            const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
+            for (int e = 0; e < 4; ++e)
+              if (n_base + g4 + e < p.n) dst[e] = (p.cluster_mode == 2 ? dst[e] : 0.f) + a4[e];
+          }
+        }
+        cluster_sync_all();      // nobody leaves while its tile may still be read
+      } else
       for (int idx = threadIdx.x; idx < ntok * (int)(kTileRows / 4); idx += blockDim.x) {
         const int tk = idx >> 5, g4 = (idx & 31) * 4;
         const float4 val = *reinterpret_cast<const float4*>(sT + tk * kLd + g4);
@@ -419,11 +468,22 @@ cudaError_t launch_one(const GemmTcPlan& plan, const KernelParams& kp, const CUt
   cfg.blockDim = dim3(128, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  if (pdl) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (kp.cluster_mode && plan.splits > 1) {          // the K splits of a tile: one cluster along grid y
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 1;
+    attr[na].val.clusterDim.y = (unsigned)plan.splits;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = pdl ? 1 : 0;
+  cfg.numAttrs = na;
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, kp, a, a2, b);
 }
 
@@ -449,7 +509,7 @@ int make_weight_tmap(CUtensorMap* out, const void* w, int rows, int cols) {
   return make_tmap_bf16_2d(out, w, (uint64_t)rows, (uint64_t)cols, kTileRows);
 }
 
-GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_sms) {
+GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_sms, int split_cap) {
   GemmTcPlan pl{};
   pl.passes = (m + 255) / 256;
   const int per = (m + pl.passes - 1) / pl.passes;
@@ -459,7 +519,8 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
   // split K so that one wave of CTAs covers the SMs with as few K blocks per CTA as possible
   int best = 1;
   long long best_cost = -1;
-  const int max_splits = allow_split ? (pl.kb_total < 32 ? pl.kb_total : 32) : 1;
+  const int cap = split_cap < 32 ? split_cap : 32;
+  const int max_splits = allow_split ? (pl.kb_total < cap ? pl.kb_total : cap) : 1;
   const long long slots = (long long)n_sms * (pl.passes > 1 ? 2 : 1);   // several passes: two CTAs per SM
   for (int s = 1; s <= max_splits; ++s) {
     const long long per_cta = (pl.kb_total + s - 1) / s;
@@ -482,7 +543,7 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
   pl.stages = stages;
   pl.smem_bytes = stages * (int)stage_bytes;
   // calls of many tokens stage the accumulator tile for vector reductions: nt rows of 132 floats
-  if (pl.nt > 32 && !dual && pl.smem_bytes < pl.nt * ((int)kTileRows + 4) * 4) pl.smem_bytes = pl.nt * ((int)kTileRows + 4) * 4;
+  if (!dual && pl.smem_bytes < pl.nt * ((int)kTileRows + 4) * 4) pl.smem_bytes = pl.nt * ((int)kTileRows + 4) * 4;
   pl.smem_bytes += 1024;
   uint32_t cols = 32;
   while (cols < (uint32_t)pl.nt * (dual ? 2u : 1u)) cols <<= 1;
@@ -495,8 +556,10 @@ int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStr
   kp.m = g.m; kp.n = g.n; kp.k = g.k;
   kp.nt = plan.nt; kp.passes = plan.passes; kp.kb_total = plan.kb_total; kp.splits = plan.splits;
   kp.stages = plan.stages; kp.tmem_cols = (uint32_t)plan.tmem_cols;
-  kp.wide_add = (epi == GEMM_EPI_ADD && plan.nt > 32 && g.ldo % 4 == 0 &&
+  kp.wide_add = (epi == GEMM_EPI_ADD && (plan.nt > 32 || g.cluster_mode) && g.ldo % 4 == 0 &&
                  (reinterpret_cast<uintptr_t>(g.out) & 15) == 0) ? 1 : 0;
+  kp.cluster_mode = (kp.wide_add && plan.splits <= 8) ? g.cluster_mode : 0;
+  if (g.cluster_mode && !kp.cluster_mode) return VVS_ERR_SHAPE;   // the caller planned for a cluster
   kp.scratch = g.scratch; kp.ld_scratch = g.ld_scratch; kp.counters = g.counters; kp.status = g.status;
   kp.out = g.out; kp.ldo = g.ldo;
   kp.q = g.q; kp.kv_k = g.kv_k; kp.kv_v = g.kv_v; kp.slot_pos = g.slot_pos;

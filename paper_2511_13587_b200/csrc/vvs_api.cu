@@ -326,12 +326,22 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   T* act = static_cast<T*>(ws.act);
   T* hid = o->hidden ? static_cast<T*>(o->hidden) : static_cast<T*>(ws.hid);
 
-  const GemmTcPlan p_qkv = plan_gemm_tc(M, 3 * d, d, false, true, ctx->n_sms);
-  const GemmTcPlan p_o = plan_gemm_tc(M, d, d, false, true, ctx->n_sms);
+  const GemmTcPlan p_qkv = plan_gemm_tc(M, 3 * d, d, false, true, ctx->n_sms, (md.deterministic != 0) ? 8 : 32);
+  const GemmTcPlan p_o = plan_gemm_tc(M, d, d, false, true, ctx->n_sms, (md.deterministic != 0) ? 8 : 32);
   const GemmTcPlan p_gu = plan_gemm_tc(M, ff, d, true, true, ctx->n_sms);
-  const GemmTcPlan p_g1 = plan_gemm_tc(M, ff, d, false, true, ctx->n_sms);   // gate and up as two launches
-  const bool wide = M > 64;
-  const GemmTcPlan p_down = plan_gemm_tc(M, d, ff, false, true, ctx->n_sms);
+  const GemmTcPlan p_g1 = plan_gemm_tc(M, ff, d, false, true, ctx->n_sms, (md.deterministic != 0) ? 8 : 32);   // gate and up as two launches
+  // "wide": split-K sums into fp32, rotation / attention per (sequence, head), element-wise gate.  Taken
+  // above 64 tokens, and by every call of a fixed-order context that the streaming chain kernel does
+  // not serve (the fused-epilogue projections below add their splits in arrival order)
+  const bool stream_chain = ctx->use_chain && md.deterministic && ctx->cs_packed && chain_stream_applicable(md, R, Tn);
+  const bool wide = M > 64 || (md.deterministic != 0 && !stream_chain);
+  // many tokens in a context that asked for fixed-order sums: the K splits of a projection tile are a
+  // thread-block cluster (at most 8 CTAs, the portable size) that adds its partial tiles in rank order
+  // through distributed shared memory; otherwise the splits add into L2 in arrival order (faster)
+  const bool fixed_order = wide && md.deterministic != 0;
+  const int cap = fixed_order ? 8 : 32;
+  const int cm_store = fixed_order ? 1 : 0, cm_add = fixed_order ? 2 : 0;
+  const GemmTcPlan p_down = plan_gemm_tc(M, d, ff, false, true, ctx->n_sms, cap);
   CUtensorMap tm_xn, tm_attn, tm_act, tm_q, tm_k, tm_v;
   const uint64_t kv_total_rows = (uint64_t)md.n_layers * a->kv_rows * md.n_heads * md.s_max;
   if (make_tmap_bf16_2d(&tm_q, q, (uint64_t)M, (uint64_t)d, Tn <= 16 ? 16u : 32u) != VVS_OK ||
@@ -364,7 +374,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   base.kv_rows = a->kv_rows; base.t_len = Tn; base.act = act; base.ff = ff;
 
   int rc = VVS_OK;
-  if (ctx->use_chain && md.deterministic && ctx->cs_packed && chain_stream_applicable(md, R, Tn)) {
+  if (stream_chain) {
     // at most 32 tokens: embedding and every decoder layer run as one persistent dataflow kernel
     CUtensorMap ck, cv;
     const uint32_t kb = (uint32_t)chain_stream_kb(md);
@@ -391,7 +401,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     if (a->tree_parent) return run_tree_decisions(ctx, hid, a, o, s);
     return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
   }
-  if (ctx->use_chain && fused_chain_applicable(md, R, Tn)) {
+  if (ctx->use_chain && !md.deterministic && fused_chain_applicable(md, R, Tn)) {
     // at most 32 tokens: the whole decoder chain runs as one persistent kernel
     FusedChainArgs fc{};
     fc.md = &md; fc.n_rows = R; fc.n_images = B; fc.t_len = Tn; fc.kv_rows = a->kv_rows; fc.n_sms = ctx->n_sms;
@@ -435,6 +445,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
       // sum into fp32 followed by one thread per element for rotation, rounding and cache append
       GemmTcArgs g = base;
       g.n = 3 * d; g.k = d; g.tm_a = &W.w_qkv; g.tm_b = &tm_xn; g.out = ws.qkv; g.ldo = 3 * d;
+      g.cluster_mode = cm_store;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_qkv, g, s));
       if (rows_attention) {
         // rotation, rounding, cache append and attention of each (sequence, head) in one kernel
@@ -458,6 +469,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     if (rc == VVS_OK) {
       GemmTcArgs g = base;
       g.n = d; g.k = d; g.tm_a = &W.w_o; g.tm_b = &tm_attn; g.out = ws.x; g.ldo = d;
+      g.cluster_mode = cm_add;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_o, g, s));
     }
     if (rows_norm)
@@ -467,6 +479,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     if (rc == VVS_OK && wide) {
       GemmTcArgs g = base;
       g.n = ff; g.k = d; g.tm_a = &W.w_gate; g.tm_b = &tm_xn; g.out = ws.gu; g.ldo = 2 * ff;
+      g.cluster_mode = cm_store;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_g1, g, s));
       g.tm_a = &W.w_up; g.out = ws.gu + ff;
       if (rc == VVS_OK) VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_g1, g, s));
@@ -479,6 +492,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     if (rc == VVS_OK) {
       GemmTcArgs g = base;
       g.n = d; g.k = ff; g.tm_a = &W.w_down; g.tm_b = &tm_act; g.out = ws.x; g.ldo = d;
+      g.cluster_mode = cm_add;
       VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_gemm_tc(GEMM_EPI_ADD, p_down, g, s));
     }
   }

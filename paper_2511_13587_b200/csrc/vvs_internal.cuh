@@ -224,6 +224,10 @@ struct GemmTcArgs {
   bool pdl;
   float* scratch; int ld_scratch; int* counters; int32_t* status;
   float* out; int ldo;         // STORE / ADD
+  int cluster_mode;            // ADD with many tokens: 0 = split-K sums added with reductions in arrival order;
+                               // 1 / 2 = the K splits of a tile form a thread-block cluster that adds its partial
+                               // tiles in rank order through distributed shared memory and then stores (1) or adds
+                               // to (2) `out`, each element by exactly one thread: no atomics, repeatable bits
   __nv_bfloat16* q; __nv_bfloat16* kv_k; __nv_bfloat16* kv_v;  // QKV
   const int32_t* slot_pos; const float* rope_cos; const float* rope_sin;
   int d, n_heads, hd, s_max, layer, kv_rows, t_len;
@@ -231,7 +235,7 @@ struct GemmTcArgs {
 };
 int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 int make_weight_tmap(CUtensorMap* out, const void* w, int rows, int cols);
-GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_sms);
+GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_sms, int split_cap = 32);
 int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStream_t s);
 void launch_rope_table(const int32_t* cache_len, const int32_t* tree_parent, int n_images, int n_forced,
                        const Workspace& ws, const vvs_model_desc& md, int n_rows,

@@ -187,14 +187,16 @@ def test_7b_shape_small_bf16(deterministic):
                           (B7_SMALL, 2, 2, 17, [377, 128])])           # head_dim 128, 19 rows, 76 tokens
 def test_per_projection_kernels_head_dims_and_long_blocks(ms, n_images, n_forced, k, fills):
     """More than 32 block tokens: the per-projection tensor-core kernels, with both head
-    dimensions and with more than 16 query rows per sequence."""
+    dimensions and with more than 16 query rows per sequence; arrival-order sums (fused projection
+    epilogues up to 64 tokens) and fixed-order sums (cluster reduction)."""
     case = H.build_case(ms, 61 + k, n_images, 2, n_forced, k, fills, q_noise=0.8)
-    run = H.GpuRunner(ms, case["w"], 2 * n_images, n_forced + k)
-    gpu = run.verify(case)
-    assert gpu["launches"] > 20
     ora = H.run_oracle(case)
-    _check_end_to_end(case, gpu, ora)
-    run.close()
+    for deterministic in (False, True):
+        run = H.GpuRunner(ms, case["w"], 2 * n_images, n_forced + k, deterministic=deterministic)
+        gpu = run.verify(case)
+        assert gpu["launches"] > 20
+        _check_end_to_end(case, gpu, ora)
+        run.close()
 
 
 @pytest.mark.parametrize("ms,n_forced,k,fills",
@@ -207,11 +209,12 @@ def test_row_batched_attention_edges(ms, n_forced, k, fills):
     n_images = len(fills)
     case = H.build_case_independent(ms, 83 + k, n_images, 2, n_forced, k, fills, logit_std=0.5)
     assert n_images * 2 * (n_forced + k) > 64
-    run = H.GpuRunner(ms, case["w"], 2 * n_images, n_forced + k)
-    gpu = run.verify(case)
     ora = H.run_oracle(case)
-    _check_end_to_end(case, gpu, ora)
-    run.close()
+    for deterministic in (False, True):
+        run = H.GpuRunner(ms, case["w"], 2 * n_images, n_forced + k, deterministic=deterministic)
+        gpu = run.verify(case)
+        _check_end_to_end(case, gpu, ora)
+        run.close()
 
 
 @pytest.mark.parametrize("deterministic", [True, False])
@@ -325,6 +328,18 @@ def test_repeatable_across_calls():
         for key in ("accept_len", "next_token", "new_len", "hidden"):
             np.testing.assert_array_equal(c_[key], d_[key], err_msg=key)
         np.testing.assert_array_equal(c_["accept_len"], a["accept_len"])
+        run.close()
+    # more than 32 block tokens in a fixed-order context: the K splits of every projection are a
+    # cluster that adds its partial tiles in rank order (36, 72 and 288 tokens: one, one and two passes)
+    for n_images, fills in ((2, [50, 400]), (4, [10, 200, 333, 574]), (16, list(range(5, 5 + 16 * 35, 35)))):
+        c2 = H.build_case_independent(ms, 171 + n_images, n_images, 2, 1, 8, fills, logit_std=0.7)
+        run = H.GpuRunner(ms, c2["w"], 2 * n_images, 9, deterministic=True)
+        a = run.verify(c2)
+        b = run.verify(c2)
+        assert a["launches"] > 20
+        for key in ("accept_len", "next_token", "accept_mask", "new_len", "target_probs", "hidden", "kv_k", "kv_v"):
+            np.testing.assert_array_equal(a[key], b[key], err_msg=key)
+        H.check_replay(c2, a)
         run.close()
     run = H.GpuRunner(ms, case["w"], 4, 9, deterministic=False)
     a = run.verify(case)
