@@ -108,25 +108,34 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const T* __restrict_
 
 // The same for many rows of a bf16 context: one warp per row, 16-byte loads, no shared memory; as a
 // programmatic dependent of the projection before it (the row is read after griddepcontrol.wait).
-__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* __restrict__ x,
+__global__ void __launch_bounds__(128) rmsnorm_rows_kernel(const float* __restrict__ x,
                                                            const __nv_bfloat16* __restrict__ scale,
                                                            __nv_bfloat16* __restrict__ out, int m, int d, float eps) {
+  constexpr int kKeep = 12;            // 16-byte pieces of the row a lane keeps in registers (d <= 1536)
   const int lane = threadIdx.x & 31, row_i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (row_i >= m) return;
   const float* row = x + (size_t)row_i * d;
+  float4 keep[kKeep];
+#pragma unroll
+  for (int u = 0; u < kKeep; ++u) {
+    const int i = lane * 4 + u * 128;
+    keep[u] = i < d ? *reinterpret_cast<const float4*>(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   float ss = 0.f;
-  for (int i = lane * 4; i < d; i += 128) {
-    const float4 v = __ldcg(reinterpret_cast<const float4*>(row + i));
+#pragma unroll
+  for (int u = 0; u < kKeep; ++u)
+    ss += keep[u].x * keep[u].x + keep[u].y * keep[u].y + keep[u].z * keep[u].z + keep[u].w * keep[u].w;
+  for (int i = lane * 4 + kKeep * 128; i < d; i += 128) {
+    const float4 v = *reinterpret_cast<const float4*>(row + i);
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   const float rs = rsqrtf(ss / (float)d + eps);
   __nv_bfloat16* o = out + (size_t)row_i * d;
-  for (int i = lane * 4; i < d; i += 128) {
-    const float4 v = __ldcg(reinterpret_cast<const float4*>(row + i));
+  auto emit = [&](int i, const float4& v) {
     const uint2 g = *reinterpret_cast<const uint2*>(scale + i);
     const __nv_bfloat162 g0 = *reinterpret_cast<const __nv_bfloat162*>(&g.x);
     const __nv_bfloat162 g1 = *reinterpret_cast<const __nv_bfloat162*>(&g.y);
@@ -136,7 +145,13 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* __restri
     pk.x = *reinterpret_cast<uint32_t*>(&r0);
     pk.y = *reinterpret_cast<uint32_t*>(&r1);
     *reinterpret_cast<uint2*>(o + i) = pk;
+  };
+#pragma unroll
+  for (int u = 0; u < kKeep; ++u) {
+    const int i = lane * 4 + u * 128;
+    if (i < d) emit(i, keep[u]);
   }
+  for (int i = lane * 4 + kKeep * 128; i < d; i += 128) emit(i, *reinterpret_cast<const float4*>(row + i));
 }
 
 template <typename T>
@@ -160,7 +175,7 @@ static cudaError_t launch_dependent(const void* fn, dim3 grid, dim3 block, void*
 void launch_rmsnorm_rows(const float* x, const __nv_bfloat16* scale, __nv_bfloat16* out, int m, int d, float eps,
                          bool pdl, cudaStream_t s) {
   void* args[] = {&x, &scale, &out, &m, &d, &eps};
-  launch_dependent(reinterpret_cast<const void*>(rmsnorm_rows_kernel), dim3((m + 7) / 8), dim3(256), args, pdl, s);
+  launch_dependent(reinterpret_cast<const void*>(rmsnorm_rows_kernel), dim3((m + 3) / 4), dim3(128), args, pdl, s);
 }
 
 // ---------------------------------------------------------------------------------------------
