@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(kThreads) attention_rows_kernel(AttentionRowsA
   using L = Layout<HD>;
   constexpr int NC = L::NC, NJ = HD / 8, HALF = HD / 2;
   extern __shared__ __align__(1024) uint8_t smem[];
-  const int h = blockIdx.x, r = blockIdx.y;
+  const int h = blockIdx.x, r = a.seq_order[blockIdx.y];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
   const int T = a.t_len, d = a.d;
   const int fill = a.cache_len[r];

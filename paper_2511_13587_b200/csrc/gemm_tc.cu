@@ -379,15 +379,29 @@ gemm_tc_kernel(const KernelParams p, const __grid_constant__ CUtensorMap tm_a,
 // still go to cache slot fill + t.
 __global__ void rope_table_kernel(const int32_t* __restrict__ cache_len, const float* __restrict__ inv_freq,
                                   const int32_t* __restrict__ tree_parent, int n_images, int n_forced,
-                                  int32_t* __restrict__ slot_pos, uint32_t* __restrict__ anc_mask,
+                                  int32_t* __restrict__ slot_pos, int32_t* __restrict__ seq_order,
+                                  uint32_t* __restrict__ anc_mask,
                                   float* __restrict__ rope_cos, float* __restrict__ rope_sin, int t_len, int hd,
                                   int s_max, int rope_mode, int grid_w, int n_prefix, int32_t* status,
                                   unsigned* clear_words, int n_clear) {
   __shared__ int s_depth;
   const int m = blockIdx.x, r = m / t_len, t = m % t_len;
   // the stage counters of the chain kernel that follows in the stream start from zero
-  if (blockIdx.x == 0)
+  if (blockIdx.x == 0) {
     for (int i = threadIdx.x; i < n_clear; i += blockDim.x) clear_words[i] = 0u;
+    // sequences by descending fill level (ties by index): the row-batched attention starts its longest
+    // (sequence, head) items first, so that the short ones fill the tail of the grid
+    const int n_rows = gridDim.x / t_len;
+    for (int i = threadIdx.x; i < n_rows; i += blockDim.x) {
+      const int fi = cache_len[i];
+      int rank = 0;
+      for (int j = 0; j < n_rows; ++j) {
+        const int fj = cache_len[j];
+        rank += (fj > fi || (fj == fi && j < i)) ? 1 : 0;
+      }
+      seq_order[rank] = i;
+    }
+  }
   const int fill = cache_len[r];
   const bool ok = fill >= 0 && fill + t_len <= s_max;
   if (!ok && threadIdx.x == 0) atomicOr(status, VVS_DEV_CACHE_OVERFLOW);
@@ -583,7 +597,7 @@ void launch_rope_table(const int32_t* cache_len, const int32_t* tree_parent, int
                        const Workspace& ws, const vvs_model_desc& md, int n_rows, int t_len, cudaStream_t s,
                        unsigned* clear_words, int n_clear) {
   rope_table_kernel<<<n_rows * t_len, 64, 0, s>>>(cache_len, ws.rope_inv_freq, tree_parent, n_images, n_forced,
-                                                  ws.slot_pos, ws.anc_mask, ws.rope_cos, ws.rope_sin, t_len,
+                                                  ws.slot_pos, ws.seq_order, ws.anc_mask, ws.rope_cos, ws.rope_sin, t_len,
                                                   md.head_dim, md.s_max, md.rope_mode, md.rope_grid_w, md.n_prefix,
                                                   ws.status, clear_words, n_clear);
 }

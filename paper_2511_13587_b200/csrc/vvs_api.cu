@@ -47,6 +47,7 @@ size_t layout(const vvs_model_desc& d, Workspace& ws, char* base) {
       const size_t wide = 3 * dm > 2 * ff ? 3 * dm : 2 * ff;
       const size_t tiles = (wide + 127) / 128, passes = (M + 255) / 256;
       c.take(ws.slot_pos, M * 4);
+      c.take(ws.seq_order, (size_t)d.max_rows * 4);
       c.take(ws.rope_cos, M * (size_t)(d.head_dim / 2) * 4);
       c.take(ws.rope_sin, M * (size_t)(d.head_dim / 2) * 4);
       c.take(ws.sk_scratch, M * wide * 4);
@@ -362,7 +363,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   const bool rows_attention = wide && attention_rows_applicable(md, Tn);
   AttentionRowsArgs ar{};
   ar.qkv = ws.qkv; ar.kv_k = kv_k; ar.kv_v = kv_v; ar.cache_len = a->cache_len; ar.rope_cos = ws.rope_cos;
-  ar.rope_sin = ws.rope_sin; ar.anc_mask = ws.anc_mask; ar.out = attn; ar.d = d; ar.n_heads = md.n_heads;
+  ar.rope_sin = ws.rope_sin; ar.anc_mask = ws.anc_mask; ar.seq_order = ws.seq_order; ar.out = attn; ar.d = d; ar.n_heads = md.n_heads;
   ar.hd = md.head_dim; ar.s_max = md.s_max; ar.kv_rows = a->kv_rows; ar.t_len = Tn; ar.n_rows = R; ar.pdl = ctx->use_pdl;
 
   GemmTcArgs base{};

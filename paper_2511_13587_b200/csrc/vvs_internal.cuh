@@ -67,6 +67,7 @@ struct Workspace {
   float* rope_inv_freq = nullptr;  // [head_dim/2] angle per unit coordinate of each pair
   // tensor-core path
   int32_t* slot_pos = nullptr;   // [M] cache slot of each block row, -1 if its sequence overflows
+  int32_t* seq_order = nullptr;  // [R] sequences by descending fill level (longest attention items first)
   uint32_t* anc_mask = nullptr;  // [M] bit j set: block row j of the same sequence is visible (ancestor or self)
   double* tree_res = nullptr;    // [2][max_rows, V] residuals of the tree walk (ping-pong)
   int32_t* tree_path = nullptr;  // [max_rows, 32] accepted nodes when the caller does not ask for them
@@ -264,6 +265,7 @@ struct AttentionRowsArgs {
   const float* rope_cos;       // [M, hd / 2] rotation table of the step
   const float* rope_sin;
   const uint32_t* anc_mask;    // [M] visible block rows per block row
+  const int32_t* seq_order;    // [R] the sequence CTA row y works on: longest caches first
   __nv_bfloat16* out;          // [M, d]
   int d, n_heads, hd, s_max, layer, kv_rows, t_len, n_rows;
   bool pdl;
