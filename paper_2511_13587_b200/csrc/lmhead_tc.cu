@@ -208,30 +208,38 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
         p.part_s[(size_t)tile * p.bt + row0 + tid] = sum;
       }
       // ---- 3. logits of the drafted tokens and of their neighbours that live in this tile --------
+      // One warp per (image, draft) pair of the pass; its lanes walk the draft's neighbour row (one
+      // coalesced load of the column indices per 32 neighbours) and pick the entries of this tile.
       if (p.n_draft_max > 0) {
         const int kk_max = p.relaxed ? p.nbr_k : 1;
-        const int per_img = p.n_draft_max * kk_max;
         const int b0 = row0 / p.rows_per_seq, b1 = (row0 + nd - 1) / p.rows_per_seq;
-        for (int e = b0 * per_img + tid; e < (b1 + 1) * per_img; e += 128) {
-          const int b = e / per_img, rem = e - b * per_img;
-          const int i = rem / kk_max, jj = rem - i * kk_max;
+        const int n_pairs = (b1 - b0 + 1) * p.n_draft_max;
+        if (kk_max <= 1) {                                  // strict: one thread per pair
+          for (int pr = tid; pr < n_pairs; pr += 128) {
+            const int b = b0 + pr / p.n_draft_max, i = pr % p.n_draft_max;
+            const int r = b * p.rows_per_seq + p.first_row + i - row0;
+            if (r < 0 || r >= nd) continue;
+            const int x = p.drafts[(size_t)b * p.drafts_ld + i] - p.vocab_offset;
+            if (x >= 0 && x < p.v && (x >> 7) == tile) p.l_tok[b * p.n_draft_max + i] = sL[r * kTileLd + (x & 127)];
+          }
+        } else
+        for (int pr = warp; pr < n_pairs; pr += 4) {
+          const int b = b0 + pr / p.n_draft_max, i = pr % p.n_draft_max;
           const int r = b * p.rows_per_seq + p.first_row + i - row0;   // decision row inside the pass
           if (r < 0 || r >= nd) continue;
           const int x = p.drafts[(size_t)b * p.drafts_ld + i] - p.vocab_offset;
           if (x < 0 || x >= p.v) continue;                            // reported by the acceptance kernel
-          if (jj == 0) {
-            if ((x >> 7) == tile) p.l_tok[b * p.n_draft_max + i] = sL[r * kTileLd + (x & 127)];
-          } else {
-            const int beg = p.row_ptr[x], len = p.row_ptr[x + 1] - beg;
-            if (jj < len) {
-              const int c = p.col[beg + jj];
-              const bool ok = c >= 0 && c < p.v;
-              if (!ok) {
-                atomicOr(p.status, VVS_DEV_BAD_NEIGHBOUR);
-                if (tile == 0) p.l_nbr[((size_t)b * p.n_draft_max + i) * p.kmax + jj] = -CUDART_INF_F;
-              } else if ((c >> 7) == tile) {
-                p.l_nbr[((size_t)b * p.n_draft_max + i) * p.kmax + jj] = sL[r * kTileLd + (c & 127)];
-              }
+          if (lane == 0 && (x >> 7) == tile) p.l_tok[b * p.n_draft_max + i] = sL[r * kTileLd + (x & 127)];
+          const int beg = p.row_ptr[x], len = p.row_ptr[x + 1] - beg;
+          const int kk = kk_max < len ? kk_max : len;
+          float* dst = p.l_nbr + ((size_t)b * p.n_draft_max + i) * p.kmax;
+          for (int jj = 1 + lane; jj < kk; jj += 32) {
+            const int c = p.col[beg + jj];
+            if (c < 0 || c >= p.v) {
+              atomicOr(p.status, VVS_DEV_BAD_NEIGHBOUR);
+              if (tile == 0) dst[jj] = -CUDART_INF_F;
+            } else if ((c >> 7) == tile) {
+              dst[jj] = sL[r * kTileLd + (c & 127)];
             }
           }
         }
