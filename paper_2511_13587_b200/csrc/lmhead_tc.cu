@@ -58,6 +58,11 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
   return false;
 }
 
+// NM = codebook tiles of 128 rows per CTA.  With NM = 2 the feature tile of a k-block is read from L2
+// once for 256 codes (two MMAs on one B operand, two accumulators side by side in TMEM): half the
+// feature traffic per flop, which is what bounds the kernel at large batch; used when the codebook
+// still gives every SM a CTA.  The logit tile then reuses the (idle) pipeline stages.
+template <int NM>
 __global__ void __launch_bounds__(128, 1)
 lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b) {
   extern __shared__ uint8_t smem_raw[];
@@ -69,12 +74,14 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
-  const int tile = blockIdx.x;
+  const int tile0 = blockIdx.x * NM;
   const int C = p.n_cfg;
   const uint32_t half_bytes = (uint32_t)p.nd_pad * kBlockK * 2u;     // one box of feature rows
   const uint32_t b_bytes = half_bytes * (uint32_t)C;
-  const uint32_t stage_bytes = kATileBytes + b_bytes;
-  float* sL = reinterpret_cast<float*>(smem + (size_t)p.stages * stage_bytes);   // [nd_pad][kTileLd]
+  constexpr uint32_t a_bytes = kATileBytes * NM;
+  const uint32_t stage_bytes = a_bytes + b_bytes;
+  // [nd_pad][kTileLd]; with two tiles per CTA it lies over the stages, which are idle during an epilogue
+  float* sL = reinterpret_cast<float*>(NM == 2 ? smem : smem + (size_t)p.stages * stage_bytes);
   const int nt = p.nd_pad * C;
 
   if (tid == 0) {
@@ -112,11 +119,14 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
         const int n_pre = p.kb_total < p.stages ? p.kb_total : p.stages;
         for (int i = 0; i < n_pre; ++i) {
           mbar_expect_tx(&full_bar[i], stage_bytes);
-          tma_load_2d(smem + (size_t)i * stage_bytes, &tm_a, &full_bar[i], i * (int)kBlockK, tile * (int)kTileRows);
+#pragma unroll
+          for (int m = 0; m < NM; ++m)
+            tma_load_2d(smem + (size_t)i * stage_bytes + m * kATileBytes, &tm_a, &full_bar[i], i * (int)kBlockK,
+                        (tile0 + m) * (int)kTileRows);
         }
         pdl_wait();
         for (int i = 0; i < n_pre; ++i) {
-          uint8_t* b = smem + (size_t)i * stage_bytes + kATileBytes;
+          uint8_t* b = smem + (size_t)i * stage_bytes + a_bytes;
           tma_load_2d(b, &tm_b, &full_bar[i], i * (int)kBlockK, row0);
           if (C == 2) tma_load_2d(b + half_bytes, &tm_b, &full_bar[i], i * (int)kBlockK, p.bt + row0);
         }
@@ -132,9 +142,11 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
         }
         uint8_t* st = smem + (size_t)stage * stage_bytes;
         mbar_expect_tx(&full_bar[stage], stage_bytes);
-        tma_load_2d(st, &tm_a, &full_bar[stage], kb * (int)kBlockK, tile * (int)kTileRows);
-        tma_load_2d(st + kATileBytes, &tm_b, &full_bar[stage], kb * (int)kBlockK, row0);
-        if (C == 2) tma_load_2d(st + kATileBytes + half_bytes, &tm_b, &full_bar[stage], kb * (int)kBlockK, p.bt + row0);
+#pragma unroll
+        for (int m = 0; m < NM; ++m)
+          tma_load_2d(st + m * kATileBytes, &tm_a, &full_bar[stage], kb * (int)kBlockK, (tile0 + m) * (int)kTileRows);
+        tma_load_2d(st + a_bytes, &tm_b, &full_bar[stage], kb * (int)kBlockK, row0);
+        if (C == 2) tma_load_2d(st + a_bytes + half_bytes, &tm_b, &full_bar[stage], kb * (int)kBlockK, p.bt + row0);
       }
     } else if (warp == 1 && lane == 0) {
       // ---- MMA issuer --------------------------------------------------------------------------
@@ -149,11 +161,15 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
         }
         tc_fence_after();
         const uint32_t a_addr = smem_u32(smem + (size_t)stage * stage_bytes);
-        const uint32_t b_addr = a_addr + kATileBytes;
+        const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
-        for (uint32_t k16 = 0; k16 < kBlockK / 16; ++k16)
-          mma_bf16(tmem_base, smem_desc_sw128(a_addr + k16 * 32), smem_desc_sw128(b_addr + k16 * 32), idesc,
-                   (kb > 0 || k16 > 0) ? 1u : 0u);
+        for (uint32_t k16 = 0; k16 < kBlockK / 16; ++k16) {
+          const uint64_t bd = smem_desc_sw128(b_addr + k16 * 32);
+#pragma unroll
+          for (uint32_t m = 0; m < (uint32_t)NM; ++m)
+            mma_bf16(tmem_base + m * (uint32_t)nt, smem_desc_sw128(a_addr + m * kATileBytes + k16 * 32), bd, idesc,
+                     (kb > 0 || k16 > 0) ? 1u : 0u);
+        }
         mma_commit(&empty_bar[stage]);
       }
       if (ok) mma_commit(&acc_bar);
@@ -169,10 +185,13 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
     }
     tc_fence_after();
 
+    for (int mt = 0; mt < NM; ++mt) {
+    const int tile = tile0 + mt;
+    if (tile * (int)kTileRows >= p.v) break;                        // the codebook ends before this tile
     // ---- 1. guided logits of this thread's codebook row, for every decision row of the pass ------
     const int n = tile * (int)kTileRows + tid;
     const bool n_ok = n < p.v;
-    const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t t_row = tmem_base + (uint32_t)(mt * nt) + ((uint32_t)(warp * 32) << 16);
     for (int c0 = 0; c0 < p.nd_pad && c0 < nd; c0 += 16) {
       float lc[16], lu[16];
       tmem_ld16(t_row + c0, lc);
@@ -245,6 +264,8 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
         }
       }
     }
+    if (NM == 2) __syncthreads();                                 // the logit tile is reused by the next codebook tile
+    }
     tc_fence_before();
     __syncthreads();
   }
@@ -270,21 +291,29 @@ int launch_lmhead_tc(const LmHeadArgs& a, cudaStream_t s) {
   p.l_tok = a.l_tok; p.l_nbr = a.l_nbr;
   p.row_mode = a.row_mode; p.sel_row = a.sel_row; p.stat_m = a.stat_m; p.stat_inv = a.stat_inv; p.p_row = a.p_row;
   const int nt = p.nd_pad * a.n_cfg;
-  const uint32_t stage_bytes = kATileBytes + (uint32_t)nt * kBlockK * 2u;
+  // two codebook tiles per CTA when 256-row tiles still give every SM a CTA (the feature tile is then
+  // read once per 256 codes); the logit tile lies over the stages in that case
+  const int n_sms_hint = 120;
+  const bool two = a.v >= 2 * (int)kTileRows * n_sms_hint && 2 * nt <= 512;
+  const uint32_t stage_bytes = kATileBytes * (two ? 2u : 1u) + (uint32_t)nt * kBlockK * 2u;
   const size_t tile_bytes = a.row_mode ? 0 : (size_t)p.nd_pad * kTileLd * 4;
-  int stages = (int)((220 * 1024 - tile_bytes) / stage_bytes);
+  int stages = (int)((220 * 1024 - (two ? 0 : tile_bytes)) / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages > p.kb_total) stages = p.kb_total;
   if (stages < 1) return VVS_ERR_SHAPE;
   p.stages = stages;
   uint32_t cols = 32;
-  while (cols < (uint32_t)nt) cols <<= 1;
+  while (cols < (uint32_t)nt * (two ? 2u : 1u)) cols <<= 1;
   p.tmem_cols = cols;
-  const size_t smem = (size_t)stages * stage_bytes + tile_bytes + 1024;
+  size_t smem = (size_t)stages * stage_bytes + (two ? 0 : tile_bytes);
+  if (two && smem < tile_bytes) smem = tile_bytes;
+  smem += 1024;
   if (smem > 226 * 1024) return VVS_ERR_SHAPE;
-  if (ensure_dynamic_smem(reinterpret_cast<const void*>(lmhead_tc_kernel), 226 * 1024) != cudaSuccess) return VVS_ERR_CUDA;
+  const void* fn = two ? reinterpret_cast<const void*>(lmhead_tc_kernel<2>) : reinterpret_cast<const void*>(lmhead_tc_kernel<1>);
+  if (ensure_dynamic_smem(fn, 226 * 1024) != cudaSuccess) return VVS_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((a.v + (int)kTileRows - 1) / (int)kTileRows, 1, 1);
+  const int rows_per_cta = (int)kTileRows * (two ? 2 : 1);
+  cfg.gridDim = dim3((a.v + rows_per_cta - 1) / rows_per_cta, 1, 1);
   cfg.blockDim = dim3(128, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
@@ -293,7 +322,9 @@ int launch_lmhead_tc(const LmHeadArgs& a, cudaStream_t s) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = a.pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, lmhead_tc_kernel, p, *a.tm_a, *a.tm_b) == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
+  const cudaError_t e = two ? cudaLaunchKernelEx(&cfg, lmhead_tc_kernel<2>, p, *a.tm_a, *a.tm_b)
+                            : cudaLaunchKernelEx(&cfg, lmhead_tc_kernel<1>, p, *a.tm_a, *a.tm_b);
+  return e == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
 }
 
 int lmhead_box_rows(int bt) {
