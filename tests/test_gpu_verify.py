@@ -218,6 +218,24 @@ def test_row_batched_attention_edges(ms, n_forced, k, fills):
 
 
 @pytest.mark.parametrize("deterministic", [True, False])
+def test_small_call_on_a_shape_the_streaming_kernel_does_not_take(deterministic):
+    """d_ff = 880 is not a multiple of 32, so a fixed-order context cannot use the streaming whole-chain
+    kernel: its 18-token call goes through the per-projection kernels with cluster reductions (and must
+    still repeat bit for bit); the arrival-order context keeps the split-K whole-chain kernel."""
+    ms = replace(XL_SMALL, name="llamagen_xl_small_ff880", d_ff=880)
+    case = H.build_case(ms, 97, 1, 2, 1, 8, [211])
+    run = H.GpuRunner(ms, case["w"], 2, 9, deterministic=deterministic)
+    gpu = run.verify(case)
+    _check_end_to_end(case, gpu, H.run_oracle(case))
+    if deterministic:
+        assert gpu["launches"] > 20
+        again = run.verify(case)
+        for key in ("accept_len", "next_token", "target_probs", "hidden", "kv_k", "kv_v"):
+            np.testing.assert_array_equal(gpu[key], again[key], err_msg=key)
+    run.close()
+
+
+@pytest.mark.parametrize("deterministic", [True, False])
 def test_ragged_drafts_forced_prefix_and_cache_edges(deterministic):
     """n_draft below K (including 0), two forced rows, an empty cache and a cache that the block
     fills to capacity."""
