@@ -33,12 +33,12 @@ using bf16 = __nv_bfloat16;
 // per SM) and 8 warps or 2 slots are within 2 % of one another; 32-key blocks are 5 % slower.
 constexpr int kWarps = 4;
 constexpr int kThreads = 32 * kWarps;
-constexpr int kKB = 64;        // cached keys per staged block
 constexpr int kStages = 3;
 constexpr int kMaxT = 32;      // block rows per sequence
 
 template <int HD>
 struct Layout {
+  static constexpr int kKB = HD == 64 ? 64 : 32;       // cached keys per staged block (16 KB of K + V either way)
   static constexpr int NC = HD / 64;                   // 128-byte column groups per K / V row
   static constexpr int kTile = kKB * 128;              // one column group of a staged block
   static constexpr int kStage = 2 * NC * kTile;        // K then V
@@ -48,7 +48,7 @@ struct Layout {
   static constexpr int kRegs = (HD / 8) * 4 + 4;
   static constexpr int kOffScratch = 0;                // the merge buffers reuse the ring once it has drained
   static constexpr int kBytes = kOffQ + kMaxT * HD * 2;
-  static_assert((kWarps / 2) * kRegs * 32 * 4 <= kStages * kStage, "merge buffers must fit in the ring");
+  static_assert((kWarps / 2 + 2) * kRegs * 32 * 4 <= kStages * kStage, "merge buffers must fit in the ring");
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -57,11 +57,21 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+  return v;
+}
 
 template <int HD>
 __global__ void __launch_bounds__(kThreads) attention_rows_kernel(AttentionRowsArgs a) {
   using L = Layout<HD>;
-  constexpr int NC = L::NC, NJ = HD / 8, HALF = HD / 2;
+  constexpr int NC = L::NC, NJ = HD / 8, HALF = HD / 2, kKB = L::kKB;
   extern __shared__ __align__(1024) uint8_t smem[];
   const int h = blockIdx.x, r = a.seq_order[blockIdx.y];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
@@ -69,14 +79,21 @@ __global__ void __launch_bounds__(kThreads) attention_rows_kernel(AttentionRowsA
   const int fill = a.cache_len[r];
   const bool ok = fill >= 0 && fill + T <= a.s_max;
   const size_t row_base = ((size_t)(a.layer * a.kv_rows + r) * a.n_heads + h) * a.s_max;
-  const int nb = ok ? (fill + kKB - 1) / kKB : 0;
+  // Few (sequence, head) items: the key blocks of an item are dealt to the S CTAs of a cluster (rank =
+  // blockIdx.z takes blocks rank, rank + S, ...; the last rank also the block's own keys); rank 0 merges
+  // the partial results in rank order through distributed shared memory and writes the output.
+  const int S = (int)gridDim.z, rank = (int)blockIdx.z;
+  const int nb_all = ok ? (fill + kKB - 1) / kKB : 0;
+  const int nb = nb_all > rank ? (nb_all - rank + S - 1) / S : 0;      // this CTA's blocks
+  const bool own_keys = rank == S - 1;
   const uint32_t s_base = tc::smem_u32(smem);
 
   // 16-byte chunks of block `blk` (keys blk*64 .. ), K and V, into its ring slot; rows at or beyond
   // `fill` are not requested (the slices mask them)
-  auto request = [&](int blk) {
-    if (blk < nb) {
-      const uint32_t stage = s_base + (uint32_t)(blk % kStages) * L::kStage;
+  auto request = [&](int j) {
+    if (j < nb) {
+      const int blk = rank + j * S;
+      const uint32_t stage = s_base + (uint32_t)(j % kStages) * L::kStage;
       const int rows = min(kKB, fill - blk * kKB);
       const int per_row = HD / 8, n = rows * per_row;
       const bf16* k_src = a.kv_k + (row_base + (size_t)blk * kKB) * HD;
@@ -128,10 +145,12 @@ __global__ void __launch_bounds__(kThreads) attention_rows_kernel(AttentionRowsA
     if (idx < T * HALF) {
       const int t = idx / HALF, i = idx - t * HALF;
       float* src = a.qkv + (size_t)(r * T + t) * 3 * d + h * HD + 2 * i;
-      const float2 z = make_float2(0.f, 0.f);                // split-K sums are added into this buffer:
-      *reinterpret_cast<float2*>(src) = z;                   // leave it zero for the next layer
-      *reinterpret_cast<float2*>(src + d) = z;
-      *reinterpret_cast<float2*>(src + 2 * d) = z;
+      if (S == 1) {                                          // (a cluster clears after every rank has read)
+        const float2 z = make_float2(0.f, 0.f);              // split-K sums are added into this buffer:
+        *reinterpret_cast<float2*>(src) = z;                 // leave it zero for the next layer
+        *reinterpret_cast<float2*>(src + d) = z;
+        *reinterpret_cast<float2*>(src + 2 * d) = z;
+      }
       const uint32_t qp = pack2(q2[u].x * cs[u] - q2[u].y * sn[u], q2[u].x * sn[u] + q2[u].y * cs[u]);
       const uint32_t kp = pack2(k2[u].x * cs[u] - k2[u].y * sn[u], k2[u].x * sn[u] + k2[u].y * cs[u]);
       const uint32_t vp = pack2(v2[u].x, v2[u].y);
@@ -140,7 +159,7 @@ __global__ void __launch_bounds__(kThreads) attention_rows_kernel(AttentionRowsA
       const uint32_t off = (uint32_t)cg * L::kNewTile + t * 128 + (((ch ^ (t & 7))) << 4) + (col & 7) * 2;
       *reinterpret_cast<uint32_t*>(s_new + off) = kp;
       *reinterpret_cast<uint32_t*>(s_new + NC * L::kNewTile + off) = vp;
-      if (ok) {
+      if (ok && own_keys) {
         const size_t slot = (row_base + fill + t) * HD + col;
         *reinterpret_cast<uint32_t*>(a.kv_k + slot) = kp;
         *reinterpret_cast<uint32_t*>(a.kv_v + slot) = vp;
@@ -179,15 +198,16 @@ __global__ void __launch_bounds__(kThreads) attention_rows_kernel(AttentionRowsA
 
   // ---- cached keys ---------------------------------------------------------------------------------
 #pragma unroll 1
-  for (int blk = 0; blk < nb; ++blk) {
-    request(blk + kStages - 1);
+  for (int j = 0; j < nb; ++j) {
+    const int blk = rank + j * S;
+    request(j + kStages - 1);
     cp_async_wait<kStages - 1>();
     __syncthreads();
-    const uint32_t k_base = s_base + (uint32_t)(blk % kStages) * L::kStage;
+    const uint32_t k_base = s_base + (uint32_t)(j % kStages) * L::kStage;
     const uint32_t v_base = k_base + NC * L::kTile;
 #pragma unroll 1
     for (int sl = 0; sl < kKB / 16; ++sl) {
-      if (((blk * (kKB / 16) + sl) & (wpm - 1)) != kg) continue;
+      if (((j * (kKB / 16) + sl) & (wpm - 1)) != kg) continue;
       const int left = fill - (blk * kKB + sl * 16);
       if (left <= 0) break;
       uint32_t vis[2];
@@ -199,7 +219,7 @@ __global__ void __launch_bounds__(kThreads) attention_rows_kernel(AttentionRowsA
   }
   cp_async_wait<0>();
   // ---- the block's own keys: ancestors and the row itself, by the last warp of each m-tile ----------
-  if (ok && kg == wpm - 1) {
+  if (ok && own_keys && kg == wpm - 1) {
     const uint32_t k_base = tc::smem_u32(s_new), v_base = k_base + NC * L::kNewTile;
     for (int sl = 0; sl <= mt && sl * 16 < T; ++sl) {
       uint32_t vis[2];
@@ -250,7 +270,56 @@ __global__ void __launch_bounds__(kThreads) attention_rows_kernel(AttentionRowsA
     }
     __syncthreads();
   }
-  if (kg == 0) {
+  if (S > 1) {
+    // ---- merge the ranks of the cluster: every rank publishes its m-tiles' state, rank 0 folds them in
+    float* xslot = scratch + (size_t)(kWarps / 2 + mt) * kRegs * 32;
+    if (kg == 0 && rank != 0) {
+#pragma unroll
+      for (int j = 0; j < NJ; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) xslot[(j * 4 + e) * 32 + lane] = st.o[j][e];
+      xslot[(NJ * 4 + 0) * 32 + lane] = st.m[0];
+      xslot[(NJ * 4 + 1) * 32 + lane] = st.m[1];
+      xslot[(NJ * 4 + 2) * 32 + lane] = st.l[0];
+      xslot[(NJ * 4 + 3) * 32 + lane] = st.l[1];
+    }
+    cluster_sync_all();
+    if (rank == 0) {
+      // every rank has read its q / k / v sums long ago: clear them for the next layer
+      for (int idx = tid; idx < T * HALF; idx += kThreads) {
+        const int t = idx / HALF, i = idx - t * HALF;
+        float* src = a.qkv + (size_t)(r * T + t) * 3 * d + h * HD + 2 * i;
+        const float2 z = make_float2(0.f, 0.f);
+        *reinterpret_cast<float2*>(src) = z;
+        *reinterpret_cast<float2*>(src + d) = z;
+        *reinterpret_cast<float2*>(src + 2 * d) = z;
+      }
+      if (kg == 0) {
+        const uint32_t xaddr = tc::smem_u32(xslot);
+#pragma unroll 1
+        for (int q = 1; q < S; ++q) {
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const float mo = ld_cluster_f32(xaddr + (uint32_t)((NJ * 4 + i) * 32 + lane) * 4u, (uint32_t)q);
+            const float lo = ld_cluster_f32(xaddr + (uint32_t)((NJ * 4 + 2 + i) * 32 + lane) * 4u, (uint32_t)q);
+            const float m_new = fmaxf(st.m[i], mo);
+            const float m_safe = m_new == -CUDART_INF_F ? 0.f : m_new;
+            const float aa = ex2(st.m[i] - m_safe), bb = ex2(mo - m_safe);
+            st.m[i] = m_new;
+            st.l[i] = st.l[i] * aa + lo * bb;
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) {
+              const float o0 = ld_cluster_f32(xaddr + (uint32_t)((j * 4 + 2 * i) * 32 + lane) * 4u, (uint32_t)q);
+              const float o1 = ld_cluster_f32(xaddr + (uint32_t)((j * 4 + 2 * i + 1) * 32 + lane) * 4u, (uint32_t)q);
+              st.o[j][2 * i] = st.o[j][2 * i] * aa + o0 * bb;
+              st.o[j][2 * i + 1] = st.o[j][2 * i + 1] * aa + o1 * bb;
+            }
+          }
+        }
+      }
+    }
+  }
+  if (kg == 0 && rank == 0) {
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
       const int t = mt * 16 + g + 8 * i;
@@ -263,6 +332,7 @@ __global__ void __launch_bounds__(kThreads) attention_rows_kernel(AttentionRowsA
       }
     }
   }
+  if (S > 1) cluster_sync_all();      // no rank leaves while rank 0 may still read its state
 }
 
 template <int HD>
@@ -271,15 +341,34 @@ int launch_hd(const AttentionRowsArgs& a, cudaStream_t s) {
   if (ensure_dynamic_smem(reinterpret_cast<const void*>(attention_rows_kernel<HD>), L::kBytes) != cudaSuccess)
     return VVS_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(a.n_heads, a.n_rows, 1);
+  // few (sequence, head) items: split each item's keys over a cluster of 2, 4 or 8 CTAs, as long as
+  // the grid still fits the GPU at three CTAs per SM and a rank keeps a dozen key blocks of a full cache
+  // (measured: the 7B shape, 64 items of up to 75 blocks, is fastest split four ways, 3.65 against 4.06 ms
+  // per step; the XL shape, 40 items of up to 10 blocks, is fastest unsplit)
+  const int blocks_max = (a.s_max + L::kKB - 1) / L::kKB;
+  int split = 1;
+  while (split < 8 && (long long)a.n_heads * a.n_rows * split * 2 <= 3LL * a.n_sms && blocks_max >= 12 * split)
+    split *= 2;
+  cfg.gridDim = dim3(a.n_heads, a.n_rows, split);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = L::kBytes;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  if (a.pdl) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (split > 1) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 1;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = (unsigned)split;
+    ++na;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = a.pdl ? 1 : 0;
+  cfg.numAttrs = na;
   return cudaLaunchKernelEx(&cfg, attention_rows_kernel<HD>, a) == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;
 }
 

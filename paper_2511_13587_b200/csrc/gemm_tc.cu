@@ -535,7 +535,20 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
   long long best_cost = -1;
   const int cap = split_cap < 32 ? split_cap : 32;
   const int max_splits = allow_split ? (pl.kb_total < cap ? pl.kb_total : cap) : 1;
-  const long long slots = (long long)n_sms * (pl.passes > 1 ? 2 : 1);   // several passes: two CTAs per SM
+  // CTAs per SM the plan counts on.  Several token passes: two (one's epilogue overlaps the other's loads).
+  // One pass of a single weight matrix: up to five small CTAs of at least two stages each -- more
+  // independent weight streams per SM (measured at 18 tokens: 1.27 -> 1.09 ms per step at the XL shape,
+  // 4.87 -> 4.06 ms at the 7B shape; three to eight per SM are within 3 % of one another).
+  const uint32_t stage_b = kATileBytes * (dual ? 2u : 1u) + (uint32_t)pl.nt * kBlockK * 2u;
+  int cps = 1;
+  if (pl.passes > 1) {
+    cps = 2;
+  } else if (allow_split && !dual) {
+    cps = (int)(218u * 1024u / (2u * stage_b));
+    cps = cps > 5 ? 5 : cps < 1 ? 1 : cps;
+    if (split_cap <= 8 && cps > 2) cps = 2;   // cluster reduction: fewer, longer CTAs (1.52 / 4.42 ms against 1.68 / 4.8 at five)
+  }
+  const long long slots = (long long)n_sms * cps;
   for (int s = 1; s <= max_splits; ++s) {
     const long long per_cta = (pl.kb_total + s - 1) / s;
     const long long waves = ((long long)pl.tiles * s * pl.passes + slots - 1) / slots;
@@ -550,7 +563,7 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
   pl.splits = best;
   const uint32_t stage_bytes = kATileBytes * (dual ? 2u : 1u) + (uint32_t)pl.nt * kBlockK * 2u;
   const int per_cta = (pl.kb_total + pl.splits - 1) / pl.splits;
-  int stages = ((pl.passes > 1 ? 110 : 200) * 1024) / (int)stage_bytes;   // two CTAs per SM when passes are CTAs
+  int stages = ((cps == 1 ? 200 : cps == 2 ? 110 : 218 / cps) * 1024) / (int)stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages > per_cta) stages = per_cta;
   if (stages < 1) stages = 1;
@@ -570,6 +583,7 @@ int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStr
   kp.m = g.m; kp.n = g.n; kp.k = g.k;
   kp.nt = plan.nt; kp.passes = plan.passes; kp.kb_total = plan.kb_total; kp.splits = plan.splits;
   kp.stages = plan.stages; kp.tmem_cols = (uint32_t)plan.tmem_cols;
+  // (at 32 tokens and fewer the staged vector reductions were measured no faster than scalar ones)
   kp.wide_add = (epi == GEMM_EPI_ADD && (plan.nt > 32 || g.cluster_mode) && g.ldo % 4 == 0 &&
                  (reinterpret_cast<uintptr_t>(g.out) & 15) == 0) ? 1 : 0;
   kp.cluster_mode = (kp.wide_add && plan.splits <= 8) ? g.cluster_mode : 0;

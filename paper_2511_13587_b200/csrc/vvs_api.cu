@@ -334,8 +334,16 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   // "wide": split-K sums into fp32, rotation / attention per (sequence, head), element-wise gate.  Taken
   // above 64 tokens, and by every call of a fixed-order context that the streaming chain kernel does
   // not serve (the fused-epilogue projections below add their splits in arrival order)
-  const bool stream_chain = ctx->use_chain && md.deterministic && ctx->cs_packed && chain_stream_applicable(md, R, Tn);
-  const bool wide = M > 64 || (md.deterministic != 0 && !stream_chain);
+  const bool stream_chain = ctx->use_chain_kernels && md.deterministic && ctx->cs_packed && chain_stream_applicable(md, R, Tn);
+  // VVS_DEBUG_CHAIN_KERNELS (read at vvs_create) selects the previous generation, kept for comparison
+  // and still parity-tested: for calls of at most 32 tokens a persistent whole-chain kernel -- the
+  // streaming one (fixed-order contexts) or the split-K tcgen05 one with grid barriers (arrival-order
+  // contexts) -- and for 33-64 tokens in arrival-order contexts the fused-epilogue projections with
+  // the split-KV attention kernel.  Measured slower than the per-projection kernels below at both
+  // benchmark shapes (XL: 1.31 / 1.77 ms against 1.09 / 1.52; 7B: 5.33 / 6.24 against 3.65 / 4.42).
+  const bool legacy = ctx->use_chain_kernels && !md.deterministic;
+  const bool fused_chain = legacy && fused_chain_applicable(md, R, Tn);
+  const bool wide = !stream_chain && !fused_chain && (M > 64 || !legacy);
   // many tokens in a context that asked for fixed-order sums: the K splits of a projection tile are a
   // thread-block cluster (at most 8 CTAs, the portable size) that adds its partial tiles in rank order
   // through distributed shared memory; otherwise the splits add into L2 in arrival order (faster)
@@ -364,7 +372,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
   AttentionRowsArgs ar{};
   ar.qkv = ws.qkv; ar.kv_k = kv_k; ar.kv_v = kv_v; ar.cache_len = a->cache_len; ar.rope_cos = ws.rope_cos;
   ar.rope_sin = ws.rope_sin; ar.anc_mask = ws.anc_mask; ar.seq_order = ws.seq_order; ar.out = attn; ar.d = d; ar.n_heads = md.n_heads;
-  ar.hd = md.head_dim; ar.s_max = md.s_max; ar.kv_rows = a->kv_rows; ar.t_len = Tn; ar.n_rows = R; ar.pdl = ctx->use_pdl;
+  ar.hd = md.head_dim; ar.s_max = md.s_max; ar.kv_rows = a->kv_rows; ar.t_len = Tn; ar.n_rows = R; ar.n_sms = ctx->n_sms; ar.pdl = ctx->use_pdl;
 
   GemmTcArgs base{};
   base.m = M; base.pdl = ctx->use_pdl; base.status = ws.status;
@@ -402,7 +410,7 @@ int run_verify_tc(vvs_ctx* ctx, const vvs_verify_args* a, const vvs_verify_out* 
     if (a->tree_parent) return run_tree_decisions(ctx, hid, a, o, s);
     return run_decisions<T>(ctx, hid, Tn, a->n_forced - 1, a->block + a->n_forced, Tn, a, o, true, s);
   }
-  if (ctx->use_chain && !md.deterministic && fused_chain_applicable(md, R, Tn)) {
+  if (fused_chain) {
     // at most 32 tokens: the whole decoder chain runs as one persistent kernel
     FusedChainArgs fc{};
     fc.md = &md; fc.n_rows = R; fc.n_images = B; fc.t_len = Tn; fc.kv_rows = a->kv_rows; fc.n_sms = ctx->n_sms;
@@ -656,7 +664,7 @@ int vvs_create(const vvs_model_desc* desc, vvs_ctx** out) {
   ctx->tensor_core_path = desc->dtype == VVS_DTYPE_BF16 && !std::getenv("VVS_DEBUG_GENERIC");
   ctx->use_pdl = !std::getenv("VVS_DEBUG_NO_PDL");
   ctx->use_graph = !std::getenv("VVS_DEBUG_NO_GRAPH");
-  ctx->use_chain = !std::getenv("VVS_DEBUG_NO_CHAIN");
+  ctx->use_chain_kernels = std::getenv("VVS_DEBUG_CHAIN_KERNELS") != nullptr;
   if (cudaStreamCreateWithFlags(&ctx->capture_stream, cudaStreamNonBlocking) != cudaSuccess) {
     cudaGetLastError();
     ctx->capture_stream = nullptr;
@@ -667,7 +675,7 @@ int vvs_create(const vvs_model_desc* desc, vvs_ctx** out) {
     ctx->n_sms = 148;
   if (ctx->tensor_core_path && desc->n_layers > 0 && chain_stream_configure() != VVS_OK) {
     cudaGetLastError();
-    ctx->use_chain = false;
+    ctx->use_chain_kernels = false;
   }
   *out = ctx;
   return VVS_OK;
@@ -746,7 +754,7 @@ int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w) {
       // private copy of the layer weights in the streaming order of the chain kernel
       if (ctx->cs_packed) { cudaFree(ctx->cs_packed); ctx->cs_packed = nullptr; }
       if (ctx->cs_d_plan) { cudaFree(ctx->cs_d_plan); ctx->cs_d_plan = nullptr; }
-      if (ctx->use_chain && md.deterministic && chain_stream_applicable(md, 1, 1) &&
+      if (ctx->use_chain_kernels && md.deterministic && chain_stream_applicable(md, 1, 1) &&
           chain_stream_plan(md, ctx->n_sms, ctx->cs_plan)) {
         const size_t pbytes = chain_stream_packed_bytes(md, ctx->cs_plan);
         const size_t plbytes = ctx->cs_plan.cta.size() * sizeof(ChainCtaPlan);

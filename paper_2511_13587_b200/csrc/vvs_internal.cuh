@@ -149,7 +149,7 @@ struct vvs_ctx {
   vvs::Layer* layers = nullptr;  // host array [n_layers]
   bool tensor_core_path = false;     // bf16 contexts unless VVS_DEBUG_GENERIC is set
   bool use_pdl = true;               // programmatic dependent launch of the tensor-core GEMMs
-  bool use_chain = true;             // whole-chain persistent kernel for calls of at most 32 tokens
+  bool use_chain_kernels = false;  // debug: the persistent whole-chain kernels for calls of at most 32 tokens
   vvs::LayerMaps* layer_maps = nullptr;  // host array [n_layers]
   std::vector<const __nv_bfloat16*> chain_norms;  // host [n_layers][2] norm-scale pointers
   vvs::ChainStreamPlan cs_plan;        // streaming chain kernel: split of the weights over the CTAs
@@ -267,7 +267,7 @@ struct AttentionRowsArgs {
   const uint32_t* anc_mask;    // [M] visible block rows per block row
   const int32_t* seq_order;    // [R] the sequence CTA row y works on: longest caches first
   __nv_bfloat16* out;          // [M, d]
-  int d, n_heads, hd, s_max, layer, kv_rows, t_len, n_rows;
+  int d, n_heads, hd, s_max, layer, kv_rows, t_len, n_rows, n_sms;
   bool pdl;
 };
 bool attention_rows_applicable(const vvs_model_desc& md, int t_len);

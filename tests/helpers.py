@@ -123,11 +123,23 @@ class GpuRunner:
     """Owns a library context plus device copies of one case's weights."""
 
     def __init__(self, ms: ModelShape, w: dict, max_rows: int, max_block: int, max_nbr_k: int = 1,
-                 deterministic: bool = True):
+                 deterministic: bool = True, chain_kernels: bool = False):
+        """chain_kernels: create the context with the library's debug switch that selects the persistent
+        whole-chain kernels (and, for 33-64 tokens, the fused-epilogue projections) instead of the
+        per-projection kernels; the switch is read when the context is created."""
+        import os
         from paper_2511_13587_b200 import binding as vb
         self.vb = vb
         self.ms = ms
-        self.ctx = vb.vvs_create(vb.make_desc(ms, max_rows, max_block, max_nbr_k, deterministic))
+        old = os.environ.pop("VVS_DEBUG_CHAIN_KERNELS", None)
+        if chain_kernels:
+            os.environ["VVS_DEBUG_CHAIN_KERNELS"] = "1"
+        try:
+            self.ctx = vb.vvs_create(vb.make_desc(ms, max_rows, max_block, max_nbr_k, deterministic))
+        finally:
+            os.environ.pop("VVS_DEBUG_CHAIN_KERNELS", None)
+            if old is not None:
+                os.environ["VVS_DEBUG_CHAIN_KERNELS"] = old
         self.wd = weights_to_dev(w)
         vb.vvs_bind_weights(self.ctx, self.wd)
 

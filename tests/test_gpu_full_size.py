@@ -20,16 +20,17 @@ from vvs_synth.configs import B7, CONFIGS, MODE_RELAXED, XL
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("chain_kernels", [False, True])
 @pytest.mark.parametrize("deterministic", [True, False])
-def test_config1_full_llamagen_xl_shape(deterministic):
-    """Fill 477 needs four 128-key chunks per (sequence, head), i.e. more attention work items
-    than SMs, and the block's own rows straddle no chunk boundary; the small-shape tests cover
-    the other fills.  Both whole-chain kernels: fixed-order sums and arrival-order sums."""
+def test_config1_full_llamagen_xl_shape(deterministic, chain_kernels):
+    """Fill 477: eight 64-key blocks per (sequence, head) in the per-projection path; four 128-key
+    chunks per item, i.e. more attention work items than SMs, in the whole-chain kernels.  Fixed-order
+    and arrival-order sums on both generations of kernels."""
     wl, fill = CONFIGS[1], 477
     case = H.build_case(wl.shape, wl.seed + fill, 1, 2, 1, 8, [fill], cfg_scale=wl.cfg_scale, q_noise=0.3)
-    run = H.GpuRunner(wl.shape, case["w"], 2, 9, deterministic=deterministic)
+    run = H.GpuRunner(wl.shape, case["w"], 2, 9, deterministic=deterministic, chain_kernels=chain_kernels)
     gpu = run.verify(case)
-    assert gpu["launches"] < 40            # the whole-chain kernel ran, not one kernel per projection
+    assert (gpu["launches"] < 40) == chain_kernels      # one persistent kernel, or one kernel per projection
     ora = H.run_oracle(case)
     _check_end_to_end(case, gpu, ora)
     print("configs[1] full size: accept_len", gpu["accept_len"], "oracle", ora["accept_len"])
@@ -80,13 +81,14 @@ def test_config1_full_shape_candidate_tree():
     from test_gpu_tree import TREE_A, _check_tree
     wl, fill = CONFIGS[1], 477
     case = H.build_tree_case(wl.shape, wl.seed + 1, 1, 2, 1, TREE_A, [fill], cfg_scale=wl.cfg_scale, q_noise=0.3)
-    run = H.GpuRunner(wl.shape, case["w"], 2, 9)
-    gpu = H.run_tree_gpu(run, case)
-    assert gpu["launches"] < 40
     ora = H.run_tree_oracle(case)
-    _check_tree(case, gpu, ora)
-    print("configs[1] tree: accept path", gpu["accept_path"][0][:gpu["accept_len"][0]], "oracle", ora["accept_path"])
-    run.close()
+    for deterministic, chain_kernels in ((False, False), (True, False), (False, True)):
+        run = H.GpuRunner(wl.shape, case["w"], 2, 9, deterministic=deterministic, chain_kernels=chain_kernels)
+        gpu = H.run_tree_gpu(run, case)
+        assert (gpu["launches"] < 40) == chain_kernels
+        _check_tree(case, gpu, ora)
+        print("configs[1] tree: accept path", gpu["accept_path"][0][:gpu["accept_len"][0]], "oracle", ora["accept_path"])
+        run.close()
 
 
 @pytest.mark.parametrize("fill", [1, 583])
@@ -96,11 +98,13 @@ def test_config1_full_shape_cache_edges(fill):
     wl = CONFIGS[1]
     assert fill + 9 <= wl.shape.s_max
     case = H.build_case(wl.shape, wl.seed + fill, 1, 2, 1, 8, [fill], cfg_scale=wl.cfg_scale, q_noise=0.3)
-    run = H.GpuRunner(wl.shape, case["w"], 2, 9)
-    gpu = run.verify(case)
-    assert gpu["launches"] < 40
-    _check_end_to_end(case, gpu, H.run_oracle(case))
-    run.close()
+    ora = H.run_oracle(case)
+    for deterministic, chain_kernels in ((False, False), (True, False), (True, True), (False, True)):
+        run = H.GpuRunner(wl.shape, case["w"], 2, 9, deterministic=deterministic, chain_kernels=chain_kernels)
+        gpu = run.verify(case)
+        assert (gpu["launches"] < 40) == chain_kernels
+        _check_end_to_end(case, gpu, ora)
+        run.close()
 
 
 def test_config2_full_depth_batch16_relaxed():
@@ -123,8 +127,7 @@ def test_config2_full_depth_batch16_relaxed():
         run.close()
 
 
-@pytest.mark.parametrize("deterministic", [True, False])
-def test_config3_full_depth_7b(deterministic):
+def test_config3_full_depth_7b():
     """configs[3] as the benchmark runs it: 32 layers of the 7B shape (d = 4096, 32 heads of 128, MLP
     11008), 8192 codes inside a 65536-row head, fill 1500, one image with guidance, both whole-chain
     kernels.  The 13 GB of weights are drawn on the GPU (seeded) and copied to the host for the
@@ -151,18 +154,28 @@ def test_config3_full_depth_7b(deterministic):
           for _ in range(2)]
     case = H.build_case_independent(ms, wl.seed, 1, 2, 1, 8, [fill], cfg_scale=wl.cfg_scale, logit_std=1.0, w=w,
                                     kv=(bits(kv[0]), bits(kv[1])))
+    import os
     from paper_2511_13587_b200 import binding as vb
-    run = H.GpuRunner.__new__(H.GpuRunner)       # weights are on the device already: no second copy
-    run.vb, run.ms, run.wd = vb, ms, wd
-    run.ctx = vb.vvs_create(vb.make_desc(ms, 2, t_len, 1, deterministic))
-    vb.vvs_bind_weights(run.ctx, wd)
-    gpu = run.verify(case, kv_keep=fill + t_len)
-    assert gpu["launches"] < 40            # a whole-chain kernel
-    assert gpu["kv_rest_untouched"]        # slots beyond the block, compared on the device
     # the oracle only touches cache slots below fill + T: hand it that part (float64 copies of the
     # whole 2384-slot caches would be 10 GB)
     small = dict(case, kv_k=case["kv_k"][:, :, :, :fill + t_len], kv_v=case["kv_v"][:, :, :, :fill + t_len])
     ora = H.run_oracle(small)
-    _check_end_to_end(small, gpu, ora)
-    print("configs[3] full depth: accept_len", gpu["accept_len"].tolist(), "oracle", ora["accept_len"].tolist())
-    run.close()
+    # per-projection kernels with arrival-order and with fixed-order sums (what the benchmark times), then
+    # the two whole-chain kernels behind the library's debug switch
+    for deterministic, chain_kernels in ((False, False), (True, False), (False, True), (True, True)):
+        run = H.GpuRunner.__new__(H.GpuRunner)       # weights are on the device already: no second copy
+        run.vb, run.ms, run.wd = vb, ms, wd
+        if chain_kernels:
+            os.environ["VVS_DEBUG_CHAIN_KERNELS"] = "1"
+        try:
+            run.ctx = vb.vvs_create(vb.make_desc(ms, 2, t_len, 1, deterministic))
+        finally:
+            os.environ.pop("VVS_DEBUG_CHAIN_KERNELS", None)
+        vb.vvs_bind_weights(run.ctx, wd)
+        gpu = run.verify(case, kv_keep=fill + t_len)
+        assert (gpu["launches"] < 40) == chain_kernels
+        assert gpu["kv_rest_untouched"]        # slots beyond the block, compared on the device
+        _check_end_to_end(small, gpu, ora)
+        print("configs[3] full depth", (deterministic, chain_kernels), "accept_len", gpu["accept_len"].tolist(),
+              "oracle", ora["accept_len"].tolist())
+        run.close()

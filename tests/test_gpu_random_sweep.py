@@ -34,12 +34,12 @@ def test_random_chain_and_tree_calls(sweep_seed):
         if tree:
             parent = [-1] + list(range(f - 1)) + [int(rng.integers(f - 1, c)) for c in range(f, t_len)]
             case = H.build_tree_case(ms, seed, n_images, n_cfg, f, parent, fills, cfg_scale=cfg_scale, q_noise=q_noise)
-            run = H.GpuRunner(ms, case["w"], n_images * n_cfg, t_len)
+            run = H.GpuRunner(ms, case["w"], n_images * n_cfg, t_len, deterministic=bool(i & 1), chain_kernels=bool(i & 2))
             gpu = H.run_tree_gpu(run, case)
             _check_tree(case, gpu, H.run_tree_oracle(case))
         else:
             case = H.build_case(ms, seed, n_images, n_cfg, f, k, fills, cfg_scale=cfg_scale, q_noise=q_noise)
-            run = H.GpuRunner(ms, case["w"], n_images * n_cfg, t_len)
+            run = H.GpuRunner(ms, case["w"], n_images * n_cfg, t_len, deterministic=bool(i & 1), chain_kernels=bool(i & 2))
             gpu = run.verify(case)
             _check_end_to_end(case, gpu, H.run_oracle(case))
         run.close()
