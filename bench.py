@@ -28,15 +28,12 @@ sys.path.insert(0, ROOT)
 from vvs_synth import gen, philox  # noqa: E402
 from vvs_synth.configs import CONFIGS, MODE_RELAXED  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the whole-chain kernel, from the ncu
-# captures summarised under profiles/.  Keyed by (workload, fixed-order sums); each entry names the
-# kernel's source file and the first 16 hex digits of that file's SHA-256 when the counters were
-# taken: the line reports null once the file has changed since.
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE STEP (all launches of a verify call), summed over an
+# ncu capture summarised under profiles/.  Keyed by (workload, fixed-order sums); each entry names the
+# kernel sources the step runs and the first 16 hex digits of the SHA-256 over their concatenation when
+# the counters were taken: the line reports null, and says why, once any of them has changed.
+STEP_SOURCES = ("gemm_tc.cu", "attention_rows.cu", "kernels_generic.cu", "lmhead_tc.cu", "kernels_decide.cu")
 NCU_CAPTURES = {
-    (1, False): ("paper_2511_13587_b200/csrc/fused_chain.cu", "76919ebd16cc78e6", 1.4800e9,
-                 "profiles/fused_chain_kernel_configs1_ncu_full.txt"),
-    (1, True): ("paper_2511_13587_b200/csrc/chain_stream.cu", "59094e79f0fee11d", 1.4597e9,
-                "profiles/chain_stream_kernel_configs1_ncu_full.txt"),
 }
 N_TRIALS = 32           # distinct (fill, block, draft) inputs cycled through the steps
 DRAFT_LOGIT_STD = 1.0   # target-independent drafter: q = softmax(N(0, std^2))
@@ -67,16 +64,22 @@ def aggregate_value(world: int, drafts_per_step: float, steps: int, ms_total: fl
     return world * drafts_per_step * steps / (ms_total * 1e-3)
 
 
-def ncu_traffic(index: int, deterministic: bool, chain: bool):
-    """(bytes per launch, where they come from) for the dominant kernel, or (None, reason)."""
+def sources_hash() -> str:
+    h = hashlib.sha256()
+    for name in STEP_SOURCES:
+        with open(os.path.join(ROOT, "paper_2511_13587_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(index: int, deterministic: bool, chain_kernels: bool):
+    """(DRAM bytes of one step, where they come from), or (None, reason)."""
     e = NCU_CAPTURES.get((index, deterministic))
-    if not chain or e is None:
-        return None, "no ncu capture of this kernel and workload under profiles/"
-    src, sha, nbytes, summary = e
-    with open(os.path.join(ROOT, src), "rb") as fh:
-        cur = hashlib.sha256(fh.read()).hexdigest()[:16]
-    if cur != sha:
-        return None, f"{summary} is stale: {src} has changed since the capture"
+    if chain_kernels or e is None:
+        return None, "no ncu capture of this configuration under profiles/"
+    sha, nbytes, summary = e
+    if sources_hash() != sha:
+        return None, f"{summary} is stale: a kernel source has changed since the capture"
     return nbytes, summary
 
 
@@ -172,7 +175,7 @@ class VerifyBench:
     seeded trials and the step function that the timed regions repeat."""
 
     def __init__(self, index: int, rank: int = 0, deterministic: bool = False, n_trials: int = N_TRIALS,
-                 draft: str = "target"):
+                 draft: str = "target", chain_kernels: bool = False):
         import torch
         from paper_2511_13587_b200 import binding as vb
         from vvs_synth.configs import DTYPE_BF16
@@ -219,7 +222,15 @@ class VerifyBench:
         if index != 0 and draft == "target":
             self.kv0_k, self.kv0_v = self.kv_k.clone(), self.kv_v.clone()
         self.wd = wd
-        self.ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, wl.nbr_k, deterministic=deterministic))
+        # chain_kernels: the library's debug switch (read at context creation) that selects the persistent
+        # whole-chain kernels of the previous generation for calls of at most 32 tokens
+        os.environ.pop("VVS_DEBUG_CHAIN_KERNELS", None)
+        if chain_kernels:
+            os.environ["VVS_DEBUG_CHAIN_KERNELS"] = "1"
+        try:
+            self.ctx = vb.vvs_create(vb.make_desc(ms, r, t_len, wl.nbr_k, deterministic=deterministic))
+        finally:
+            os.environ.pop("VVS_DEBUG_CHAIN_KERNELS", None)
         vb.vvs_bind_weights(self.ctx, wd)
         if self.relaxed:
             rp, col = gen.neighbour_csr(gen.make_codebook(seed, ms.vocab, wl.latent_dim), wl.nbr_k)
@@ -366,8 +377,10 @@ class VerifyBench:
             dom_bytes = alg["total"] - ms.vocab * ms.d_model * 2
             dom_launches = cls_n[3] / n_prof
         else:
-            # wider calls: a launch per projection / attention / element-wise stage; no single kernel
-            # dominates, so the object describes the whole step (all launches of one verify call)
+            # a launch per projection / attention / element-wise stage, each overlapping its programmatic
+            # dependents: no single kernel dominates, so the object describes the whole step (all launches
+            # of one verify call).  The class times below are taken with events BETWEEN the launches, which
+            # removes that overlap: they add up to more than the step and only rank the classes.
             name = "whole step (per-projection GEMM, attention and element-wise launches together)"
             dom_ms, dom_bytes, dom_launches = ms_step, alg["total"], sum(cls_n) / n_prof
         achieved = dom_bytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
@@ -417,7 +430,8 @@ def run_ours(args) -> None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    S = VerifyBench(args.workload, rank, bool(args.deterministic), n_trials=args.trials, draft=args.draft)
+    S = VerifyBench(args.workload, rank, bool(args.deterministic), n_trials=args.trials, draft=args.draft,
+                    chain_kernels=args.chain_kernels)
     wl, ms, vb = S.wl, S.ms, S.vb
     warm = max(args.warmup, 3)
 
@@ -489,7 +503,7 @@ def run_ours(args) -> None:
     alg = algorithmic_bytes(wl, S.trials)
     ms_step = ms_region / args.steps
     roof = S.roofline(cls_ms, cls_n, n_prof, pk, ms_step)
-    roof["traffic"], roof["traffic_source"] = ncu_traffic(args.workload, bool(args.deterministic), cls_n[3] > 0)
+    roof["traffic"], roof["traffic_source"] = ncu_traffic(args.workload, bool(args.deterministic), args.chain_kernels)
     b, cfg, k, t_len = S.b, S.cfg, S.k, S.t_len
     line = {
         "metric": metric_name(wl),
@@ -505,6 +519,8 @@ def run_ours(args) -> None:
                    "n_draft": k, "block_rows": t_len, "fill": f"U[{wl.fill_lo},{wl.fill_hi}] per trial",
                    "trials": len(S.trials), "draft": S.drafter,
                    "sums": "fixed order (bitwise repeatable)" if args.deterministic else "arrival order (split-K adds in L2)",
+                   "kernels": "whole-chain kernels (previous generation, debug switch)" if args.chain_kernels
+                              else "per-projection kernels",
                    "timing": "median over `repeats` regions of `steps` steps each, every region bracketed by barrier + synchronize",
                    "l2": f"weights streamed per step ({alg['weights'] / 1e9:.2f} GB) exceed the 126 MB L2; no flush needed"
                          if alg["weights"] > 126e6 else "weights fit in L2: a latency case, not a bandwidth case",
@@ -529,11 +545,12 @@ def run_ours(args) -> None:
         dist.destroy_process_group()
 
 
-def quick_measure(index: int, deterministic: bool, steps: int, pk: dict, min_ms: float = 300.0) -> dict:
+def quick_measure(index: int, deterministic: bool, steps: int, pk: dict, min_ms: float = 300.0,
+                  chain_kernels: bool = False) -> dict:
     """A short device-resident measurement of one workload (one GPU): median step time over
     repeated regions, the step's algorithmic bytes and roofline fraction, acceptance statistics."""
     import torch
-    S = VerifyBench(index, 0, deterministic, n_trials=16)
+    S = VerifyBench(index, 0, deterministic, n_trials=16, chain_kernels=chain_kernels)
     for i in range(3):
         S.step(S.dtr[i % len(S.dtr)])
     torch.cuda.synchronize()
@@ -548,6 +565,7 @@ def quick_measure(index: int, deterministic: bool, steps: int, pk: dict, min_ms:
     res = {"workload": f"configs[{index}] {S.wl.name}", "ms_per_step": ms_step, "steps": steps, "repeats": len(regions),
            "drafts_per_s": S.drafts_per_step(steps) / (ms_step * 1e-3), "launches_per_step": launches,
            "sums": "fixed order" if deterministic else "arrival order",
+           "kernels": "whole-chain (previous generation)" if chain_kernels else "per-projection",
            "algorithmic_bytes": alg["total"], "step_frac_of_measured_hbm": alg["total"] / (ms_step * 1e-3) / 1e9 / pk["hbm_gbs"],
            "roofline": {n: roof[n] for n in ("kernel", "achieved", "frac", "ms_per_launch", "class_ms_per_step")},
            "acceptance": S.acceptance(), "device_status": S.vb.vvs_device_status(S.ctx)}
@@ -558,6 +576,8 @@ def quick_measure(index: int, deterministic: bool, steps: int, pk: dict, min_ms:
 def other_workloads(args, pk: dict) -> dict:
     """The workloads beside the headline one, each measured briefly on this GPU."""
     out = {"configs[1] fixed-order sums": quick_measure(1, True, 64, pk),
+           "configs[1] whole-chain kernel, arrival-order sums": quick_measure(1, False, 64, pk, chain_kernels=True),
+           "configs[1] whole-chain kernel, fixed-order sums": quick_measure(1, True, 64, pk, chain_kernels=True),
            "configs[0]": quick_measure(0, False, 256, pk, min_ms=100.0),
            "configs[2]": quick_measure(2, False, 16, pk),
            "configs[2] fixed-order sums": quick_measure(2, True, 16, pk),
@@ -909,6 +929,9 @@ def main() -> None:
     ap.add_argument("--workload", type=int, default=1, choices=[0, 1, 2, 3, 4, 5, 6])
     ap.add_argument("--deterministic", type=int, default=0, choices=[0, 1],
                     help="1: fixed-order sums (bitwise repeatable), 0: arrival-order split-K sums (faster)")
+    ap.add_argument("--chain-kernels", action="store_true",
+                    help="time the persistent whole-chain kernels of the previous generation (calls of at most 32 "
+                         "tokens) instead of the per-projection kernels")
     ap.add_argument("--cpu-steps", type=int, default=2)   # 5-16 s of host time at configs[1], depending on the host
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--min-ms", type=float, default=500.0,

@@ -101,17 +101,14 @@ typedef struct vvs_model_desc {
   int32_t deterministic; /* bf16 contexts:
                             1 = every sum of the decoder is taken in a fixed order, so the same call
                                 gives the same bits every time (target_probs, hidden, the appended
-                                K / V rows and hence next_token); vvs_bind_weights then keeps a private
-                                re-packed copy of the layer weights (as many bytes again, device memory);
-                            0 = split-K partial sums are added in L2 in arrival order: faster (see
-                                the measured numbers in the repository's notes), the last bits of the
-                                logits differ from run to run, and a residual sample over many nearly
-                                equally likely codes need not repeat.
-                            With 1, calls of at most 32 block tokens (n_images * n_cfg * T) run the
-                            streaming whole-chain kernel; larger calls split each projection's K range
-                            over a thread-block cluster that adds its partial tiles in rank order through
-                            distributed shared memory (about a quarter slower than the arrival-order
-                            reductions).  float32 contexts are always repeatable. */
+                                K / V rows and hence next_token): the K splits of a projection tile
+                                form a thread-block cluster that adds its partial tiles in rank order
+                                through distributed shared memory, each output written by one thread;
+                            0 = split-K partial sums are added in L2 in arrival order: faster (a
+                                quarter to a third per step; measured numbers in the repository's
+                                notes), the last bits of the logits differ from run to run, and a
+                                residual sample over many nearly equally likely codes need not repeat.
+                            float32 contexts are always repeatable. */
 } vvs_model_desc;
 
 /* Per-layer weights, device, type T.  Projection matrices are [out_features, in_features]
@@ -143,10 +140,10 @@ int vvs_destroy(vvs_ctx* ctx);
 /* Scratch bytes vvs_create will allocate for this description (host computation only). */
 int vvs_workspace_bytes(const vvs_model_desc* desc, size_t* out_bytes);
 
-/* Bind caller-owned weights.  Checks non-NULL and 16-byte alignment (VVS_ERR_ALIGN).  Contexts
- * created with deterministic = 1 also build their re-packed copy of the layer weights here (a
- * device allocation of the layers' size and a one-time packing kernel; synchronises the device);
- * the caller's layer weights are still read by calls of more than 32 block tokens. */
+/* Bind caller-owned weights.  Checks non-NULL and 16-byte alignment (VVS_ERR_ALIGN).  Nothing is
+ * copied: the weights must stay valid and unchanged while the context uses them.  (Only under the
+ * debug switch VVS_DEBUG_CHAIN_KERNELS, read by vvs_create, a fixed-order context also builds a
+ * re-packed device copy of the layer weights here for its streaming whole-chain kernel.) */
 int vvs_bind_weights(vvs_ctx* ctx, const vvs_weights* w);
 
 /* Bind the latent-space neighbour table used by relaxed acceptance (Sec. 2, LANTERN rule):

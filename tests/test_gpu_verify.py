@@ -51,10 +51,17 @@ def _check_end_to_end(case, gpu, ora):
     # 2e-3 absolute, except where a single probability is so large (the 7B-width head has logits
     # of std > 1) that its relative bound allows more
     assert (dp < np.maximum(tol["p_abs"], tol["p_rel"] * ora["target_probs"])).all()
-    # relative error (= guided-logit error) of every probability that is not negligible: at least a
-    # tenth of the uniform level 1 / V (the far tail of ~1e5 entries per call reaches any fixed sigma)
+    # guided-logit error of every probability that is not negligible (at least a tenth of the uniform
+    # level 1 / V; the far tail of ~1e5 entries per call reaches any fixed sigma), measured where it is
+    # exact, as |log(p / p_oracle)|, against the 5-sigma logit error of a row whose feature error is at
+    # the worst-row allowance of the feature check above
     notable = ora["target_probs"] >= 0.1 / ms.vocab
-    assert (dp[notable] / ora["target_probs"][notable]).max() < tol["p_rel"]
+    worst_row = 1.5 if h_err.size > 32 else 1.25
+    with np.errstate(divide="ignore"):
+        log_err = np.abs(np.log(gpu["target_probs"][notable] / ora["target_probs"][notable]))
+    print(f"largest guided-logit error {log_err.max():.3f} (bound {worst_row * tol['p_rel']:.3f}); "
+          f"feature error rms {np.sqrt(np.mean(h_err ** 2)):.4f}, worst row {h_err.max():.4f} (bound {tol['h_rel']:.4f})")
+    assert log_err.max() < worst_row * tol["p_rel"]
     np.testing.assert_allclose(gpu["target_probs"].sum(-1), 1.0, atol=1e-4)
     # appended K/V are compared per (layer, head, slot) row of head_dim elements: in a deep network
     # the error of such a short row scatters around the feature error, hence twice the bound there
