@@ -73,6 +73,11 @@ __device__ __forceinline__ void final_chunk(const KernelParams& p, int n, int to
       if (n < p.n) p.out[(size_t)tok * p.ldo + n] = v[j];
     } else if constexpr (EPI == GEMM_EPI_ADD) {
       if (n < p.n) atomicAdd(&p.out[(size_t)tok * p.ldo + n], v[j]);
+    } else if constexpr (EPI == GEMM_EPI_ADD2) {          // two matrices, sums added side by side: out[tok, n], out[tok, ff + n]
+      if (n < p.n) {
+        atomicAdd(&p.out[(size_t)tok * p.ldo + n], v[j]);
+        atomicAdd(&p.out[(size_t)tok * p.ldo + p.ff + n], v2[j]);
+      }
     } else if constexpr (EPI == GEMM_EPI_SWIGLU) {
       if (n < p.n) {
         const float g = v[j];
@@ -122,7 +127,7 @@ template <int EPI>
 __global__ void __launch_bounds__(128, 1)
 gemm_tc_kernel(const KernelParams p, const __grid_constant__ CUtensorMap tm_a,
                const __grid_constant__ CUtensorMap tm_a2, const __grid_constant__ CUtensorMap tm_b) {
-  constexpr bool DUAL = (EPI == GEMM_EPI_SWIGLU);
+  constexpr bool DUAL = (EPI == GEMM_EPI_SWIGLU || EPI == GEMM_EPI_ADD2);
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages];
   __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
@@ -245,7 +250,7 @@ gemm_tc_kernel(const KernelParams p, const __grid_constant__ CUtensorMap tm_a,
 
     const int n = tile * (int)kTileRows + warp * 32 + lane;  // weight row of this thread = TMEM lane
     const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
-    const bool fixup = (EPI != GEMM_EPI_ADD) && p.splits > 1;
+    const bool fixup = (EPI != GEMM_EPI_ADD && EPI != GEMM_EPI_ADD2) && p.splits > 1;
     bool do_final = true;
     if (fixup) {
       for (int c0 = 0; c0 < p.nt && tok0 + c0 < p.m; c0 += 16) {
@@ -543,7 +548,7 @@ GemmTcPlan plan_gemm_tc(int m, int n, int k, bool dual, bool allow_split, int n_
   int cps = 1;
   if (pl.passes > 1) {
     cps = 2;
-  } else if (allow_split && !dual) {
+  } else if (allow_split) {
     cps = (int)(218u * 1024u / (2u * stage_b));
     cps = cps > 5 ? 5 : cps < 1 ? 1 : cps;
     if (split_cap <= 8 && cps > 2) cps = 2;   // cluster reduction: fewer, longer CTAs (1.52 / 4.42 ms against 1.68 / 4.8 at five)
@@ -602,6 +607,7 @@ int launch_gemm_tc(int epi, const GemmTcPlan& plan, const GemmTcArgs& g, cudaStr
     case GEMM_EPI_ADD: e = launch_one<GEMM_EPI_ADD>(plan, kp, *g.tm_a, a2, *g.tm_b, plan.tiles, g.pdl, s); break;
     case GEMM_EPI_QKV: e = launch_one<GEMM_EPI_QKV>(plan, kp, *g.tm_a, a2, *g.tm_b, plan.tiles, g.pdl, s); break;
     case GEMM_EPI_SWIGLU: e = launch_one<GEMM_EPI_SWIGLU>(plan, kp, *g.tm_a, a2, *g.tm_b, plan.tiles, g.pdl, s); break;
+    case GEMM_EPI_ADD2: e = launch_one<GEMM_EPI_ADD2>(plan, kp, *g.tm_a, a2, *g.tm_b, plan.tiles, g.pdl, s); break;
     default: return VVS_ERR_INVALID_ARG;
   }
   return e == cudaSuccess ? VVS_OK : VVS_ERR_CUDA;

@@ -213,7 +213,7 @@ void launch_row_stats(const float* logits, float* part_m, float* part_s, int n_r
                       cudaStream_t s);
 
 // ---- tensor-core projection GEMM, gemm_tc.cu ----------------------------------------------------
-enum { GEMM_EPI_STORE = 0, GEMM_EPI_ADD = 1, GEMM_EPI_QKV = 2, GEMM_EPI_SWIGLU = 3 };
+enum { GEMM_EPI_STORE = 0, GEMM_EPI_ADD = 1, GEMM_EPI_QKV = 2, GEMM_EPI_SWIGLU = 3, GEMM_EPI_ADD2 = 4 };
 struct GemmTcPlan {
   int nt, passes, tiles, kb_total, splits, stages, smem_bytes, tmem_cols;
 };
