@@ -154,6 +154,55 @@ __global__ void __launch_bounds__(128) rmsnorm_rows_kernel(const float* __restri
   for (int i = lane * 4 + kKeep * 128; i < d; i += 128) emit(i, *reinterpret_cast<const float4*>(row + i));
 }
 
+// Few rows: one CTA of 128 threads per row (every thread holds at most kKeepB 16-byte pieces), so the
+// row's loads are all in flight at once and the kernel is two dependent memory round trips long.
+__global__ void __launch_bounds__(128) rmsnorm_row_block_kernel(const float* __restrict__ x,
+                                                                const __nv_bfloat16* __restrict__ scale,
+                                                                __nv_bfloat16* __restrict__ out, int d, float eps) {
+  constexpr int kKeepB = 8;            // d <= 4096
+  __shared__ float red[4];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  uint2 g[kKeepB];
+#pragma unroll
+  for (int u = 0; u < kKeepB; ++u) {                  // the scale is an input of the whole step: before the wait
+    const int i = tid * 4 + u * 512;
+    g[u] = i < d ? *reinterpret_cast<const uint2*>(scale + i) : make_uint2(0u, 0u);
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const float* row = x + (size_t)blockIdx.x * d;
+  float4 keep[kKeepB];
+  float ss = 0.f;
+#pragma unroll
+  for (int u = 0; u < kKeepB; ++u) {
+    const int i = tid * 4 + u * 512;
+    keep[u] = i < d ? *reinterpret_cast<const float4*>(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll
+  for (int u = 0; u < kKeepB; ++u)
+    ss += keep[u].x * keep[u].x + keep[u].y * keep[u].y + keep[u].z * keep[u].z + keep[u].w * keep[u].w;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if (lane == 0) red[warp] = ss;
+  __syncthreads();
+  const float rs = rsqrtf((red[0] + red[1] + red[2] + red[3]) / (float)d + eps);
+  __nv_bfloat16* o = out + (size_t)blockIdx.x * d;
+#pragma unroll
+  for (int u = 0; u < kKeepB; ++u) {
+    const int i = tid * 4 + u * 512;
+    if (i < d) {
+      const __nv_bfloat162 g0 = *reinterpret_cast<const __nv_bfloat162*>(&g[u].x);
+      const __nv_bfloat162 g1 = *reinterpret_cast<const __nv_bfloat162*>(&g[u].y);
+      __nv_bfloat162 r0 = __floats2bfloat162_rn(keep[u].x * rs * __bfloat162float(g0.x), keep[u].y * rs * __bfloat162float(g0.y));
+      __nv_bfloat162 r1 = __floats2bfloat162_rn(keep[u].z * rs * __bfloat162float(g1.x), keep[u].w * rs * __bfloat162float(g1.y));
+      uint2 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&r0);
+      pk.y = *reinterpret_cast<uint32_t*>(&r1);
+      *reinterpret_cast<uint2*>(o + i) = pk;
+    }
+  }
+}
+
 template <typename T>
 void launch_rmsnorm(const float* x, const T* scale, T* out, int m, int d, float eps, cudaStream_t s) {
   rmsnorm_kernel<T><<<m, 256, 0, s>>>(x, scale, out, d, eps);
@@ -174,6 +223,11 @@ static cudaError_t launch_dependent(const void* fn, dim3 grid, dim3 block, void*
 
 void launch_rmsnorm_rows(const float* x, const __nv_bfloat16* scale, __nv_bfloat16* out, int m, int d, float eps,
                          bool pdl, cudaStream_t s) {
+  if (m <= 64 && d <= 4096) {          // few rows: a CTA per row
+    void* args1[] = {&x, &scale, &out, &d, &eps};
+    launch_dependent(reinterpret_cast<const void*>(rmsnorm_row_block_kernel), dim3(m), dim3(128), args1, pdl, s);
+    return;
+  }
   void* args[] = {&x, &scale, &out, &m, &d, &eps};
   launch_dependent(reinterpret_cast<const void*>(rmsnorm_rows_kernel), dim3((m + 3) / 4), dim3(128), args, pdl, s);
 }
