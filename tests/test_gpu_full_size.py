@@ -46,6 +46,19 @@ def test_config1_full_llamagen_xl_shape(deterministic, chain_kernels):
     if deterministic:
         np.testing.assert_array_equal(gpu2["next_token"], gpu["next_token"])
         np.testing.assert_array_equal(gpu2["hidden"], gpu["hidden"])
+    else:
+        # the token of the call without probabilities, checked without them: on the residual row built
+        # from the CHECKED call's probabilities, the CDF interval of the returned code must contain the
+        # sample point u (two runs move a CDF over 16384 codes by far less than the 5e-3 allowed here)
+        k, f = case["n_draft_max"], case["n_forced"]
+        for b in range(case["n_images"]):
+            n = int(gpu2["accept_len"][b])
+            row = gpu["target_probs"][b][f - 1 + n].astype(np.float32)
+            r = np.maximum(np.float32(0), row - case["draft_probs"][b][n]) if n < k else row
+            cdf = np.cumsum(r.astype(np.float64)) / float(r.astype(np.float64).sum())
+            t = int(gpu2["next_token"][b]) - ms.vocab_offset
+            lo, hi, u = (cdf[t - 1] if t > 0 else 0.0), cdf[t], float(case["uniforms"][b][k])
+            assert lo - 5e-3 <= u <= hi + 5e-3, (b, t, lo, u, hi)
     run.close()
 
 
