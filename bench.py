@@ -404,17 +404,15 @@ def timed_regions(fn_region, steps: int, world: int, barrier, min_ms: float = 50
                   device="cuda"):
     """Repeats a `steps`-long timed region (each one bracketed by barrier + synchronize, its device
     time taken as the maximum over ranks) until at least `min_ms` of device time has been
-    measured.  Returns the list of region times (ms)."""
+    measured.  Every rank sees the same (all-reduced) region times, so all ranks stop after the
+    same region.  Returns the list of region times (ms)."""
     times = []
-    target = None
     while True:
         barrier()
         t = max_over_ranks([fn_region(steps)], world, device=device)[0]
         barrier()
         times.append(t)
-        if target is None:     # every rank derives the same repeat count from the same number
-            target = int(min(max_repeats, max(1, np.ceil(min_ms / max(t, 1e-3)))))
-        if len(times) >= target:
+        if sum(times) >= min_ms or len(times) >= max_repeats:
             return times
 
 

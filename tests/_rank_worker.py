@@ -28,8 +28,8 @@ def main() -> None:
     # the slowest rank decides the time of the whole job
     ms_total, ms_e2e = bench.max_over_ranks([10.0 + rank, 20.0 - rank], world)
     drafts = float(trial["n_draft"].sum())
-    # repeated timed regions: the rank-dependent region times must give every rank the same repeat
-    # count (it follows from the maximum over ranks of the first region), or the barriers deadlock
+    # repeated timed regions: the rank-dependent region times must make every rank stop after the same
+    # region (the stop rule sees only all-reduced times), or the barriers deadlock
     calls = []
 
     def region(steps):

@@ -32,8 +32,8 @@ def test_two_replicas_draw_their_own_inputs_and_share_the_slowest_time(tmp_path)
     assert res["fills"][0] != res["fills"][1]                 # different seeds, different cache fills
     assert res["ms_total"] == 11.0 and res["ms_e2e"] == 20.0  # element-wise maximum over the ranks
     assert abs(res["value"] - 2 * res["drafts"] * 4 / 11e-3) < 1e-6
-    # ceil(500 / 71) = 8 regions of 4 steps, each timed as the slower rank's 70 + i
-    assert res["regions"] == [71.0 + i for i in range(8)] and res["region_calls"] == [4] * 8
+    # regions of 4 steps, each timed as the slower rank's 70 + i, until 500 ms are covered: 71 + ... + 77 = 518
+    assert res["regions"] == [71.0 + i for i in range(7)] and res["region_calls"] == [4] * 7
 
 
 def test_reference_arm_runs_on_rank_0_only(tmp_path):
