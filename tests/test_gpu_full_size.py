@@ -40,7 +40,10 @@ def test_config1_full_llamagen_xl_shape(deterministic, chain_kernels):
     # (margins far above that) must repeat, the residual sample over 16384 almost equally likely
     # codes need not and is only checked for range.
     gpu2 = run.verify(case, want_probs=False)
-    np.testing.assert_array_equal(gpu2["accept_len"], gpu["accept_len"])
+    clear = np.ones(case["n_images"], bool)
+    if not deterministic:       # a decision within the run-to-run distance of its threshold may flip
+        clear = (H.replay_decisions(case, gpu["target_probs"])["margins"][:, :case["n_draft_max"]] > 2e-2).all(axis=1)
+    np.testing.assert_array_equal(gpu2["accept_len"][clear], gpu["accept_len"][clear])
     ms = wl.shape
     assert ((gpu2["next_token"] >= ms.vocab_offset) & (gpu2["next_token"] < ms.vocab_offset + ms.vocab)).all()
     if deterministic:
@@ -54,6 +57,8 @@ def test_config1_full_llamagen_xl_shape(deterministic, chain_kernels):
         # differences are correlated over the codebook a CDF value moves by up to about 1e-2 (5.3e-3 seen)
         k, f = case["n_draft_max"], case["n_forced"]
         for b in range(case["n_images"]):
+            if not clear[b]:
+                continue
             n = int(gpu2["accept_len"][b])
             row = gpu["target_probs"][b][f - 1 + n].astype(np.float32)
             r = np.maximum(np.float32(0), row - case["draft_probs"][b][n]) if n < k else row

@@ -124,9 +124,15 @@ def test_xl_shape_small_bf16_cfg(n_images, fills, deterministic, chain_kernels):
     _check_end_to_end(case, gpu, ora)
     # outputs not requested are not needed for the decisions
     gpu2 = run.verify(case, want_probs=False, want_hidden=False)
-    np.testing.assert_array_equal(gpu2["accept_len"], gpu["accept_len"])
     if deterministic:
+        np.testing.assert_array_equal(gpu2["accept_len"], gpu["accept_len"])
         np.testing.assert_array_equal(gpu2["next_token"], gpu["next_token"])
+    else:
+        # two arrival-order calls differ in the last bits: a decision may flip only where the uniform
+        # sits within that distance of its ratio
+        m = H.replay_decisions(case, gpu["target_probs"])["margins"][:, :8]
+        clear = (m > 1e-2).all(axis=1)
+        np.testing.assert_array_equal(gpu2["accept_len"][clear], gpu["accept_len"][clear])
     run.close()
 
 
