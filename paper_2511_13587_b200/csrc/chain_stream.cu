@@ -1,6 +1,11 @@
 // The decoder chain of the verify step (embedding + every layer) as ONE persistent dataflow kernel
 // for calls of at most 32 block tokens (bf16).
 //
+// Status: previous generation.  The per-projection kernels (gemm_tc.cu, attention_rows.cu) with
+// programmatic dependent launch were measured faster at both benchmark shapes and are the default;
+// this kernel runs only in contexts created under the debug switch VVS_DEBUG_CHAIN_KERNELS with
+// fixed-order sums, and stays parity-tested.
+//
 // At this size the step is a chain of ~180 dependent small projections that together stream the
 // whole model once: the HBM stream and the latency of the dependency chain both matter.  Design:
 //
@@ -37,9 +42,7 @@
 //
 // Tensor cores: warp-level mma.sync on purpose.  At <= 32 tokens a tcgen05.mma (M = 128) issued by
 // one thread every ~68 cycles does no more work per cycle than the four sub-cores' warp MMAs, and
-// its TMEM round trip and operand staging sit on the critical path of every stage; the tcgen05
-// kernels of this library serve the calls with enough tokens to fill them (projection GEMMs above
-// 32 tokens, LM head).
+// its TMEM round trip and operand staging sit on the critical path of every stage.
 #include <math_constants.h>
 
 #include <algorithm>

@@ -1,5 +1,10 @@
 // The decoder chain of the verify step as ONE persistent kernel (bf16, at most 32 block tokens).
 //
+// Status: previous generation.  The per-projection kernels (gemm_tc.cu, attention_rows.cu) with
+// programmatic dependent launch were measured faster at both benchmark shapes and are the default;
+// this kernel runs only in contexts created under the debug switch VVS_DEBUG_CHAIN_KERNELS with
+// arrival-order sums, and stays parity-tested.
+//
 // A batch-1 verify step is a chain of ~180 dependent small projections: run as separate kernels
 // it is bound by launch, fill and drain latency, not by the weight stream.  Here one CTA per SM
 // stays resident for the whole chain and the work of every phase is cut into fixed shares:

@@ -9,10 +9,20 @@
 // activation tiles are staged by TMA into 128-byte-swizzled shared memory, one elected thread
 // issues the MMAs, accumulators live in TMEM, and the four warps read them back (tcgen05.ld) for
 // a fused epilogue:
-//   ADD     x[tok, n] += acc                       (output / down projection onto the residual)
-//   QKV     rotate q, k pairs, write q and append k, v to the KV cache
-//   SWIGLU  act[tok, n] = silu(gate) * up          (two weight tiles, two accumulators)
+//   ADD     out[tok, n] += acc                     (every projection of the default path: fp32 sums that
+//                                                   the next kernel rotates / gates / normalises)
+//   ADD2    the same for two weight matrices sharing the activation tile (gate and up as one launch)
+//   QKV     rotate q, k pairs, write q and append k, v to the KV cache      (debug-switch path, 33-64 tokens)
+//   SWIGLU  act[tok, n] = silu(gate) * up          (two weight tiles, two accumulators; same path)
 //   STORE   out[tok, n] = acc
+// How the split-K sums of ADD meet: (a) scalar reductions into L2 in arrival order (at most 32 tokens
+// per pass); (b) above that the accumulator tile is staged token-major in shared memory and every
+// thread adds four consecutive columns with one vector reduction; (c) in fixed-order contexts the
+// K splits of a tile are the CTAs of one thread-block cluster: each rank sums its share of the token
+// rows over all ranks' staged tiles in rank order through distributed shared memory and is the only
+// writer of those outputs (no atomics, repeatable bits).
+// Planning: two CTAs per SM when the tokens need several passes, up to five small CTAs (two stages
+// each) for a single pass: more independent weight streams per SM.
 // Split-K partial sums of the non-linear epilogues are added into a zeroed fp32 scratch; the CTA
 // that arrives last on the tile's counter applies the epilogue and re-zeroes what it read, so no
 // CTA ever waits for another.  Weight tiles are requested before griddepcontrol.wait, i.e. while
