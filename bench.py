@@ -661,19 +661,21 @@ SWEEP_POINTS = (
 )
 
 
-def epilogue_sweep(steps: int, pk: dict) -> dict:
+def epilogue_sweep(steps: int, pk: dict, only=None) -> dict:
     """Points of the acceptance-epilogue sweep through vvs_epilogue (LM head + guidance + softmax +
     decisions on given features), inputs drawn on the device.  Every point carries its time, the
     LM-head TFLOP/s (2 M d V over the whole call, which runs the LM head, the decision kernels and
     the one-row-per-image second pass), the bytes per second of the codebook stream, each as a
     fraction of the measured peak, and the measured acceptance rate.  The drafter row of a
-    position is softmax(log p + scale * Gumbel noise), p the library's own target row."""
+    position is softmax(log p + scale * Gumbel noise), p the library's own target row.  `only`
+    picks one point by its index (for a profiler capture of a single shape)."""
     import torch
     from paper_2511_13587_b200 import binding as vb
     from vvs_synth.configs import ModelShape
     points = []
     csr = {}
-    for d, v, b, k, c, mode, nbr_k, noise, temp in SWEEP_POINTS:
+    chosen = SWEEP_POINTS if only is None else SWEEP_POINTS[only:only + 1]
+    for d, v, b, k, c, mode, nbr_k, noise, temp in chosen:
         ms = ModelShape("epilogue", 0, d, 0, 0, 0, v)
         rows = k + 1
         ctx = vb.vvs_create(vb.make_desc(ms, b * c, rows, max(1, nbr_k)))
@@ -768,7 +770,7 @@ def run_epilogue_sweep(args) -> None:
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    print(json.dumps(epilogue_sweep(args.steps, peaks())))
+    print(json.dumps(epilogue_sweep(args.steps, peaks(), only=args.sweep_point)))
 
 
 # ---------------------------------------------------------------------------------------------
@@ -929,6 +931,8 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, choices=[0, 1, 2, 3, 4, 5, 6])
+    ap.add_argument("--sweep-point", type=int, default=None, choices=range(len(SWEEP_POINTS)),
+                    help="with --workload 4: run this one point of the sweep only")
     ap.add_argument("--deterministic", type=int, default=0, choices=[0, 1],
                     help="1: fixed-order sums (bitwise repeatable), 0: arrival-order split-K sums (faster)")
     ap.add_argument("--chain-kernels", action="store_true",

@@ -74,7 +74,7 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
-  const int tile0 = blockIdx.x * NM;
+  const int tile0 = blockIdx.y * NM;
   const int C = p.n_cfg;
   const uint32_t half_bytes = (uint32_t)p.nd_pad * kBlockK * 2u;     // one box of feature rows
   const uint32_t b_bytes = half_bytes * (uint32_t)C;
@@ -109,13 +109,17 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
   uint32_t it_p = 0, it_c = 0;
   bool alive = true;
 
-  for (int pass = 0; pass < p.passes && alive; ++pass) {
+  // The CTAs of one codebook tile sit next to each other on grid x and deal the passes among
+  // themselves: they stream the same weight rows at the same time, so all but one of them find
+  // those rows in L2, and the work comes in units of one pass instead of one whole tile.
+  int iter = 0;
+  for (int pass = blockIdx.x; pass < p.passes && alive; pass += gridDim.x, ++iter) {
     const int row0 = pass * 128;                                  // first decision row of the pass
     const int nd = p.bt - row0 < 128 ? p.bt - row0 : 128;
     if (warp == 0 && lane == 0) {
       // ---- TMA producer: weights may be requested before the features exist ------------------
       int kb = 0;
-      if (pass == 0) {
+      if (iter == 0) {
         const int n_pre = p.kb_total < p.stages ? p.kb_total : p.stages;
         for (int i = 0; i < n_pre; ++i) {
           mbar_expect_tx(&full_bar[i], stage_bytes);
@@ -176,7 +180,7 @@ lmhead_tc_kernel(const LmParams p, const __grid_constant__ CUtensorMap tm_a, con
     }
     __syncwarp();
     pdl_wait();
-    bool got = wait_or_abort(&acc_bar, pass & 1, &s_abort);
+    bool got = wait_or_abort(&acc_bar, iter & 1, &s_abort);
     if (!got) s_abort = 1;
     if (__syncthreads_or(got ? 0 : 1)) {
       if (tid == 0) atomicOr(p.status, VVS_DEV_TIMEOUT);
@@ -294,10 +298,16 @@ int launch_lmhead_tc(const LmHeadArgs& a, cudaStream_t s) {
   // two codebook tiles per CTA when 256-row tiles still give every SM a CTA (the feature tile is then
   // read once per 256 codes); the logit tile lies over the stages in that case
   const int n_sms_hint = 120;
-  const bool two = a.v >= 2 * (int)kTileRows * n_sms_hint && 2 * nt <= 512;
+  // (row mode streams the codebook once for a few feature rows: single tiles, and where the codebook
+  // has two of them for every SM, CTAs small enough to sit two to an SM, so that one CTA's fill and
+  // epilogue hide behind the other's stream)
+  const bool two = !a.row_mode && a.v >= 2 * (int)kTileRows * n_sms_hint && 2 * nt <= 512;
   const uint32_t stage_bytes = kATileBytes * (two ? 2u : 1u) + (uint32_t)nt * kBlockK * 2u;
   const size_t tile_bytes = a.row_mode ? 0 : (size_t)p.nd_pad * kTileLd * 4;
-  int stages = (int)((220 * 1024 - (two ? 0 : tile_bytes)) / stage_bytes);
+  const int n_sms = a.n_sms > 0 ? a.n_sms : 148;
+  const bool small_ctas = a.row_mode && nt <= 256 && (a.v + 127) / 128 >= 2 * n_sms;
+  const size_t smem_budget = small_ctas ? 108 * 1024 : 220 * 1024;
+  int stages = (int)((smem_budget - (two ? 0 : tile_bytes)) / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages > p.kb_total) stages = p.kb_total;
   if (stages < 1) return VVS_ERR_SHAPE;
@@ -313,7 +323,16 @@ int launch_lmhead_tc(const LmHeadArgs& a, cudaStream_t s) {
   if (ensure_dynamic_smem(fn, 226 * 1024) != cudaSuccess) return VVS_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   const int rows_per_cta = (int)kTileRows * (two ? 2 : 1);
-  cfg.gridDim = dim3((a.v + rows_per_cta - 1) / rows_per_cta, 1, 1);
+  const int tiles = (a.v + rows_per_cta - 1) / rows_per_cta;
+  // CTAs per codebook tile: the count that needs the fewest rounds of (one pass on every SM); the
+  // smaller count on a tie (fewer pipeline fills)
+  int share = 1;
+  long best = -1;
+  for (int g = 1; g <= p.passes; ++g) {
+    const long rounds = (long)((tiles * g + n_sms - 1) / n_sms) * ((p.passes + g - 1) / g);
+    if (best < 0 || rounds < best) { best = rounds; share = g; }
+  }
+  cfg.gridDim = dim3(share, tiles, 1);
   cfg.blockDim = dim3(128, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;

@@ -180,7 +180,7 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
       return VVS_ERR_CUDA;
     LmHeadArgs la{};
     la.v = V; la.k = md.d_model; la.bt = BT; la.n_cfg = C; la.tm_a = &ctx->lm_map; la.tm_b = &tm_hid;
-    la.pdl = ctx->use_pdl; la.cfg_scale = a->cfg_scale; la.inv_temp = 1.f / a->temperature;
+    la.pdl = ctx->use_pdl; la.n_sms = ctx->n_sms; la.cfg_scale = a->cfg_scale; la.inv_temp = 1.f / a->temperature;
     // few decision rows: the guided logits are written out (under a megabyte at 9 rows) and the
     // sampled row is read back from them; otherwise a second pass over the head recomputes it
     float* lbuf = o->target_probs ? o->target_probs : (BT <= 64 ? ws.logits_small : nullptr);
@@ -206,7 +206,7 @@ int run_decisions(vvs_ctx* ctx, const T* hid, int rows_per_seq, int first_row, c
     VVS_LAUNCH(VVS_PROF_OTHER, launch_gather_sel_rows(hid, ws.sel_row, ws.sel_hid, B, C, BT, md.d_model, s));
     LmHeadArgs lr{};
     lr.v = V; lr.k = md.d_model; lr.bt = B; lr.n_cfg = C; lr.tm_a = &ctx->lm_map; lr.tm_b = &tm_sel;
-    lr.pdl = ctx->use_pdl; lr.cfg_scale = a->cfg_scale; lr.inv_temp = 1.f / a->temperature; lr.status = ws.status;
+    lr.pdl = ctx->use_pdl; lr.n_sms = ctx->n_sms; lr.cfg_scale = a->cfg_scale; lr.inv_temp = 1.f / a->temperature; lr.status = ws.status;
     lr.row_mode = 1; lr.sel_row = ws.sel_row; lr.stat_m = ws.stat_m; lr.stat_inv = ws.stat_inv; lr.p_row = ws.p_row;
     VVS_LAUNCH(VVS_PROF_GEMM, rc = launch_lmhead_tc(lr, s));
     if (rc != VVS_OK) return rc;
@@ -283,7 +283,7 @@ int run_tree_decisions(vvs_ctx* ctx, const __nv_bfloat16* hid, const vvs_verify_
     return VVS_ERR_CUDA;
   LmHeadArgs la{};
   la.v = V; la.k = md.d_model; la.bt = BT; la.n_cfg = C; la.tm_a = &ctx->lm_map; la.tm_b = &tm_hid;
-  la.pdl = ctx->use_pdl; la.cfg_scale = a->cfg_scale; la.inv_temp = 1.f / a->temperature;
+  la.pdl = ctx->use_pdl; la.n_sms = ctx->n_sms; la.cfg_scale = a->cfg_scale; la.inv_temp = 1.f / a->temperature;
   la.part_m = ws.part_m; la.part_s = ws.part_s; la.logits_out = o->target_probs; la.status = ws.status;
   la.rows_per_seq = Tn; la.first_row = a->n_forced - 1; la.n_draft_max = 0;
   la.vocab_offset = md.vocab_offset; la.relaxed = 0; la.nbr_k = 1; la.kmax = md.max_nbr_k; la.drafts_ld = Tn;

@@ -279,6 +279,7 @@ struct LmHeadArgs {
   const CUtensorMap* tm_a;       // codebook rows of w_lm [v, k]
   const CUtensorMap* tm_b;       // features [n_cfg * bt, k] (cond rows, then uncond rows), box rows = lmhead_box_rows(bt)
   bool pdl;
+  int n_sms;                     // SMs of the device (0: 148)
   float cfg_scale, inv_temp;
   float* part_m; float* part_s;  // [n_tiles, bt] softmax partials per 128-code tile
   float* logits_out;             // optional [bt, v] guided logits
