@@ -34,10 +34,10 @@ from vvs_synth.configs import CONFIGS, MODE_RELAXED  # noqa: E402
 # the counters were taken: the line reports null, and says why, once any of them has changed.
 STEP_SOURCES = ("gemm_tc.cu", "attention_rows.cu", "kernels_generic.cu", "lmhead_tc.cu", "kernels_decide.cu")
 NCU_CAPTURES = {
-    (1, False): ("1a33dec3f0789e8f", 1.5709e+09, "profiles/verify_step_configs1_per_projection_launch_list_and_counters.txt"),
-    (1, True): ("1a33dec3f0789e8f", 1.5459e+09, "profiles/verify_step_configs1_per_projection_launch_list_and_counters.txt"),
-    (2, False): ("1a33dec3f0789e8f", 4.4630e+09, "profiles/verify_step_configs2_launch_list_and_counters.txt"),
-    (2, True): ("1a33dec3f0789e8f", 4.0170e+09, "profiles/verify_step_configs2_launch_list_and_counters.txt"),
+    (1, False): ("1748279beacd934c", 1.5709e+09, "profiles/verify_step_configs1_per_projection_launch_list_and_counters.txt"),
+    (1, True): ("1748279beacd934c", 1.5459e+09, "profiles/verify_step_configs1_per_projection_launch_list_and_counters.txt"),
+    (2, False): ("1748279beacd934c", 4.4629e+09, "profiles/verify_step_configs2_launch_list_and_counters.txt"),
+    (2, True): ("1748279beacd934c", 4.0170e+09, "profiles/verify_step_configs2_launch_list_and_counters.txt"),
 }
 N_TRIALS = 32           # distinct (fill, block, draft) inputs cycled through the steps
 DRAFT_LOGIT_STD = 1.0   # target-independent drafter: q = softmax(N(0, std^2))
