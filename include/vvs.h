@@ -80,7 +80,8 @@ typedef struct vvs_model_desc {
   int32_t n_heads;
   int32_t head_dim;      /* 64 or 128 */
   int32_t d_ff;          /* SwiGLU inner width */
-  int32_t vocab;         /* V: size of the image codebook = number of logits per position */
+  int32_t vocab;         /* V: size of the image codebook = number of logits per position;
+                            at most 65535 * 128 (VVS_ERR_SHAPE beyond) */
   int32_t vocab_offset;  /* first row of the image codebook inside w_lm and the id space */
   int32_t lm_rows;       /* rows of w_lm (>= vocab_offset + vocab) */
   int32_t tok_rows;      /* rows of tok_emb */

@@ -103,6 +103,7 @@ int check_desc(const vvs_model_desc* d) {
   if (d->rope_mode < VVS_ROPE_NONE || d->rope_mode > VVS_ROPE_2D_GRID) return VVS_ERR_INVALID_ARG;
   if (d->n_layers < 0 || d->d_model <= 0 || d->vocab <= 0 || d->vocab_offset < 0) return VVS_ERR_SHAPE;
   if (d->lm_rows < d->vocab_offset + d->vocab) return VVS_ERR_SHAPE;
+  if (d->vocab > 65535 * 128) return VVS_ERR_SHAPE;      // the LM head puts one 128-code tile on each grid row
   if (d->d_model % 8) return VVS_ERR_SHAPE;
   if (d->max_rows < 1 || d->max_block < 1 || d->max_block > 32 || d->max_nbr_k < 1) return VVS_ERR_SHAPE;
   if (d->n_layers > 0) {

@@ -49,6 +49,10 @@ def test_host_side_argument_errors_need_no_gpu():
     d = vb.make_desc(TINY, 1, 5)
     d.n_heads = 3
     assert vb.lib.vvs_workspace_bytes(ctypes.byref(d), ctypes.byref(out)) == -2
+    d = vb.make_desc(TINY, 1, 5)
+    d.vocab = 65535 * 128 + 1                   # beyond the LM head's grid
+    d.lm_rows = d.vocab_offset + d.vocab
+    assert vb.lib.vvs_workspace_bytes(ctypes.byref(d), ctypes.byref(out)) == -2
     assert vb.lib.vvs_workspace_bytes(None, ctypes.byref(out)) == -1
     assert vb.lib.vvs_verify(None, None, None, None) == -1
     assert vb.lib.vvs_destroy(None) == -1
